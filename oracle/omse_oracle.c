@@ -1,0 +1,328 @@
+/*
+ * CPU oracle for the constrained-MMSE quantization path of "Low-bit Quantization of
+ * Neural Networks for Efficient Inference" (Choukroun et al., arXiv:1902.06822).
+ *
+ * THIS FILE IS TEST INFRASTRUCTURE.  It is a plain, slow, one-element-at-a-time
+ * restatement of what the method computes, written so that it can be checked against
+ * the paper by eye.  The CUDA library shares no code with it and never calls it; only
+ * the tests, the smoke check and the benchmark's CPU-baseline leg may load it.
+ *
+ * Everything is evaluated in the order the paper states it, with no blocking, fusion
+ * or reordering.  Decisions that produce an integer (the codes) are taken in IEEE
+ * binary32 exactly as Section 3.1 writes them (divide, round to nearest, saturate);
+ * every sum is accumulated in binary64.
+ *
+ * Parity pins (tests marked "not gpu"): exact piecewise-quadratic optimum by breakpoint
+ * enumeration on tiny tensors, hand-worked examples, on-grid inputs, the no-offset
+ * uniform quantizer of Section 3.1, invariants of Sections 3.4/3.5, pack round trip.
+ * No function in this file is "parity unpinned".
+ *
+ * The optional OpenMP pragmas only distribute independent kernels (rows) or independent
+ * candidates over threads; each row / candidate is still computed serially.
+ */
+#include <float.h>
+#include <math.h>
+#include <stddef.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* status bits reported per call (data-dependent conditions, never an error) */
+#define ORACLE_STATUS_NONFINITE 1u /* a NaN or Inf was seen in the input            */
+#define ORACLE_STATUS_DEGENERATE 2u /* a segment had no usable scale (all zero/tiny) */
+
+int omse_oracle_max_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* Section 3.1: the quantization range Z_p.  Unsigned {0..2^p-1}; signed {-2^(p-1)..2^(p-1)-1}. */
+void omse_oracle_grid_bounds(int bits, int is_signed, int *lo, int *hi)
+{
+    if (is_signed) {
+        *lo = -(1 << (bits - 1));
+        *hi = (1 << (bits - 1)) - 1;
+    } else {
+        *lo = 0;
+        *hi = (1 << bits) - 1;
+    }
+}
+
+/* Section 3.1, operator [.]_Zp applied to T_i/alpha (Section 3.4, optimal codes given alpha):
+ * binary32 division, round to nearest (ties to even: the default IEEE mode), then saturate. */
+static int code_of(float x, float alpha, int lo, int hi)
+{
+    float r = rintf(x / alpha);
+    if (r < (float)lo) r = (float)lo;
+    if (r > (float)hi) r = (float)hi;
+    if (r != r) r = 0.0f; /* NaN input: any in-range code */
+    return (int)r;
+}
+
+/* Section 3.4, objective ||T - alpha*T~||_F^2 for the codes that alpha implies. */
+static double sse_of(const float *x, int64_t k, float alpha, int lo, int hi)
+{
+    double s = 0.0;
+    for (int64_t i = 0; i < k; ++i) {
+        double d = (double)x[i] - (double)alpha * (double)code_of(x[i], alpha, lo, hi);
+        s += d * d;
+    }
+    return s;
+}
+
+double omse_oracle_sse_at(const float *x, int64_t k, float alpha, int bits, int is_signed)
+{
+    int lo, hi;
+    omse_oracle_grid_bounds(bits, is_signed, &lo, &hi);
+    return sse_of(x, k, alpha, lo, hi);
+}
+
+void omse_oracle_codes(const float *x, int64_t n, float alpha, int bits, int is_signed, int8_t *codes)
+{
+    int lo, hi;
+    omse_oracle_grid_bounds(bits, is_signed, &lo, &hi);
+    for (int64_t i = 0; i < n; ++i)
+        codes[i] = (alpha > 0.0f) ? (int8_t)code_of(x[i], alpha, lo, hi) : (int8_t)0;
+}
+
+/* The candidate scales of the line search (Section 3.4: "a given grid"): C points spaced
+ * linearly in (0, hi_frac*max|x|], every operation in binary32. */
+float omse_oracle_candidate(float max_abs, float hi_frac, int n_cand, int c)
+{
+    float a_hi = hi_frac * max_abs;
+    float step = a_hi / (float)n_cand;
+    return (float)(c + 1) * step;
+}
+
+static float max_abs_of(const float *x, int64_t k, uint32_t *status)
+{
+    float m = 0.0f;
+    for (int64_t i = 0; i < k; ++i) {
+        float a = fabsf(x[i]);
+        if (!(a <= FLT_MAX)) *status |= ORACLE_STATUS_NONFINITE;
+        if (a > m) m = a;
+    }
+    return m;
+}
+
+/* Closed-form scale for fixed codes (least squares of the Section 3.4 objective in alpha),
+ * alternated with re-quantization as in the alternating scheme the paper cites; applied
+ * `iters` times starting from `alpha`. */
+static float refine_from(const float *x, int64_t k, float alpha, int lo, int hi, int iters)
+{
+    for (int it = 0; it < iters; ++it) {
+        int64_t sqq = 0;
+        double sxq = 0.0;
+        for (int64_t i = 0; i < k; ++i) {
+            int q = code_of(x[i], alpha, lo, hi);
+            sqq += (int64_t)q * q;
+            sxq += (double)x[i] * (double)q;
+        }
+        if (sqq == 0) break;
+        float a_new = (float)(sxq / (double)sqq);
+        if (!(a_new >= FLT_MIN) || !(a_new <= FLT_MAX)) break;
+        alpha = a_new;
+    }
+    return alpha;
+}
+
+/*
+ * The quantization mapping phi(T, p) of Section 3.4 on one segment x[0..k):
+ *   grid line search over n_cand scales, lowest index on ties, then `refine_iters`
+ *   closed-form polish steps, then the final codes and squared error.
+ * start_idx < 0: run the search.  start_idx >= 0: skip the search and start the polish
+ *   from that candidate (used by the harness when two candidates tie).
+ * Outputs: *alpha, *sse (binary64), *best_idx (-1 for a degenerate segment),
+ *   codes[k] (nullable), sse_curve[n_cand] (nullable; +inf for unusable candidates).
+ * Degenerate segment (max|x| == 0, or every candidate below FLT_MIN): alpha = 0,
+ *   all codes 0, sse = sum x^2, best_idx = -1.
+ */
+void omse_oracle_phi(const float *x, int64_t k, int bits, int is_signed, int n_cand, float hi_frac,
+                     int refine_iters, int start_idx, float *alpha, double *sse, int32_t *best_idx,
+                     int8_t *codes, double *sse_curve, uint32_t *status)
+{
+    int lo, hi;
+    uint32_t st = 0;
+    omse_oracle_grid_bounds(bits, is_signed, &lo, &hi);
+    float m = max_abs_of(x, k, &st);
+
+    int best = -1;
+    double best_sse = INFINITY;
+    if (start_idx >= 0) {
+        best = start_idx;
+        best_sse = 0.0;
+        if (!(omse_oracle_candidate(m, hi_frac, n_cand, best) >= FLT_MIN)) best = -1;
+    } else {
+        for (int c = 0; c < n_cand; ++c) {
+            float a = omse_oracle_candidate(m, hi_frac, n_cand, c);
+            double s = INFINITY;
+            if (a >= FLT_MIN && a <= FLT_MAX) s = sse_of(x, k, a, lo, hi);
+            if (sse_curve) sse_curve[c] = s;
+            if (s < best_sse) {
+                best_sse = s;
+                best = c;
+            }
+        }
+    }
+
+    if (best < 0) {
+        double s = 0.0;
+        for (int64_t i = 0; i < k; ++i) s += (double)x[i] * (double)x[i];
+        *alpha = 0.0f;
+        *sse = s;
+        *best_idx = -1;
+        if (codes) memset(codes, 0, (size_t)k);
+        *status |= st | ORACLE_STATUS_DEGENERATE;
+        return;
+    }
+
+    float a = omse_oracle_candidate(m, hi_frac, n_cand, best);
+    a = refine_from(x, k, a, lo, hi, refine_iters);
+    *alpha = a;
+    *sse = sse_of(x, k, a, lo, hi);
+    *best_idx = best;
+    if (codes)
+        for (int64_t i = 0; i < k; ++i) codes[i] = (int8_t)code_of(x[i], a, lo, hi);
+    *status |= st;
+}
+
+/* Kernel-wise quantization (Section 3.3): phi applied independently to each of the
+ * n_kernels contiguous segments of kernel_len elements.  start_idx is nullable. */
+void omse_oracle_quantize_rows(const float *w, int64_t n_kernels, int64_t kernel_len, int bits,
+                               int is_signed, int n_cand, float hi_frac, int refine_iters,
+                               const int32_t *start_idx, float *alpha, double *sse,
+                               int32_t *best_idx, int8_t *codes, uint32_t *status)
+{
+    uint32_t st_all = 0;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 1) reduction(| : st_all)
+#endif
+    for (int64_t s = 0; s < n_kernels; ++s) {
+        uint32_t st = 0;
+        omse_oracle_phi(w + s * kernel_len, kernel_len, bits, is_signed, n_cand, hi_frac,
+                        refine_iters, start_idx ? start_idx[s] : -1, &alpha[s], &sse[s],
+                        &best_idx[s], codes ? codes + s * kernel_len : NULL, NULL, &st);
+        st_all |= st;
+    }
+    *status |= st_all;
+}
+
+/* Per-tensor search (Section 3.7, one beta for a whole activation tensor): the same phi on
+ * one segment of n elements, with the independent candidates spread over threads. */
+void omse_oracle_activation_scale(const float *x, int64_t n, int bits, int is_signed, int n_cand,
+                                  float hi_frac, int refine_iters, float *alpha, double *sse,
+                                  int32_t *best_idx, double *sse_curve, uint32_t *status)
+{
+    int lo, hi;
+    uint32_t st = 0;
+    omse_oracle_grid_bounds(bits, is_signed, &lo, &hi);
+    float m = max_abs_of(x, n, &st);
+    double *curve = sse_curve ? sse_curve : (double *)malloc(sizeof(double) * (size_t)n_cand);
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 1)
+#endif
+    for (int c = 0; c < n_cand; ++c) {
+        float a = omse_oracle_candidate(m, hi_frac, n_cand, c);
+        curve[c] = (a >= FLT_MIN && a <= FLT_MAX) ? sse_of(x, n, a, lo, hi) : INFINITY;
+    }
+    int best = -1;
+    double best_sse = INFINITY;
+    for (int c = 0; c < n_cand; ++c)
+        if (curve[c] < best_sse) {
+            best_sse = curve[c];
+            best = c;
+        }
+    if (!sse_curve) free(curve);
+    /* polish and final error from the chosen candidate (serial, as in phi) */
+    omse_oracle_phi(x, n, bits, is_signed, n_cand, hi_frac, refine_iters, best >= 0 ? best : 0,
+                    alpha, sse, best_idx, NULL, NULL, &st);
+    if (best < 0) *best_idx = -1;
+    *status |= st;
+}
+
+/*
+ * Algorithm 1 (alternating optimisation for multiple quantization) on one segment:
+ * for each sweep, for j = 1..n: r = T - sum_{i != j} alpha_i T~^i, (alpha_j, T~^j) = phi(r, p_j).
+ * All alpha_i and T~^i start at zero, so the first sweep quantizes the residual of the
+ * previous approximation (Section 3.7, "one iteration only").  The residual is formed in
+ * binary32 by successive fused multiply-adds in increasing i.
+ * Outputs (last sweep): alpha[n], sse[n] (error after tensors 1..j were updated),
+ * best_idx[n], codes[n][k]; r_scratch[k] is caller-provided scratch.
+ */
+static void alg1_segment(const float *x, int64_t k, const int *bits, int is_signed, int n_cand,
+                         float hi_frac, int refine_iters, int n_tensors, int n_sweeps,
+                         int64_t out_stride, float *alpha, double *sse, int32_t *best_idx,
+                         int8_t *codes, int64_t code_stride, float *r, uint32_t *status)
+{
+    for (int j = 0; j < n_tensors; ++j) {
+        alpha[j * out_stride] = 0.0f;
+        memset(codes + j * code_stride, 0, (size_t)k);
+    }
+    for (int sweep = 0; sweep < n_sweeps; ++sweep) {
+        for (int j = 0; j < n_tensors; ++j) {
+            for (int64_t e = 0; e < k; ++e) {
+                float v = x[e];
+                for (int i = 0; i < n_tensors; ++i)
+                    if (i != j)
+                        v = fmaf(-alpha[i * out_stride], (float)codes[i * code_stride + e], v);
+                r[e] = v;
+            }
+            double s_j;
+            omse_oracle_phi(r, k, bits[j], is_signed, n_cand, hi_frac, refine_iters, -1,
+                            &alpha[j * out_stride], &s_j, &best_idx[j * out_stride],
+                            codes + j * code_stride, NULL, status);
+            sse[j * out_stride] = s_j;
+        }
+    }
+}
+
+void omse_oracle_residual_rows(const float *t, int64_t n_kernels, int64_t kernel_len,
+                               const int *bits, int is_signed, int n_cand, float hi_frac,
+                               int refine_iters, int n_tensors, int n_sweeps, float *alpha,
+                               double *sse, int32_t *best_idx, int8_t *codes, uint32_t *status)
+{
+    /* layouts: alpha/sse/best_idx [n_tensors][n_kernels]; codes [n_tensors][n_kernels*kernel_len] */
+    int64_t n = n_kernels * kernel_len;
+    uint32_t st_all = 0;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 1) reduction(| : st_all)
+#endif
+    for (int64_t s = 0; s < n_kernels; ++s) {
+        uint32_t st = 0;
+        float *r = (float *)malloc(sizeof(float) * (size_t)kernel_len);
+        alg1_segment(t + s * kernel_len, kernel_len, bits, is_signed, n_cand, hi_frac, refine_iters,
+                     n_tensors, n_sweeps, n_kernels, alpha + s, sse + s, best_idx + s,
+                     codes + s * kernel_len, n, r, &st);
+        free(r);
+        st_all |= st;
+    }
+    *status |= st_all;
+}
+
+/* INT4 code emission.  The paper fixes no byte layout; this library's layout is: element e
+ * (flat, row-major) goes to byte e/2, even e in bits 0-3, odd e in bits 4-7, the nibble being
+ * the low four bits of the two's-complement code; a trailing odd element leaves bits 4-7 zero. */
+void omse_oracle_pack_int4(const int8_t *codes, int64_t n, uint8_t *packed)
+{
+    for (int64_t b = 0; b < (n + 1) / 2; ++b) {
+        uint8_t lo = (uint8_t)codes[2 * b] & 0xF;
+        uint8_t hi = (2 * b + 1 < n) ? ((uint8_t)codes[2 * b + 1] & 0xF) : 0;
+        packed[b] = (uint8_t)(lo | (hi << 4));
+    }
+}
+
+void omse_oracle_unpack_int4(const uint8_t *packed, int64_t n, int is_signed, int8_t *codes)
+{
+    for (int64_t e = 0; e < n; ++e) {
+        int v = (packed[e >> 1] >> ((e & 1) * 4)) & 0xF;
+        if (is_signed && v >= 8) v -= 16;
+        codes[e] = (int8_t)v;
+    }
+}

@@ -1,0 +1,203 @@
+"""ctypes front end of the CPU oracle (``omse_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: the CUDA library never imports this module.  It compiles the
+C file with gcc on first use and exposes the oracle's functions on numpy arrays.
+Every function's arithmetic lives in the C file; this module only marshals arguments.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "omse_oracle.c")
+_LIB = os.path.join(_HERE, "libomse_oracle.so")
+
+STATUS_NONFINITE = 1
+STATUS_DEGENERATE = 2
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle (no fast-math, no contraction) and return the library path."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-std=c99", "-fopenmp", "-ffp-contract=off", "-fno-fast-math",
+               "-shared", "-fPIC", "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is not None:
+        return _lib
+    lib = C.CDLL(build())
+    f32p, f64p = C.POINTER(C.c_float), C.POINTER(C.c_double)
+    i32p, i8p, u8p, u32p = C.POINTER(C.c_int32), C.POINTER(C.c_int8), C.POINTER(C.c_uint8), C.POINTER(C.c_uint32)
+    lib.omse_oracle_max_threads.restype = C.c_int
+    lib.omse_oracle_grid_bounds.argtypes = [C.c_int, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_int)]
+    lib.omse_oracle_sse_at.restype = C.c_double
+    lib.omse_oracle_sse_at.argtypes = [f32p, C.c_int64, C.c_float, C.c_int, C.c_int]
+    lib.omse_oracle_codes.argtypes = [f32p, C.c_int64, C.c_float, C.c_int, C.c_int, i8p]
+    lib.omse_oracle_candidate.restype = C.c_float
+    lib.omse_oracle_candidate.argtypes = [C.c_float, C.c_float, C.c_int, C.c_int]
+    lib.omse_oracle_phi.argtypes = [f32p, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_float, C.c_int, C.c_int,
+                                    f32p, f64p, i32p, i8p, f64p, u32p]
+    lib.omse_oracle_quantize_rows.argtypes = [f32p, C.c_int64, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_float,
+                                              C.c_int, i32p, f32p, f64p, i32p, i8p, u32p]
+    lib.omse_oracle_activation_scale.argtypes = [f32p, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_float, C.c_int,
+                                                 f32p, f64p, i32p, f64p, u32p]
+    lib.omse_oracle_residual_rows.argtypes = [f32p, C.c_int64, C.c_int64, C.POINTER(C.c_int), C.c_int, C.c_int,
+                                              C.c_float, C.c_int, C.c_int, C.c_int, f32p, f64p, i32p, i8p, u32p]
+    lib.omse_oracle_pack_int4.argtypes = [i8p, C.c_int64, u8p]
+    lib.omse_oracle_unpack_int4.argtypes = [u8p, C.c_int64, C.c_int, i8p]
+    _lib = lib
+    return lib
+
+
+def _p(a, ct):
+    return None if a is None else a.ctypes.data_as(C.POINTER(ct))
+
+
+def _c32(v) -> float:
+    return float(np.float32(v))
+
+
+def _f32(x):
+    return np.ascontiguousarray(x, dtype=np.float32)
+
+
+def max_threads() -> int:
+    return int(_load().omse_oracle_max_threads())
+
+
+def grid_bounds(bits: int, is_signed: bool):
+    lo, hi = C.c_int(), C.c_int()
+    _load().omse_oracle_grid_bounds(bits, int(is_signed), C.byref(lo), C.byref(hi))
+    return lo.value, hi.value
+
+
+def candidate(max_abs: float, hi_frac: float, n_cand: int, c: int) -> float:
+    return float(_load().omse_oracle_candidate(_c32(max_abs), _c32(hi_frac), n_cand, c))
+
+
+def sse_at(x, alpha: float, bits: int, is_signed: bool) -> float:
+    x = _f32(x).ravel()
+    return float(_load().omse_oracle_sse_at(_p(x, C.c_float), x.size, _c32(alpha), bits, int(is_signed)))
+
+
+def codes(x, alpha: float, bits: int, is_signed: bool) -> np.ndarray:
+    x = _f32(x)
+    out = np.empty(x.shape, dtype=np.int8)
+    _load().omse_oracle_codes(_p(x, C.c_float), x.size, _c32(alpha), bits, int(is_signed), _p(out, C.c_int8))
+    return out
+
+
+@dataclass
+class PhiResult:
+    alpha: float
+    sse: float
+    best_idx: int
+    codes: np.ndarray | None
+    sse_curve: np.ndarray | None
+    status: int
+
+
+def phi(x, bits=4, is_signed=True, n_cand=256, hi_frac=1.0, refine_iters=3, start_idx=-1,
+        want_codes=True, want_curve=False) -> PhiResult:
+    """The quantization mapping of Section 3.4 on one segment."""
+    x = _f32(x).ravel()
+    a, s, i, st = C.c_float(), C.c_double(), C.c_int32(), C.c_uint32(0)
+    q = np.empty(x.size, dtype=np.int8) if want_codes else None
+    curve = np.empty(n_cand, dtype=np.float64) if want_curve else None
+    _load().omse_oracle_phi(_p(x, C.c_float), x.size, bits, int(is_signed), n_cand, _c32(hi_frac),
+                            refine_iters, start_idx, C.byref(a), C.byref(s), C.byref(i),
+                            _p(q, C.c_int8), _p(curve, C.c_double), C.byref(st))
+    return PhiResult(a.value, s.value, i.value, q, curve, st.value)
+
+
+@dataclass
+class RowsResult:
+    alpha: np.ndarray      # [S] float32
+    sse: np.ndarray        # [S] float64
+    best_idx: np.ndarray   # [S] int32
+    codes: np.ndarray | None  # [S, K] int8
+    status: int
+
+
+def quantize_rows(w, bits=4, is_signed=True, n_cand=256, hi_frac=1.0, refine_iters=3, start_idx=None,
+                  want_codes=True) -> RowsResult:
+    """Kernel-wise phi over the rows of a 2-D array [n_kernels, kernel_len] (Section 3.3)."""
+    w = _f32(w)
+    assert w.ndim == 2
+    S, K = w.shape
+    alpha = np.empty(S, np.float32)
+    sse = np.empty(S, np.float64)
+    idx = np.empty(S, np.int32)
+    q = np.empty((S, K), np.int8) if want_codes else None
+    st = C.c_uint32(0)
+    si = None if start_idx is None else np.ascontiguousarray(start_idx, dtype=np.int32)
+    _load().omse_oracle_quantize_rows(_p(w, C.c_float), S, K, bits, int(is_signed), n_cand, _c32(hi_frac),
+                                      refine_iters, _p(si, C.c_int32), _p(alpha, C.c_float), _p(sse, C.c_double),
+                                      _p(idx, C.c_int32), _p(q, C.c_int8), C.byref(st))
+    return RowsResult(alpha, sse, idx, q, st.value)
+
+
+def activation_scale(x, bits=4, is_signed=False, n_cand=2048, hi_frac=1.0, refine_iters=3,
+                     want_curve=True) -> PhiResult:
+    """Per-tensor phi (Section 3.7) with the candidates spread over the host threads."""
+    x = _f32(x).ravel()
+    a, s, i, st = C.c_float(), C.c_double(), C.c_int32(), C.c_uint32(0)
+    curve = np.empty(n_cand, dtype=np.float64) if want_curve else None
+    _load().omse_oracle_activation_scale(_p(x, C.c_float), x.size, bits, int(is_signed), n_cand,
+                                         _c32(hi_frac), refine_iters, C.byref(a), C.byref(s), C.byref(i),
+                                         _p(curve, C.c_double), C.byref(st))
+    return PhiResult(a.value, s.value, i.value, None, curve, st.value)
+
+
+@dataclass
+class ResidualResult:
+    alpha: np.ndarray      # [n_tensors, S]
+    sse: np.ndarray        # [n_tensors, S] float64: error after tensors 1..j
+    best_idx: np.ndarray   # [n_tensors, S]
+    codes: np.ndarray      # [n_tensors, S, K] int8
+    status: int
+
+
+def residual_rows(t, bits=(4, 4), is_signed=True, n_cand=1024, hi_frac=1.0, refine_iters=3,
+                  n_sweeps=1) -> ResidualResult:
+    """Algorithm 1 (Section 3.5) applied kernel-wise; n_sweeps=1 is the residual scheme of Section 3.7."""
+    t = _f32(t)
+    assert t.ndim == 2
+    S, K = t.shape
+    n = len(bits)
+    b = (C.c_int * n)(*bits)
+    alpha = np.zeros((n, S), np.float32)
+    sse = np.zeros((n, S), np.float64)
+    idx = np.zeros((n, S), np.int32)
+    q = np.zeros((n, S, K), np.int8)
+    st = C.c_uint32(0)
+    _load().omse_oracle_residual_rows(_p(t, C.c_float), S, K, b, int(is_signed), n_cand, _c32(hi_frac),
+                                      refine_iters, n, n_sweeps, _p(alpha, C.c_float), _p(sse, C.c_double),
+                                      _p(idx, C.c_int32), _p(q, C.c_int8), C.byref(st))
+    return ResidualResult(alpha, sse, idx, q, st.value)
+
+
+def pack_int4(codes_) -> np.ndarray:
+    q = np.ascontiguousarray(codes_, dtype=np.int8).ravel()
+    out = np.empty((q.size + 1) // 2, np.uint8)
+    _load().omse_oracle_pack_int4(_p(q, C.c_int8), q.size, _p(out, C.c_uint8))
+    return out
+
+
+def unpack_int4(packed, n: int, is_signed: bool) -> np.ndarray:
+    p = np.ascontiguousarray(packed, dtype=np.uint8).ravel()
+    out = np.empty(n, np.int8)
+    _load().omse_oracle_unpack_int4(_p(p, C.c_uint8), n, int(is_signed), _p(out, C.c_int8))
+    return out

@@ -1,0 +1,301 @@
+"""Pins for the CPU oracle: what the paper and the mathematics fix, checked without a GPU.
+
+Each test is chosen so that a plausible slip in the oracle (dropped term, wrong sign or
+index, wrong grid bound, transposed layout) makes it fail.
+"""
+import os
+
+import numpy as np
+import pytest
+
+from oracle import omse_oracle as orc
+from paper_1902_06822_b200 import synth
+from exact_opt import exact_optimum
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _bounds(bits, signed):
+    return (-(1 << (bits - 1)), (1 << (bits - 1)) - 1) if signed else (0, (1 << bits) - 1)
+
+
+# ---------------------------------------------------------------- Section 3.1: grids, operator
+def test_grid_bounds_match_section_3_1():
+    assert orc.grid_bounds(4, True) == (-8, 7)
+    assert orc.grid_bounds(4, False) == (0, 15)
+    assert orc.grid_bounds(2, True) == (-2, 1)
+    assert orc.grid_bounds(8, True) == (-128, 127)
+    assert orc.grid_bounds(8, False) == (0, 255)
+
+
+def test_rounding_is_half_to_even_then_saturates():
+    # x/alpha with alpha = 1: 0.5 -> 0, 1.5 -> 2, 2.5 -> 2, -0.5 -> 0, -1.5 -> -2, 7.5 -> 8 -> 7, -9 -> -8
+    x = np.array([0.5, 1.5, 2.5, -0.5, -1.5, 7.5, -9.0, 6.5, 100.0], np.float32)
+    assert orc.codes(x, 1.0, 4, True).tolist() == [0, 2, 2, 0, -2, 7, -8, 6, 7]
+    assert orc.codes(x, 1.0, 4, False).tolist() == [0, 2, 2, 0, 0, 8, 0, 6, 15]
+
+
+# ---------------------------------------------------------------- hand-worked example
+def test_hand_worked_two_bit_example():
+    """x = (0.9, -0.35, 0.1, 0.5), signed 2-bit grid {-2..1}, 4 candidates in (0, 0.9].
+
+    By hand: alpha = 0.225, 0.45, 0.675, 0.9 give squared errors 0.55125, 0.225, 0.196875, 0.2925
+    (codes (1,-2,0,1), (1,-1,0,1), (1,-1,0,1), (1,0,0,1)); the third wins.  With codes (1,-1,0,1)
+    the least-squares scale is (0.9+0.35+0.5)/3 = 0.58333..., which re-quantizes to the same codes,
+    and the error is 0.31667^2 + 0.23333^2 + 0.1^2 + 0.08333^2 = 0.171667.
+    """
+    x = np.array([0.9, -0.35, 0.1, 0.5], np.float32)
+    r0 = orc.phi(x, bits=2, is_signed=True, n_cand=4, refine_iters=0, want_curve=True)
+    np.testing.assert_allclose(r0.sse_curve, [0.55125, 0.225, 0.196875, 0.2925], rtol=1e-6)
+    assert r0.best_idx == 2 and r0.codes.tolist() == [1, -1, 0, 1]
+    np.testing.assert_allclose(r0.alpha, 0.675, rtol=1e-6)
+    r3 = orc.phi(x, bits=2, is_signed=True, n_cand=4, refine_iters=3)
+    np.testing.assert_allclose(r3.alpha, 1.75 / 3.0, rtol=1e-6)
+    np.testing.assert_allclose(r3.sse, 0.1716667, rtol=1e-5)
+    assert r3.codes.tolist() == [1, -1, 0, 1] and r3.best_idx == 2
+
+
+def test_lowest_index_wins_exact_ties():
+    # K = 1, x = 1: candidates 1/4, 1/2, 3/4, 1 reproduce x with codes 4, 2, (1), 1: three exact zeros.
+    r = orc.phi(np.array([1.0], np.float32), bits=4, n_cand=4, refine_iters=0, want_curve=True)
+    assert r.sse_curve.tolist() == [0.0, 0.0, 0.0625, 0.0]
+    assert r.best_idx == 0 and r.alpha == 0.25 and r.codes.tolist() == [4]
+
+
+# ---------------------------------------------------------------- Section 3.4: exact optimum (brute force)
+def _tiny_cases():
+    rng = np.random.default_rng(1234)
+    for trial in range(60):
+        k = int(rng.choice([1, 2, 3, 8, 27, 64]))
+        bits = int(rng.choice([2, 3, 4]))
+        signed = bool(rng.integers(0, 2))
+        n_cand = int(rng.choice([16, 64, 256]))
+        if trial % 2:
+            x = rng.laplace(0.0, 0.02, k)
+        else:
+            x = rng.standard_t(3, k)
+        if not signed and trial % 3 == 0:
+            x = np.abs(x)
+        yield x.astype(np.float32), bits, signed, n_cand
+
+
+@pytest.mark.parametrize("case", list(_tiny_cases()), ids=lambda c: f"K{c[0].size}-p{c[1]}-{'s' if c[2] else 'u'}-C{c[3]}")
+def test_grid_search_within_grid_resolution_of_exact_optimum(case):
+    x, bits, signed, n_cand = case
+    lo, hi = _bounds(bits, signed)
+    m = float(np.max(np.abs(x)))
+    step = m / n_cand
+    r0 = orc.phi(x, bits, signed, n_cand, 1.0, 0, want_curve=True)
+    r3 = orc.phi(x, bits, signed, n_cand, 1.0, 3)
+    # (a) nothing on (0, max|x|] beats the grid answer by more than the grid resolution allows:
+    #     ||x - a_c q*|| <= ||x - a* q*|| + |a_c - a*| ||q*||, and rounding at a_c can only do better.
+    sse_star, a_star, q_star = exact_optimum(x, lo, hi, a_max=m)
+    grid = (np.arange(n_cand) + 1) * step
+    dist = float(np.min(np.abs(grid - a_star)))
+    assert dist <= step * (1 + 1e-9)
+    bound = (np.sqrt(sse_star) + dist * np.linalg.norm(q_star)) ** 2
+    assert r0.sse <= bound * (1 + 1e-5) + 1e-30
+    # (b) the polished answer never gets worse than the grid answer
+    assert r3.sse <= r0.sse * (1 + 1e-6) + 1e-30
+    # (c) and no answer can be better than the true optimum over all alpha > 0
+    sse_glob, _, _ = exact_optimum(x, lo, hi)
+    assert sse_glob <= sse_star * (1 + 1e-12)
+    assert r3.sse >= sse_glob * (1 - 1e-6) - 1e-30
+    assert r0.sse >= sse_star * (1 - 1e-6) - 1e-30
+    # (d) the reported minimum is the minimum of the reported curve, lowest index first
+    assert r0.best_idx == int(np.argmin(r0.sse_curve))
+    assert r0.sse == pytest.approx(r0.sse_curve[r0.best_idx], rel=1e-12)
+
+
+def test_sse_curve_matches_definition_in_numpy():
+    """Section 3.4 objective at every candidate, recomputed with numpy (fp32 divide, fp64 error)."""
+    x = synth.laplace(576, 0.02, seed=11)
+    for bits, signed in [(4, True), (4, False), (3, True), (8, True)]:
+        lo, hi = _bounds(bits, signed)
+        r = orc.phi(x, bits, signed, 128, 1.0, 0, want_curve=True)
+        m = np.float32(np.max(np.abs(x)))
+        step = np.float32(m) / np.float32(128)
+        for c in (0, 1, 17, 63, 127, r.best_idx):
+            a = np.float32(c + 1) * step
+            q = np.clip(np.rint(x / a), lo, hi).astype(np.float64)
+            sse = np.sum((x.astype(np.float64) - np.float64(a) * q) ** 2)
+            assert r.sse_curve[c] == pytest.approx(sse, rel=1e-12)
+            assert orc.candidate(m, 1.0, 128, c) == float(a)
+
+
+# ---------------------------------------------------------------- special cases with closed forms
+def test_input_already_on_a_candidate_grid_is_reproduced_exactly():
+    a = 2.0 ** -5
+    k = np.array([-8, 7, 3, 0, -1, 5, 7, -8, 2, 1, -4, 6], np.float32)
+    x = k * np.float32(a)          # max|x| = 8a; with 64 candidates the step is a/8, so candidate 7 is a
+    r = orc.phi(x, 4, True, 64, 1.0, 3, want_curve=True)
+    assert r.best_idx == 7 and r.sse == 0.0 and r.alpha == a
+    assert r.codes.tolist() == k.astype(int).tolist()
+    assert np.count_nonzero(r.sse_curve == 0.0) == 1
+
+
+def test_single_element_segment_is_reproduced_after_polish():
+    for v in (0.37, -1.9, 3e-5):
+        r = orc.phi(np.array([v], np.float32), 4, True, 16, 1.0, 1)
+        assert abs(r.alpha * int(r.codes[0]) - np.float32(v)) <= 1e-6 * abs(v)
+        assert r.sse <= (1e-6 * v) ** 2
+
+
+@pytest.mark.parametrize("bits,signed", [(4, True), (3, True), (8, True), (4, False)])
+def test_one_candidate_at_max_over_L_is_the_uniform_quantizer(bits, signed):
+    """Section 3.1 without offset: alpha = max|T| / (2^(p-1) - 1), codes = [T/alpha]."""
+    lo, hi = _bounds(bits, signed)
+    x = synth.student_t3(300, seed=7, tensor_id=bits)
+    if not signed:
+        x = np.abs(x)
+    r = orc.phi(x, bits, signed, 1, 1.0 / hi, 0)
+    a_paper = float(np.max(np.abs(x))) / hi
+    assert r.alpha == pytest.approx(a_paper, rel=3e-7) and r.best_idx == 0
+    q = np.clip(np.rint(x / np.float32(r.alpha)), lo, hi).astype(np.float64)
+    assert np.array_equal(r.codes, q.astype(np.int8))
+    assert r.sse == pytest.approx(np.sum((x.astype(np.float64) - r.alpha * q) ** 2), rel=1e-12)
+    assert r.sse <= float(np.sum(x.astype(np.float64) ** 2))
+
+
+def test_eight_bit_error_follows_uniform_noise_model():
+    """No saturation, fine grid: squared error per element ~ alpha^2 / 12 (textbook rounding noise)."""
+    rng = np.random.default_rng(5)
+    x = rng.uniform(-1.0, 1.0, 20000).astype(np.float32)
+    r = orc.phi(x, 8, True, 1, 1.0 / 127, 0)
+    assert r.sse / x.size == pytest.approx(r.alpha ** 2 / 12.0, rel=0.05)
+
+
+# ---------------------------------------------------------------- invariants
+def test_invariants_on_cnn_shaped_rows():
+    w = synth.conv_layer(seed=1)[:16]
+    prev = None
+    for bits in (2, 3, 4, 8):
+        lo, hi = _bounds(bits, True)
+        res = orc.quantize_rows(w, bits, True, 256, 1.0, 3)
+        res0 = orc.quantize_rows(w, bits, True, 256, 1.0, 0)
+        assert res.codes.min() >= lo and res.codes.max() <= hi
+        assert np.all(res.sse <= res0.sse * (1 + 1e-9))             # polish never hurts
+        assert np.all(res.sse <= np.sum(w.astype(np.float64) ** 2, axis=1))
+        assert np.array_equal(res.best_idx, res0.best_idx)
+        if prev is not None:
+            assert res.sse.mean() < prev                              # error shrinks with bit width
+        prev = res.sse.mean()
+
+
+def test_power_of_two_scaling_is_exact_and_permutation_keeps_alpha():
+    x = synth.student_t3(147, seed=9)
+    r = orc.phi(x, 4, True, 256, 1.0, 3)
+    r8 = orc.phi(x * np.float32(8.0), 4, True, 256, 1.0, 3)
+    assert r8.alpha == r.alpha * 8.0 and np.array_equal(r8.codes, r.codes) and r8.best_idx == r.best_idx
+    assert r8.sse == pytest.approx(64.0 * r.sse, rel=1e-12)
+    perm = np.random.default_rng(0).permutation(x.size)
+    rp = orc.phi(x[perm], 4, True, 256, 1.0, 0)
+    r0 = orc.phi(x, 4, True, 256, 1.0, 0)
+    assert rp.alpha == r0.alpha and rp.best_idx == r0.best_idx and np.array_equal(rp.codes, r0.codes[perm])
+    assert rp.sse == pytest.approx(r0.sse, rel=1e-12)
+
+
+def test_grid_search_beats_alternation_from_the_uniform_start_somewhere():
+    """Section 3.4: alternation alone is not robust (non-convex objective); the grid is."""
+    w = synth.resnet50_weights(seed=2)[1][1][:64]       # 64 rows of a 1x1 convolution
+    grid = orc.quantize_rows(w, 4, True, 256, 1.0, 3).sse
+    alt = orc.quantize_rows(w, 4, True, 1, 1.0 / 7, 10).sse   # uniform start + 10 alternations
+    assert np.all(grid <= alt * 1.05)
+    assert np.mean(grid < alt * 0.999) > 0.25
+
+
+def test_degenerate_rows():
+    r = orc.phi(np.zeros(9, np.float32), 4, True, 16, 1.0, 3)
+    assert r.alpha == 0.0 and r.best_idx == -1 and r.sse == 0.0 and not r.codes.any()
+    assert r.status & orc.STATUS_DEGENERATE
+    r = orc.phi(np.array([1.0, np.nan, 0.5], np.float32), 4, True, 16, 1.0, 0)
+    assert r.status & orc.STATUS_NONFINITE
+
+
+# ---------------------------------------------------------------- layouts: rows, per tensor, restart
+def test_rows_per_tensor_and_restart_agree_with_single_segment_phi():
+    w = synth.sweep_tensor(27, seed=5, n_kernels=10)
+    res = orc.quantize_rows(w, 3, True, 64, 1.0, 2)
+    for s in (0, 4, 9):
+        r = orc.phi(w[s], 3, True, 64, 1.0, 2)
+        assert (r.alpha, r.sse, r.best_idx) == (res.alpha[s], res.sse[s], res.best_idx[s])
+        assert np.array_equal(r.codes, res.codes[s])
+    again = orc.quantize_rows(w, 3, True, 64, 1.0, 2, start_idx=res.best_idx)
+    assert np.array_equal(again.alpha, res.alpha) and np.array_equal(again.codes, res.codes)
+    x = synth.relu_activations(5000, seed=3)
+    a = orc.activation_scale(x, 4, False, 128, 1.0, 3)
+    r = orc.phi(x, 4, False, 128, 1.0, 3, want_curve=True)
+    assert (a.alpha, a.sse, a.best_idx) == (r.alpha, r.sse, r.best_idx)
+    assert np.array_equal(a.sse_curve, r.sse_curve)
+
+
+# ---------------------------------------------------------------- Section 3.5 / 3.7: residual, Algorithm 1
+def test_residual_quantization_bookkeeping_and_gain():
+    t = synth.laplace_with_outliers(12 * 200, 0.005, seed=4, outlier_prob=0.01).reshape(12, 200)
+    res = orc.residual_rows(t, (4, 4), True, 128, 1.0, 3, n_sweeps=1)
+    t64 = t.astype(np.float64)
+    first = orc.quantize_rows(t, 4, True, 128, 1.0, 3)
+    # tensor 1 of the first sweep is plain phi(T)
+    assert np.array_equal(res.alpha[0], first.alpha) and np.array_equal(res.codes[0], first.codes)
+    np.testing.assert_allclose(res.sse[0], first.sse, rtol=1e-12)
+    # tensor 2 is phi of the fp32 residual T - alpha1*q1
+    r1 = np.empty_like(t)
+    for s in range(12):
+        r1[s] = (t64[s] - np.float64(res.alpha[0, s]) * res.codes[0, s]).astype(np.float32)  # exact product, one rounding
+    second = orc.quantize_rows(r1, 4, True, 128, 1.0, 3)
+    assert np.array_equal(res.alpha[1], second.alpha) and np.array_equal(res.codes[1], second.codes)
+    # the reported errors are the reconstruction errors of Section 3.5's objective
+    rec1 = res.alpha[0][:, None].astype(np.float64) * res.codes[0]
+    rec2 = rec1 + res.alpha[1][:, None].astype(np.float64) * res.codes[1]
+    np.testing.assert_allclose(res.sse[0], np.sum((t64 - rec1) ** 2, axis=1), rtol=1e-9)
+    np.testing.assert_allclose(res.sse[1], np.sum((t64 - rec2) ** 2, axis=1), rtol=1e-6)
+    assert np.all(res.sse[1] < res.sse[0])                      # a second tensor shrinks the error
+    assert res.sse[1].sum() < 0.1 * res.sse[0].sum()
+
+
+def test_algorithm_1_second_sweep_uses_all_other_tensors():
+    t = synth.student_t3(5 * 96, seed=21).reshape(5, 96)
+    one = orc.residual_rows(t, (3, 3), True, 64, 1.0, 2, n_sweeps=1)
+    two = orc.residual_rows(t, (3, 3), True, 64, 1.0, 2, n_sweeps=2)
+    t64 = t.astype(np.float64)
+    # second sweep, j = 1: phi(T - alpha2*q2) with the first sweep's second tensor
+    for s in range(5):
+        r = np.float32(t64[s] - np.float64(one.alpha[1, s]) * one.codes[1, s])
+        p = orc.phi(r, 3, True, 64, 1.0, 2)
+        assert p.alpha == two.alpha[0, s] and np.array_equal(p.codes, two.codes[0, s])
+    rec = sum(two.alpha[j][:, None].astype(np.float64) * two.codes[j] for j in range(2))
+    np.testing.assert_allclose(two.sse[1], np.sum((t64 - rec) ** 2, axis=1), rtol=1e-6)
+    assert two.sse[1].sum() <= one.sse[1].sum() * 1.02
+
+
+def test_three_tensors_keep_shrinking_the_error():
+    t = synth.laplace(4 * 300, 0.01, seed=8).reshape(4, 300)
+    res = orc.residual_rows(t, (2, 2, 2), True, 64, 1.0, 2, n_sweeps=1)
+    assert np.all(res.sse[1] < res.sse[0]) and np.all(res.sse[2] < res.sse[1])
+    assert res.codes.min() >= -2 and res.codes.max() <= 1
+
+
+# ---------------------------------------------------------------- INT4 packing and compression ratio
+def test_pack_layout_by_hand_and_round_trip_over_all_bytes():
+    assert orc.pack_int4(np.array([1, -1, 7], np.int8)).tolist() == [0xF1, 0x07]
+    assert orc.pack_int4(np.array([-8, 3, 0, -2], np.int8)).tolist() == [0x38, 0xE0]
+    allbytes = np.arange(256, dtype=np.uint8)
+    for signed in (True, False):
+        q = orc.unpack_int4(allbytes, 512, signed)
+        lo, hi = _bounds(4, signed)
+        assert q.min() == lo and q.max() == hi
+        assert np.array_equal(orc.pack_int4(q), allbytes)
+        assert q[2 * 0x5A] == (0xA - 16 if signed else 0xA) and q[2 * 0x5A + 1] == 5
+
+
+def test_compression_ratio_of_resnet50_shape_set_matches_the_paper():
+    gold = dict(line.split() for line in open(os.path.join(GOLDEN, "compression_ratio.txt")) if line[0] != "#")
+    shapes = synth.resnet50_shapes()
+    n = sum(s * k for _, s, k in shapes)
+    rows = sum(s for _, s, k in shapes)
+    assert (len(shapes), n, rows) == (54, 25_502_912, 27_560)
+    packed_bytes = sum(orc.pack_int4(np.zeros(s * k, np.int8)).size for _, s, k in shapes[:3]) \
+        + sum((s * k + 1) // 2 for _, s, k in shapes[3:])
+    cr = (packed_bytes + 4 * rows) / (4 * n)           # codes + one fp32 scale per kernel over the fp32 model
+    assert float(gold["int4_non_dual_cr_approx"]) <= cr <= float(gold["resnet50_cr_with_dual_layers"]) + 5e-5
+    assert cr == pytest.approx(0.12608, abs=1e-5)

@@ -1,0 +1,150 @@
+/*
+ * omse.h - C interface of the B200 (sm_100a) constrained-MMSE quantization library.
+ *
+ * The library computes the data-parallel part of "Low-bit Quantization of Neural Networks
+ * for Efficient Inference" (Choukroun et al., arXiv:1902.06822): for a tensor T and a
+ * b-bit integer range Z_p it finds the scale alpha minimising ||T - alpha*[T/alpha]_Zp||_F^2
+ * (Section 3.4) by evaluating a grid of candidate scales and polishing the best one with
+ * the closed-form least-squares update; kernel-wise for weights (Section 3.3), per tensor
+ * for activations (Section 3.7); optionally as a sum of several low-precision tensors
+ * (Section 3.5, Algorithm 1; Section 3.7 residual form); and it emits INT4 codes.
+ *
+ * Conventions that hold for every entry point
+ *   - Every pointer named d_* is DEVICE memory owned by the caller.  It must stay valid until
+ *     the work queued by the call has finished on the context's stream.  The library keeps
+ *     no pointer after the work completes.  float/int32 buffers must be 4-byte aligned,
+ *     double buffers 8-byte aligned; there is no other alignment requirement.
+ *   - Pointers without the d_ prefix are HOST memory, read before the call returns.
+ *   - Calls only enqueue work on the context's CUDA stream and return; nothing synchronises
+ *     except omse_last_device_status() and omse_destroy().
+ *   - The return value is OMSE_OK or a negative omse_status.  Invalid arguments are
+ *     rejected before anything is enqueued.  Data-dependent conditions (NaN/Inf in the
+ *     input, an all-zero segment) never fail a call: they set bits in the device status
+ *     word (omse_last_device_status) and produce the outputs documented below.
+ *   - There is no CPU fallback: without a CUDA device omse_create() fails.
+ *
+ * Quantization range (Section 3.1): signed Z_p = {-2^(p-1) .. 2^(p-1)-1}, unsigned
+ * Z_p = {0 .. 2^p-1}.  [.]_Zp is IEEE binary32 division by alpha, round to nearest with
+ * ties to even, then saturation to the range.
+ */
+#ifndef OMSE_H
+#define OMSE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    OMSE_OK = 0,
+    OMSE_EINVAL = -1, /* NULL pointer, size or parameter out of range                 */
+    OMSE_ECUDA = -2,  /* a CUDA runtime call or a kernel launch failed                */
+    OMSE_ENOMEM = -3  /* the context workspace could not be allocated                 */
+} omse_status;
+
+/* bits of the device status word */
+#define OMSE_DEV_NONFINITE 1u  /* a NaN or Inf was read from an input tensor                          */
+#define OMSE_DEV_DEGENERATE 2u /* a segment had max|x| = 0 (or below FLT_MIN*C): alpha=0, codes 0 */
+
+/* Largest supported sizes. */
+#define OMSE_MAX_CANDIDATES 4096   /* n_cand                                                        */
+#define OMSE_MAX_KERNEL_LEN 28672  /* kernel_len of the kernel-wise entry points (one row on chip) */
+#define OMSE_MAX_KERNEL_LEN_MULTISWEEP 25600 /* with n_sweeps > 1 (row and residual both on chip)       */
+#define OMSE_MAX_TENSORS 4         /* n_tensors of omse_residual_quantize                           */
+
+/* The line-search grid of Section 3.4 ("a given grid"): n_cand scales spaced linearly in
+ * (0, hi_frac*max|x|], candidate c (0-based) being fl(fl(c+1) * fl(fl(hi_frac*max|x|)/fl(n_cand)))
+ * in binary32.  refine_iters is the number of closed-form polish steps
+ * (alpha <- <x,q>/<q,q> with q = [x/alpha]_Zp) applied to the best candidate. */
+typedef struct {
+    int32_t n_cand;       /* 1 .. OMSE_MAX_CANDIDATES                    */
+    float hi_frac;        /* > 0; 1.0 puts the last candidate at max|x| */
+    int32_t refine_iters; /* 0 .. 64                                     */
+} omse_grid;
+
+typedef struct omse_ctx omse_ctx;
+
+/* Creates a context bound to CUDA device `device` and to `cuda_stream` (a cudaStream_t, borrowed,
+ * NULL = the legacy default stream).  Allocates a small device workspace (a few MB).  One context
+ * must not be used from two host threads at once.  Returns OMSE_ECUDA if the device is absent. */
+int omse_create(omse_ctx** out, int device, void* cuda_stream);
+
+/* Waits for the stream, frees the workspace and the context. */
+int omse_destroy(omse_ctx* ctx);
+
+/* Replaces the stream later calls enqueue on (borrowed). */
+int omse_set_stream(omse_ctx* ctx, void* cuda_stream);
+
+/* Bytes of device workspace the context holds (informational). */
+size_t omse_workspace_bytes(const omse_ctx* ctx);
+
+/*
+ * Kernel-wise MMSE quantization of a weight tensor (Sections 3.3 and 3.4).
+ * d_w is row-major [n_kernels][kernel_len] binary32: row k is kernel W_lk flattened
+ * (kernel_len = c*w*h).  Each row gets its own scale.  bits in 2..8.
+ * Outputs (each nullable except d_alpha and d_sse):
+ *   d_alpha   [n_kernels] float  final scale (0 for a degenerate row)
+ *   d_sse     [n_kernels] float  ||W_lk - alpha*q||^2 at the final scale (accumulated in binary64)
+ *   d_best_idx[n_kernels] int32  winning grid index, lowest index among equal errors (-1 degenerate)
+ *   d_codes   [n_kernels*kernel_len] int8   the codes q
+ *   d_packed  [ceil(n_kernels*kernel_len/2)] uint8  the same codes as nibbles (layout: omse_pack_int4);
+ *             only for bits <= 4.
+ * Limits: 1 <= kernel_len <= OMSE_MAX_KERNEL_LEN, n_kernels >= 0 (0 enqueues nothing).
+ */
+int omse_quantize_weights(omse_ctx* ctx, const float* d_w, int64_t n_kernels, int64_t kernel_len,
+                          int bits, int is_signed, const omse_grid* grid, float* d_alpha,
+                          float* d_sse, int32_t* d_best_idx, int8_t* d_codes, uint8_t* d_packed);
+
+/*
+ * Per-tensor MMSE scale for an activation tensor (Section 3.7, first equation): one scale for
+ * all n elements of d_x.  Outputs: d_alpha[1], d_sse[1] (float), d_best_idx[1] (nullable),
+ * d_sse_curve[n_cand] (nullable, double): the squared error at every candidate, i.e. the curve of
+ * Figure 1, accumulated in binary32 blocks of 128 elements folded into binary64.
+ * n >= 0 (0 is treated as a degenerate tensor).  d_x must be 16-byte aligned (128-bit loads).
+ */
+int omse_activation_scale(omse_ctx* ctx, const float* d_x, int64_t n, int bits, int is_signed,
+                          const omse_grid* grid, float* d_alpha, float* d_sse,
+                          int32_t* d_best_idx, double* d_sse_curve);
+
+/*
+ * Multiple-tensor quantization T ~ sum_j alpha_j q^j (Section 3.5, Algorithm 1), kernel-wise.
+ * All alpha_j and q^j start at zero; each of the n_sweeps sweeps visits j = 1..n_tensors and
+ * replaces (alpha_j, q^j) by the MMSE quantization (as in omse_quantize_weights, bits[j]) of the
+ * residual T - sum_{i != j} alpha_i q^i, formed in binary32 by fused multiply-adds in increasing i.
+ * n_sweeps = 1 is the residual scheme of Section 3.7 (second equation).
+ * bits: HOST array [n_tensors].  Outputs are for the last sweep, tensor-major:
+ *   d_alpha [n_tensors][n_kernels], d_sse [n_tensors][n_kernels] (error after tensors 1..j updated),
+ *   d_codes [n_tensors][n_kernels*kernel_len] int8 (nullable when n_sweeps == 1),
+ *   d_packed[n_tensors][ceil(n_kernels*kernel_len/2)] (nullable; needs every bits[j] <= 4).
+ * Limits: 1 <= n_tensors <= OMSE_MAX_TENSORS; 1 <= n_sweeps <= 64; n_sweeps > 1 needs d_codes
+ * (the codes of the other tensors are read back from it) and
+ * kernel_len <= OMSE_MAX_KERNEL_LEN_MULTISWEEP.
+ */
+int omse_residual_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, int64_t kernel_len,
+                           const int* bits, int is_signed, const omse_grid* grid, int n_tensors,
+                           int n_sweeps, float* d_alpha, float* d_sse, int8_t* d_codes,
+                           uint8_t* d_packed);
+
+/*
+ * INT4 code emission.  The paper deploys INT4 tensors but fixes no byte layout; this library's is:
+ * element e (flat index) goes to byte e/2, even e in bits 0-3 and odd e in bits 4-7, the nibble
+ * being the low four bits of the two's-complement code; if n is odd, bits 4-7 of the last byte are 0.
+ * d_codes [n] int8 -> d_packed [ceil(n/2)] uint8.  is_signed is accepted for symmetry with the
+ * other calls and does not change the bytes.
+ */
+int omse_pack_int4(omse_ctx* ctx, const int8_t* d_codes, int64_t n, int is_signed,
+                   uint8_t* d_packed);
+
+/* Synchronises the stream, copies the device status word (OMSE_DEV_* bits OR-ed over all calls
+ * since the last read) to *host_out and clears it. */
+int omse_last_device_status(omse_ctx* ctx, uint32_t* host_out);
+
+/* Static description of a return value. */
+const char* omse_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OMSE_H */

@@ -1,0 +1,160 @@
+"""Thin ctypes binding of the C interface in include/omse.h.
+
+Argument marshalling only: every step of the method runs in the CUDA kernels of libomse.so.
+PyTorch supplies device memory and the stream; tensors are passed as raw device pointers.
+The library must be present (build it with paper_1902_06822_b200.build.build()); there is no
+fallback of any kind.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+from . import build as _build
+
+OK, EINVAL, ECUDA, ENOMEM = 0, -1, -2, -3
+DEV_NONFINITE, DEV_DEGENERATE = 1, 2
+MAX_CANDIDATES, MAX_KERNEL_LEN, MAX_KERNEL_LEN_MULTISWEEP, MAX_TENSORS = 4096, 28672, 25600, 4
+
+EXPORTS = [
+    "omse_create", "omse_destroy", "omse_set_stream", "omse_workspace_bytes", "omse_quantize_weights",
+    "omse_activation_scale", "omse_residual_quantize", "omse_pack_int4", "omse_last_device_status",
+    "omse_status_string",
+]
+
+
+class OmseGrid(C.Structure):
+    _fields_ = [("n_cand", C.c_int32), ("hi_frac", C.c_float), ("refine_iters", C.c_int32)]
+
+
+class OmseError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: {status_string(code)} ({code})")
+        self.code = code
+
+
+_lib = None
+
+
+def load_library() -> C.CDLL:
+    """dlopen libomse.so and declare the prototypes; raises if the library has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_build.LIB_PATH):
+        raise FileNotFoundError(f"{_build.LIB_PATH} is missing: run paper_1902_06822_b200.build.build() first")
+    lib = C.CDLL(_build.LIB_PATH)
+    vp, i64, i32 = C.c_void_p, C.c_int64, C.c_int
+    lib.omse_create.argtypes = [C.POINTER(vp), i32, vp]
+    lib.omse_destroy.argtypes = [vp]
+    lib.omse_set_stream.argtypes = [vp, vp]
+    lib.omse_workspace_bytes.argtypes = [vp]
+    lib.omse_workspace_bytes.restype = C.c_size_t
+    lib.omse_quantize_weights.argtypes = [vp, vp, i64, i64, i32, i32, C.POINTER(OmseGrid), vp, vp, vp, vp, vp]
+    lib.omse_activation_scale.argtypes = [vp, vp, i64, i32, i32, C.POINTER(OmseGrid), vp, vp, vp, vp]
+    lib.omse_residual_quantize.argtypes = [vp, vp, i64, i64, C.POINTER(C.c_int), i32, C.POINTER(OmseGrid), i32, i32,
+                                           vp, vp, vp, vp]
+    lib.omse_pack_int4.argtypes = [vp, vp, i64, i32, vp]
+    lib.omse_last_device_status.argtypes = [vp, C.POINTER(C.c_uint32)]
+    lib.omse_status_string.argtypes = [i32]
+    lib.omse_status_string.restype = C.c_char_p
+    for name in EXPORTS:
+        if getattr(lib, name).restype is None:
+            pass
+    _lib = lib
+    return lib
+
+
+def status_string(code: int) -> str:
+    return load_library().omse_status_string(code).decode()
+
+
+def _ptr(t: torch.Tensor | None, dtype: torch.dtype | None = None):
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous CUDA tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"expected dtype {dtype}, got {t.dtype}")
+    return C.c_void_p(t.data_ptr())
+
+
+class Context:
+    """An omse_ctx bound to a device and to the torch stream that is current at construction."""
+
+    def __init__(self, device: int | torch.device = 0, stream: torch.cuda.Stream | None = None):
+        lib = load_library()
+        dev = torch.device(device) if not isinstance(device, int) else torch.device("cuda", device)
+        self.device = dev
+        self._stream = stream if stream is not None else torch.cuda.current_stream(dev)
+        h = C.c_void_p()
+        rc = lib.omse_create(C.byref(h), dev.index or 0, C.c_void_p(self._stream.cuda_stream))
+        if rc != OK:
+            raise OmseError(rc, "omse_create")
+        self._h = h
+
+    def close(self):
+        if getattr(self, "_h", None):
+            load_library().omse_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def set_stream(self, stream: torch.cuda.Stream):
+        self._stream = stream
+        rc = load_library().omse_set_stream(self._h, C.c_void_p(stream.cuda_stream))
+        if rc != OK:
+            raise OmseError(rc, "omse_set_stream")
+
+    @property
+    def workspace_bytes(self) -> int:
+        return int(load_library().omse_workspace_bytes(self._h))
+
+    # -- the four calls of the library --------------------------------------------------------
+    def omse_quantize_weights(self, w, n_kernels, kernel_len, bits, is_signed, n_cand, hi_frac, refine_iters,
+                              alpha, sse, best_idx=None, codes=None, packed=None):
+        g = OmseGrid(n_cand, hi_frac, refine_iters)
+        rc = load_library().omse_quantize_weights(
+            self._h, _ptr(w, torch.float32), n_kernels, kernel_len, bits, int(is_signed), C.byref(g),
+            _ptr(alpha, torch.float32), _ptr(sse, torch.float32), _ptr(best_idx, torch.int32),
+            _ptr(codes, torch.int8), _ptr(packed, torch.uint8))
+        if rc != OK:
+            raise OmseError(rc, "omse_quantize_weights")
+
+    def omse_activation_scale(self, x, n, bits, is_signed, n_cand, hi_frac, refine_iters, alpha, sse,
+                              best_idx=None, sse_curve=None):
+        g = OmseGrid(n_cand, hi_frac, refine_iters)
+        rc = load_library().omse_activation_scale(
+            self._h, _ptr(x, torch.float32), n, bits, int(is_signed), C.byref(g), _ptr(alpha, torch.float32),
+            _ptr(sse, torch.float32), _ptr(best_idx, torch.int32), _ptr(sse_curve, torch.float64))
+        if rc != OK:
+            raise OmseError(rc, "omse_activation_scale")
+
+    def omse_residual_quantize(self, t, n_kernels, kernel_len, bits, is_signed, n_cand, hi_frac, refine_iters,
+                               n_sweeps, alpha, sse, codes=None, packed=None):
+        g = OmseGrid(n_cand, hi_frac, refine_iters)
+        b = (C.c_int * len(bits))(*bits)
+        rc = load_library().omse_residual_quantize(
+            self._h, _ptr(t, torch.float32), n_kernels, kernel_len, b, int(is_signed), C.byref(g), len(bits),
+            n_sweeps, _ptr(alpha, torch.float32), _ptr(sse, torch.float32), _ptr(codes, torch.int8),
+            _ptr(packed, torch.uint8))
+        if rc != OK:
+            raise OmseError(rc, "omse_residual_quantize")
+
+    def omse_pack_int4(self, codes, n, is_signed, packed):
+        rc = load_library().omse_pack_int4(self._h, _ptr(codes, torch.int8), n, int(is_signed), _ptr(packed, torch.uint8))
+        if rc != OK:
+            raise OmseError(rc, "omse_pack_int4")
+
+    def omse_last_device_status(self) -> int:
+        out = C.c_uint32(0)
+        rc = load_library().omse_last_device_status(self._h, C.byref(out))
+        if rc != OK:
+            raise OmseError(rc, "omse_last_device_status")
+        return out.value

@@ -1,0 +1,335 @@
+// Host side of the C interface declared in include/omse.h: argument checks, launch shapes, context.
+// Every step of the method runs in the kernels of omse_rows.cuh / omse_tensor.cuh; there is no
+// host arithmetic on tensor data and no CPU fallback.
+#include "../../include/omse.h"
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "omse_rows.cuh"
+#include "omse_tensor.cuh"
+
+namespace {
+
+constexpr size_t kPartialBytes = 16u << 20;   // per-block partial sums of the per-tensor search
+constexpr int kMaxSmem = 232448;              // 227 KB opt-in limit per block on sm_100
+
+struct Workspace {
+    unsigned int status;
+    unsigned int pad_[3];
+    omse::TensorState tstate;
+    double curve[OMSE_MAX_CANDIDATES];
+};
+
+}  // namespace
+
+struct omse_ctx {
+    int device;
+    cudaStream_t stream;
+    int n_sm;
+    Workspace* ws;       // device
+    double* partials;    // device, kPartialBytes
+};
+
+namespace {
+
+int cpt_for(int n_cand) { return n_cand <= 32 ? 1 : n_cand <= 64 ? 2 : n_cand <= 128 ? 4 : 8; }
+
+bool grid_ok(const omse_grid* g) {
+    return g && g->n_cand >= 1 && g->n_cand <= OMSE_MAX_CANDIDATES && g->hi_frac > 0.f &&
+           g->hi_frac <= 3.0e38f && g->refine_iters >= 0 && g->refine_iters <= 64;
+}
+
+void bounds(int bits, int is_signed, int* lo, int* hi) {
+    if (is_signed) {
+        *lo = -(1 << (bits - 1));
+        *hi = (1 << (bits - 1)) - 1;
+    } else {
+        *lo = 0;
+        *hi = (1 << bits) - 1;
+    }
+}
+
+template <int CPT>
+int launch_rows_t(omse_ctx* ctx, omse::RowArgs& a, size_t smem) {
+    static bool attr_set[64] = {};
+    if (!attr_set[ctx->device & 63]) {
+        if (cudaFuncSetAttribute(omse::rows_kernel<CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess)
+            return OMSE_ECUDA;
+        attr_set[ctx->device & 63] = true;
+    }
+    const int threads = a.groups * a.tg;
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, omse::rows_kernel<CPT>, threads, smem) != cudaSuccess || occ < 1)
+        return OMSE_ECUDA;
+    const long long n_units = (a.S + a.rows_per_unit - 1) / a.rows_per_unit;
+    long long grid = (long long)ctx->n_sm * occ;
+    if (grid > n_units) grid = n_units;
+    omse::rows_kernel<CPT><<<(unsigned)grid, threads, smem, ctx->stream>>>(a);
+    return cudaGetLastError() == cudaSuccess ? OMSE_OK : OMSE_ECUDA;
+}
+
+int launch_rows(omse_ctx* ctx, omse::RowArgs& a) {
+    const int cpt = cpt_for(a.n_cand);
+    a.tg = (((a.n_cand + cpt - 1) / cpt) + 31) & ~31;
+    const int k4 = (int)((a.K + 3) >> 2);
+    int target = a.K >= 8192 ? 512 : a.K >= 512 ? 256 : 128;
+    int groups = target / a.tg;
+    if (groups > k4 / 8) groups = k4 / 8;
+    if (groups < 1) groups = 1;
+    a.groups = groups;
+    auto smem_for = [&](int gr) {
+        return (size_t)(a.keep_x0 ? 2 : 1) * k4 * 16 + (size_t)(gr - 1) * cpt * a.tg * 8 + 64 * 8 + omse::kListCap * 4 + 8 * 4;
+    };
+    while (a.groups > 1 && smem_for(a.groups) > (size_t)kMaxSmem) a.groups >>= 1;
+    const size_t smem = smem_for(a.groups);
+    if (smem > (size_t)kMaxSmem) return OMSE_EINVAL;
+    switch (cpt) {
+        case 1: return launch_rows_t<1>(ctx, a, smem);
+        case 2: return launch_rows_t<2>(ctx, a, smem);
+        case 4: return launch_rows_t<4>(ctx, a, smem);
+        default: return launch_rows_t<8>(ctx, a, smem);
+    }
+}
+
+template <int CPT>
+int launch_tensor_sweep_t(omse_ctx* ctx, omse::TensorArgs& a, size_t smem, int* n_blocks) {
+    static bool attr_set[64] = {};
+    if (!attr_set[ctx->device & 63]) {
+        if (cudaFuncSetAttribute(omse::tensor_sweep_kernel<CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess)
+            return OMSE_ECUDA;
+        attr_set[ctx->device & 63] = true;
+    }
+    const int threads = a.groups * a.tg;
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, omse::tensor_sweep_kernel<CPT>, threads, smem) != cudaSuccess || occ < 1)
+        return OMSE_ECUDA;
+    const long long n4 = (a.n + 3) >> 2;
+    const long long n_tiles = (n4 + a.tile4 - 1) / a.tile4;
+    long long grid = (long long)ctx->n_sm * occ;
+    const long long cap = (long long)(kPartialBytes / ((size_t)a.n_cand * 8));
+    if (grid > cap) grid = cap;
+    if (grid > n_tiles) grid = n_tiles;
+    if (grid < 1) grid = 1;
+    *n_blocks = (int)grid;
+    omse::tensor_sweep_kernel<CPT><<<(unsigned)grid, threads, smem, ctx->stream>>>(a);
+    return cudaGetLastError() == cudaSuccess ? OMSE_OK : OMSE_ECUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* omse_status_string(int status) {
+    switch (status) {
+        case OMSE_OK: return "ok";
+        case OMSE_EINVAL: return "invalid argument";
+        case OMSE_ECUDA: return "CUDA runtime or launch failure";
+        case OMSE_ENOMEM: return "out of device memory";
+        default: return "unknown status";
+    }
+}
+
+int omse_create(omse_ctx** out, int device, void* cuda_stream) {
+    if (!out) return OMSE_EINVAL;
+    *out = nullptr;
+    int n_dev = 0;
+    if (cudaGetDeviceCount(&n_dev) != cudaSuccess || device < 0 || device >= n_dev) return OMSE_ECUDA;
+    if (cudaSetDevice(device) != cudaSuccess) return OMSE_ECUDA;
+    omse_ctx* c = new (std::nothrow) omse_ctx;
+    if (!c) return OMSE_ENOMEM;
+    c->device = device;
+    c->stream = static_cast<cudaStream_t>(cuda_stream);
+    c->ws = nullptr;
+    c->partials = nullptr;
+    if (cudaDeviceGetAttribute(&c->n_sm, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
+        delete c;
+        return OMSE_ECUDA;
+    }
+    if (cudaMalloc(&c->ws, sizeof(Workspace)) != cudaSuccess || cudaMalloc(&c->partials, kPartialBytes) != cudaSuccess) {
+        cudaFree(c->ws);
+        delete c;
+        cudaGetLastError();
+        return OMSE_ENOMEM;
+    }
+    if (cudaMemsetAsync(c->ws, 0, sizeof(Workspace), c->stream) != cudaSuccess) {
+        cudaFree(c->ws);
+        cudaFree(c->partials);
+        delete c;
+        return OMSE_ECUDA;
+    }
+    *out = c;
+    return OMSE_OK;
+}
+
+int omse_destroy(omse_ctx* ctx) {
+    if (!ctx) return OMSE_EINVAL;
+    cudaSetDevice(ctx->device);
+    cudaStreamSynchronize(ctx->stream);
+    cudaFree(ctx->ws);
+    cudaFree(ctx->partials);
+    delete ctx;
+    return OMSE_OK;
+}
+
+int omse_set_stream(omse_ctx* ctx, void* cuda_stream) {
+    if (!ctx) return OMSE_EINVAL;
+    ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+    return OMSE_OK;
+}
+
+size_t omse_workspace_bytes(const omse_ctx* ctx) { return ctx ? sizeof(Workspace) + kPartialBytes : 0; }
+
+int omse_last_device_status(omse_ctx* ctx, uint32_t* host_out) {
+    if (!ctx || !host_out) return OMSE_EINVAL;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return OMSE_ECUDA;
+    if (cudaMemcpyAsync(host_out, &ctx->ws->status, sizeof(uint32_t), cudaMemcpyDeviceToHost, ctx->stream) != cudaSuccess)
+        return OMSE_ECUDA;
+    if (cudaMemsetAsync(&ctx->ws->status, 0, sizeof(uint32_t), ctx->stream) != cudaSuccess) return OMSE_ECUDA;
+    return cudaStreamSynchronize(ctx->stream) == cudaSuccess ? OMSE_OK : OMSE_ECUDA;
+}
+
+int omse_quantize_weights(omse_ctx* ctx, const float* d_w, int64_t n_kernels, int64_t kernel_len, int bits,
+                          int is_signed, const omse_grid* grid, float* d_alpha, float* d_sse,
+                          int32_t* d_best_idx, int8_t* d_codes, uint8_t* d_packed) {
+    if (!ctx || !grid_ok(grid) || bits < 2 || bits > 8 || n_kernels < 0 || kernel_len < 1 ||
+        kernel_len > OMSE_MAX_KERNEL_LEN || n_kernels > (int64_t)1 << 40)
+        return OMSE_EINVAL;
+    if (d_packed && bits > 4) return OMSE_EINVAL;
+    if (n_kernels == 0) return OMSE_OK;
+    if (!d_w || !d_alpha || !d_sse) return OMSE_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(d_w) & 3) || (reinterpret_cast<uintptr_t>(d_alpha) & 3) ||
+        (reinterpret_cast<uintptr_t>(d_sse) & 3) || (reinterpret_cast<uintptr_t>(d_best_idx) & 3))
+        return OMSE_EINVAL;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return OMSE_ECUDA;
+    omse::RowArgs a;
+    memset(&a, 0, sizeof(a));
+    a.w = d_w;
+    a.S = n_kernels;
+    a.K = kernel_len;
+    a.n_cand = grid->n_cand;
+    a.hi_frac = grid->hi_frac;
+    a.refine_iters = grid->refine_iters;
+    a.n_tensors = 1;
+    a.n_sweeps = 1;
+    bounds(bits, is_signed, &a.lo[0], &a.hi[0]);
+    a.alpha = d_alpha;
+    a.sse = d_sse;
+    a.best_idx = d_best_idx;
+    a.codes = reinterpret_cast<signed char*>(d_codes);
+    a.packed = d_packed;
+    a.status = &ctx->ws->status;
+    a.rows_per_unit = (d_packed && (kernel_len & 1)) ? 2 : 1;
+    a.keep_x0 = 0;
+    return launch_rows(ctx, a);
+}
+
+int omse_residual_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, int64_t kernel_len, const int* bits,
+                           int is_signed, const omse_grid* grid, int n_tensors, int n_sweeps, float* d_alpha,
+                           float* d_sse, int8_t* d_codes, uint8_t* d_packed) {
+    if (!ctx || !grid_ok(grid) || !bits || n_tensors < 1 || n_tensors > OMSE_MAX_TENSORS || n_sweeps < 1 ||
+        n_sweeps > 64 || n_kernels < 0 || kernel_len < 1 || kernel_len > OMSE_MAX_KERNEL_LEN ||
+        n_kernels > (int64_t)1 << 40)
+        return OMSE_EINVAL;
+    for (int j = 0; j < n_tensors; ++j) {
+        if (bits[j] < 2 || bits[j] > 8) return OMSE_EINVAL;
+        if (d_packed && bits[j] > 4) return OMSE_EINVAL;
+    }
+    if (n_sweeps > 1 && (!d_codes || kernel_len > OMSE_MAX_KERNEL_LEN_MULTISWEEP)) return OMSE_EINVAL;
+    if (n_kernels == 0) return OMSE_OK;
+    if (!d_t || !d_alpha || !d_sse) return OMSE_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(d_t) & 3) || (reinterpret_cast<uintptr_t>(d_alpha) & 3) ||
+        (reinterpret_cast<uintptr_t>(d_sse) & 3))
+        return OMSE_EINVAL;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return OMSE_ECUDA;
+    omse::RowArgs a;
+    memset(&a, 0, sizeof(a));
+    a.w = d_t;
+    a.S = n_kernels;
+    a.K = kernel_len;
+    a.n_cand = grid->n_cand;
+    a.hi_frac = grid->hi_frac;
+    a.refine_iters = grid->refine_iters;
+    a.n_tensors = n_tensors;
+    a.n_sweeps = n_sweeps;
+    for (int j = 0; j < n_tensors; ++j) bounds(bits[j], is_signed, &a.lo[j], &a.hi[j]);
+    a.alpha = d_alpha;
+    a.sse = d_sse;
+    a.best_idx = nullptr;
+    a.codes = reinterpret_cast<signed char*>(d_codes);
+    a.packed = d_packed;
+    a.status = &ctx->ws->status;
+    a.rows_per_unit = (d_packed && (kernel_len & 1)) ? 2 : 1;
+    a.keep_x0 = n_sweeps > 1 ? 1 : 0;
+    return launch_rows(ctx, a);
+}
+
+int omse_activation_scale(omse_ctx* ctx, const float* d_x, int64_t n, int bits, int is_signed, const omse_grid* grid,
+                          float* d_alpha, float* d_sse, int32_t* d_best_idx, double* d_sse_curve) {
+    if (!ctx || !grid_ok(grid) || bits < 2 || bits > 8 || n < 0 || !d_alpha || !d_sse) return OMSE_EINVAL;
+    if (n > 0 && !d_x) return OMSE_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(d_x) & 15) || (reinterpret_cast<uintptr_t>(d_alpha) & 3) ||
+        (reinterpret_cast<uintptr_t>(d_sse) & 3) || (reinterpret_cast<uintptr_t>(d_best_idx) & 3) ||
+        (reinterpret_cast<uintptr_t>(d_sse_curve) & 7))
+        return OMSE_EINVAL;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return OMSE_ECUDA;
+    omse::TensorArgs a;
+    memset(&a, 0, sizeof(a));
+    a.x = d_x;
+    a.n = n;
+    a.n_cand = grid->n_cand;
+    a.hi_frac = grid->hi_frac;
+    bounds(bits, is_signed, &a.lo, &a.hi);
+    const int cpt = cpt_for(a.n_cand);
+    a.tg = (((a.n_cand + cpt - 1) / cpt) + 31) & ~31;
+    a.groups = 256 / a.tg < 1 ? 1 : 256 / a.tg;
+    a.tile4 = 1024;
+    a.st = &ctx->ws->tstate;
+    a.partials = ctx->partials;
+    a.curve = ctx->ws->curve;
+    a.curve_out = d_sse_curve;
+    a.alpha_out = d_alpha;
+    a.sse_out = d_sse;
+    a.idx_out = d_best_idx;
+    a.status = &ctx->ws->status;
+    cudaStream_t s = ctx->stream;
+
+    omse::tensor_init_kernel<<<1, 32, 0, s>>>(a.st);
+    long long pass_grid = (n + 1023) / 1024;
+    if (pass_grid > (long long)ctx->n_sm * 8) pass_grid = (long long)ctx->n_sm * 8;
+    if (pass_grid < 1) pass_grid = 1;
+    int n_blocks = 1;
+    if (n > 0) {
+        omse::tensor_absmax_kernel<<<(unsigned)pass_grid, 256, 0, s>>>(d_x, n, a.st, a.status);
+        const size_t smem = (size_t)a.tile4 * 16 + (size_t)(a.groups - 1) * cpt * a.tg * 8;
+        int rc;
+        switch (cpt) {
+            case 1: rc = launch_tensor_sweep_t<1>(ctx, a, smem, &n_blocks); break;
+            case 2: rc = launch_tensor_sweep_t<2>(ctx, a, smem, &n_blocks); break;
+            case 4: rc = launch_tensor_sweep_t<4>(ctx, a, smem, &n_blocks); break;
+            default: rc = launch_tensor_sweep_t<8>(ctx, a, smem, &n_blocks); break;
+        }
+        if (rc != OMSE_OK) return rc;
+    }
+    omse::tensor_finish_kernel<<<1, 1024, 0, s>>>(a, n_blocks);
+    omse::tensor_pass_kernel<0><<<(unsigned)pass_grid, 256, 0, s>>>(a);
+    for (int it = 0; it < grid->refine_iters; ++it) omse::tensor_pass_kernel<1><<<(unsigned)pass_grid, 256, 0, s>>>(a);
+    omse::tensor_pass_kernel<2><<<(unsigned)pass_grid, 256, 0, s>>>(a);
+    return cudaGetLastError() == cudaSuccess ? OMSE_OK : OMSE_ECUDA;
+}
+
+int omse_pack_int4(omse_ctx* ctx, const int8_t* d_codes, int64_t n, int is_signed, uint8_t* d_packed) {
+    (void)is_signed;
+    if (!ctx || n < 0) return OMSE_EINVAL;
+    if (n == 0) return OMSE_OK;
+    if (!d_codes || !d_packed) return OMSE_EINVAL;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return OMSE_ECUDA;
+    long long grid = (n / 16 + 255) / 256;
+    if (grid > (long long)ctx->n_sm * 16) grid = (long long)ctx->n_sm * 16;
+    if (grid < 1) grid = 1;
+    omse::pack_int4_kernel<<<(unsigned)grid, 256, 0, ctx->stream>>>(reinterpret_cast<const signed char*>(d_codes), n, d_packed);
+    return cudaGetLastError() == cudaSuccess ? OMSE_OK : OMSE_ECUDA;
+}
+
+}  // extern "C"

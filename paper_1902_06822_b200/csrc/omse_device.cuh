@@ -1,0 +1,247 @@
+// Device-side building blocks of the MMSE scale search for sm_100a.
+//
+// Section 3.4 of the paper reduces the constrained MSE problem to a one-dimensional search over the
+// scale alpha, the codes being [T_i/alpha]_Zp.  The search evaluates the squared error at every
+// point of a grid of scales.  Here the tensor (one kernel, or a tile of an activation tensor) sits
+// in shared memory, every thread owns a few candidate scales in registers, and all threads stream
+// the same elements (shared-memory broadcast), so the inner loop is pure FP32 arithmetic:
+//     t = x*inv_alpha + M       (M = 1.5*2^23: the add rounds to the nearest integer, ties to even)
+//     t = min(max(t, M+lo), M+hi)            only for candidates that can saturate on this tensor
+//     q = t - M ;  e = x - alpha*q ;  acc += e*e
+// written with Blackwell's packed fma.rn.f32x2 / add.rn.f32x2 on two elements at a time.
+#pragma once
+#include <cfloat>
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace omse {
+
+typedef unsigned long long u64;
+
+constexpr float kMagic = 12582912.0f;   // 1.5 * 2^23
+constexpr int kFlushEvery4 = 32;        // float4 loads between folds of the fp32 partial sums into fp64
+constexpr int kListCap = 32;            // most near-minimal candidates re-scored in fp64
+constexpr double kRescoreBand = 4e-6;   // candidates within this relative band of the fp32 minimum are re-scored
+
+__device__ __forceinline__ u64 pack2(float a, float b) {
+    u64 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ void unpack2(u64 v, float& a, float& b) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ u64 fma2(u64 a, u64 b, u64 c) {
+    u64 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ u64 add2(u64 a, u64 b) {
+    u64 d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
+// [x/alpha]_Zp exactly as Section 3.1 writes it: IEEE division, round to nearest even, saturate.
+__device__ __forceinline__ int code_of(float x, float alpha, float flo, float fhi) {
+    float r = rintf(__fdiv_rn(x, alpha));
+    r = fminf(fmaxf(r, flo), fhi);
+    return (int)r;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Candidate sweep over float4 indices [beg4, end4) of a shared-memory span.  CPT candidates per
+// thread; the first NCL of them are evaluated with saturation, the rest without.
+// acc2 holds two fp32 partial sums per candidate (even / odd element of each pair); every
+// kFlushEvery4 loads they are folded into the fp64 accumulators so that the rounding noise of the
+// fp32 sums stays near 1e-7 relative whatever the span length.
+// ---------------------------------------------------------------------------------------------
+template <int CPT, int NCL>
+__device__ __forceinline__ void sweep_range(const float4* __restrict__ xs4, int beg4, int end4,
+                                            const u64 (&inv2)[CPT], const u64 (&na2)[CPT],
+                                            double (&dacc)[CPT], float clo, float chi) {
+    const u64 M2 = pack2(kMagic, kMagic);
+    const u64 NM2 = pack2(-kMagic, -kMagic);
+    u64 acc2[CPT];
+#pragma unroll
+    for (int s = 0; s < CPT; ++s) acc2[s] = 0ull;
+    int i = beg4;
+    while (i < end4) {
+        const int stop = min(end4, i + kFlushEvery4);
+#pragma unroll 2
+        for (; i < stop; ++i) {
+            const float4 v = xs4[i];
+            const u64 xa = pack2(v.x, v.y), xb = pack2(v.z, v.w);
+#pragma unroll
+            for (int s = 0; s < CPT; ++s) {
+                u64 ta = fma2(xa, inv2[s], M2);
+                u64 tb = fma2(xb, inv2[s], M2);
+                if (s < NCL) {
+                    float a0, a1, b0, b1;
+                    unpack2(ta, a0, a1);
+                    unpack2(tb, b0, b1);
+                    a0 = fminf(fmaxf(a0, clo), chi);
+                    a1 = fminf(fmaxf(a1, clo), chi);
+                    b0 = fminf(fmaxf(b0, clo), chi);
+                    b1 = fminf(fmaxf(b1, clo), chi);
+                    ta = pack2(a0, a1);
+                    tb = pack2(b0, b1);
+                }
+                const u64 qa = add2(ta, NM2);
+                const u64 qb = add2(tb, NM2);
+                const u64 ea = fma2(na2[s], qa, xa);
+                const u64 eb = fma2(na2[s], qb, xb);
+                acc2[s] = fma2(ea, ea, acc2[s]);
+                acc2[s] = fma2(eb, eb, acc2[s]);
+            }
+        }
+#pragma unroll
+        for (int s = 0; s < CPT; ++s) {
+            float p0, p1;
+            unpack2(acc2[s], p0, p1);
+            dacc[s] += (double)(p0 + p1);
+            acc2[s] = 0ull;
+        }
+    }
+}
+
+// Dispatch on the (warp-uniform) number of leading candidates per thread that need saturation.
+template <int CPT>
+__device__ __forceinline__ void sweep_dispatch(int ncl, const float4* xs4, int beg4, int end4,
+                                               const u64 (&inv2)[CPT], const u64 (&na2)[CPT],
+                                               double (&dacc)[CPT], float clo, float chi) {
+    if (ncl <= 0) {
+        sweep_range<CPT, 0>(xs4, beg4, end4, inv2, na2, dacc, clo, chi);
+    } else if (ncl == 1) {
+        sweep_range<CPT, 1>(xs4, beg4, end4, inv2, na2, dacc, clo, chi);
+    } else if (ncl == 2 && CPT > 2) {
+        sweep_range<CPT, (CPT > 2 ? 2 : CPT)>(xs4, beg4, end4, inv2, na2, dacc, clo, chi);
+    } else if (ncl <= CPT / 2 && CPT > 4) {
+        sweep_range<CPT, CPT / 2>(xs4, beg4, end4, inv2, na2, dacc, clo, chi);
+    } else {
+        sweep_range<CPT, CPT>(xs4, beg4, end4, inv2, na2, dacc, clo, chi);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Block-wide reductions (fixed order: lanes by shuffle tree, warps in index order) so that results
+// do not depend on scheduling.  `scratch` holds at least 2*32 doubles.  All threads get the result.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ long long warp_sum(long long v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// sums a double and a 64-bit integer over the block
+__device__ __forceinline__ void block_sum2(double& d, long long& q, double* scratch) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = (blockDim.x + 31) >> 5;
+    d = warp_sum(d);
+    q = warp_sum(q);
+    long long* qs = reinterpret_cast<long long*>(scratch + 32);
+    __syncthreads();
+    if (lane == 0) {
+        scratch[warp] = d;
+        qs[warp] = q;
+    }
+    __syncthreads();
+    double dt = 0.0;
+    long long qt = 0;
+    for (int w = 0; w < nwarp; ++w) {
+        dt += scratch[w];
+        qt += qs[w];
+    }
+    d = dt;
+    q = qt;
+}
+
+__device__ __forceinline__ void block_max2(float& a, float& b, double* scratch) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = (blockDim.x + 31) >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        a = fmaxf(a, __shfl_down_sync(0xffffffffu, a, o));
+        b = fmaxf(b, __shfl_down_sync(0xffffffffu, b, o));
+    }
+    float* fs = reinterpret_cast<float*>(scratch);
+    __syncthreads();
+    if (lane == 0) {
+        fs[warp] = a;
+        fs[32 + warp] = b;
+    }
+    __syncthreads();
+    float ta = 0.f, tb = 0.f;
+    for (int w = 0; w < nwarp; ++w) {
+        ta = fmaxf(ta, fs[w]);
+        tb = fmaxf(tb, fs[32 + w]);
+    }
+    a = ta;
+    b = tb;
+}
+
+// lexicographic minimum of (value, index) over the block
+__device__ __forceinline__ void block_argmin(double& v, int& idx, double* scratch) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = (blockDim.x + 31) >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const double ov = __shfl_down_sync(0xffffffffu, v, o);
+        const int oi = __shfl_down_sync(0xffffffffu, idx, o);
+        if (ov < v || (ov == v && oi < idx)) {
+            v = ov;
+            idx = oi;
+        }
+    }
+    int* is = reinterpret_cast<int*>(scratch + 32);
+    __syncthreads();
+    if (lane == 0) {
+        scratch[warp] = v;
+        is[warp] = idx;
+    }
+    __syncthreads();
+    double bv = scratch[0];
+    int bi = is[0];
+    for (int w = 1; w < nwarp; ++w) {
+        const double ov = scratch[w];
+        const int oi = is[w];
+        if (ov < bv || (ov == bv && oi < bi)) {
+            bv = ov;
+            bi = oi;
+        }
+    }
+    v = bv;
+    idx = bi;
+}
+
+// Per-candidate constants of one thread for the grid of Section 3.4 on a tensor with max|x| = m.
+// Candidate c has alpha_c = fl(fl(c+1)*step), step = fl(fl(hi_frac*m)/fl(C)), all binary32.
+// In the sweep x/alpha_c is replaced by x*inv_c with inv_c within 2 ulp of 1/alpha_c: a code can
+// differ from the divided one only where both neighbours give the same error to ~1e-7, and the
+// winners are re-scored with true division afterwards.
+struct GridSetup {
+    float step;      // alpha step
+    float rstep;     // ~1/step
+    bool tiny;       // step so small that 1/step may overflow: use per-candidate division
+    int c_sat;       // candidates with index < c_sat may saturate on this tensor
+};
+
+__device__ __forceinline__ GridSetup grid_setup(float mpos, float mneg, float hi_frac, int n_cand,
+                                                float flo, float fhi) {
+    GridSetup g;
+    const float m = fmaxf(mpos, mneg);
+    const float a_hi = __fmul_rn(hi_frac, m);
+    g.step = __fdiv_rn(a_hi, (float)n_cand);
+    g.tiny = !(g.step > 1e-30f);
+    g.rstep = g.tiny ? 0.f : __fdiv_rn(1.0f, g.step);
+    // x*inv_c stays strictly below hi+1/2 (and above lo-1/2) for every x once
+    // c+1 > max(mpos/(hi+1/2), mneg/(1/2-lo)) / step; 1e-5 covers the rounding of inv_c and alpha_c.
+    const float need = fmaxf(mpos / (fhi + 0.5f), mneg / (0.5f - flo));
+    const float cs = g.tiny ? (float)n_cand : need * g.rstep * 1.00001f + 1.0f;
+    g.c_sat = cs >= (float)n_cand ? n_cand : (int)cs;
+    return g;
+}
+
+}  // namespace omse

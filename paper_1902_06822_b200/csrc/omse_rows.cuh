@@ -1,0 +1,353 @@
+// Kernel-wise MMSE quantization (Sections 3.3, 3.4) and Algorithm 1 (Section 3.5): one thread block
+// owns one kernel (row) at a time, staged once from HBM into shared memory; everything that follows
+// (max, candidate sweep, argmin, polish, codes, packing, residual update) reads the on-chip copy.
+#pragma once
+#include "omse_device.cuh"
+
+namespace omse {
+
+struct RowArgs {
+    const float* w;        // [S][K]
+    long long S, K;
+    int n_cand;
+    float hi_frac;
+    int refine_iters;
+    int n_tensors, n_sweeps;
+    int lo[4], hi[4];      // grid bounds per tensor (Section 3.1)
+    float* alpha;          // [n_tensors][S]
+    float* sse;            // [n_tensors][S]
+    int* best_idx;         // [S] (single tensor only), nullable
+    signed char* codes;    // [n_tensors][N], nullable
+    unsigned char* packed; // [n_tensors][ceil(N/2)], nullable
+    unsigned int* status;
+    int groups;            // element groups per block
+    int tg;                // threads per group (multiple of 32); candidate c = slot*tg + t
+    int rows_per_unit;     // 2 when nibble packing needs an even element count per unit (odd K)
+    int keep_x0;           // n_sweeps > 1: keep the original row next to the residual
+};
+
+struct PhiOut {
+    float alpha;
+    double sse;
+    int idx;
+    bool degenerate;
+};
+
+// shared-memory carve-up for one block
+struct RowSmem {
+    float* xs;        // [k4*4] current tensor (row or residual), zero padded to a multiple of 4
+    float* x0;        // [k4*4] original row (only when keep_x0)
+    double* xg;       // [(groups-1)*CPT*tg] partial sums of the other element groups
+    double* scratch;  // [64] reductions
+    int* list;        // [kListCap] near-minimal candidates
+    int* misc;        // [8]: 0 list count; 1..4 nibble carried to the next row, per tensor
+};
+
+// The quantization mapping phi of Section 3.4 on the row held in s.xs (k elements, k4 float4s).
+template <int CPT>
+__device__ PhiOut phi_block(const RowArgs& a, const RowSmem& s, int k, int k4, float flo, float fhi) {
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    const int grp = tid / a.tg, t = tid - grp * a.tg;
+    const float4* xs4 = reinterpret_cast<const float4*>(s.xs);
+    PhiOut out;
+
+    // ---- max of the positive and of the negative part (range of the grid; which candidates saturate)
+    float mpos = 0.f, mneg = 0.f;
+    for (int i = tid; i < k; i += nthr) {
+        const float v = s.xs[i];
+        if (fabsf(v) <= FLT_MAX) {
+            mpos = fmaxf(mpos, v);
+            mneg = fmaxf(mneg, -v);
+        }
+    }
+    block_max2(mpos, mneg, s.scratch);
+    const float m = fmaxf(mpos, mneg);
+    const GridSetup g = grid_setup(mpos, mneg, a.hi_frac, a.n_cand, flo, fhi);
+    const float a_last = __fmul_rn((float)a.n_cand, g.step);
+    out.alpha = 0.f;
+    out.sse = 0.0;
+    out.idx = -1;
+    out.degenerate = true;
+    if (!(m > 0.f) || !(a_last >= FLT_MIN)) return out;   // no usable scale: alpha = 0, all codes 0
+
+    // ---- per-thread candidate constants
+    u64 inv2[CPT], na2[CPT];
+    double dacc[CPT];
+#pragma unroll
+    for (int sl = 0; sl < CPT; ++sl) {
+        const int c = sl * a.tg + t;
+        const float ac = __fmul_rn((float)(c + 1), g.step);
+        float inv = g.tiny ? __fdiv_rn(1.0f, ac) : __fdiv_rn(1.0f, (float)(c + 1)) * g.rstep;
+        if (!(ac >= FLT_MIN) || c >= a.n_cand) inv = 0.f;  // unusable: evaluated harmlessly, discarded below
+        inv2[sl] = pack2(inv, inv);
+        na2[sl] = pack2(-ac, -ac);
+        dacc[sl] = 0.0;
+    }
+    const int warp_t0 = t & ~31;
+    int ncl = (g.c_sat - warp_t0 + a.tg - 1) / a.tg;
+    ncl = max(0, min(CPT, ncl));
+
+    // ---- sweep: this group's contiguous share of the row, all candidates
+    const int beg4 = (int)(((long long)k4 * grp) / a.groups);
+    const int end4 = (int)(((long long)k4 * (grp + 1)) / a.groups);
+    sweep_dispatch<CPT>(ncl, xs4, beg4, end4, inv2, na2, dacc, kMagic + flo, kMagic + fhi);
+
+    if (a.groups > 1) {
+        if (grp > 0) {
+#pragma unroll
+            for (int sl = 0; sl < CPT; ++sl) s.xg[((grp - 1) * CPT + sl) * a.tg + t] = dacc[sl];
+        }
+        __syncthreads();
+        if (grp == 0) {
+            for (int gg = 1; gg < a.groups; ++gg)
+#pragma unroll
+                for (int sl = 0; sl < CPT; ++sl) dacc[sl] += s.xg[((gg - 1) * CPT + sl) * a.tg + t];
+        }
+    }
+
+    // ---- argmin over candidates (fp32-block / fp64-fold sums), lowest index on ties
+    double bv = INFINITY;
+    int bi = 0x7fffffff;
+#pragma unroll
+    for (int sl = 0; sl < CPT; ++sl) {
+        const int c = sl * a.tg + t;
+        const float ac = __fmul_rn((float)(c + 1), g.step);
+        const bool ok = grp == 0 && c < a.n_cand && ac >= FLT_MIN;
+        dacc[sl] = ok ? dacc[sl] : INFINITY;
+        if (dacc[sl] < bv) {   // slots are in increasing c, strict < keeps the lowest index
+            bv = dacc[sl];
+            bi = c;
+        }
+    }
+    if (tid == 0) s.misc[0] = 0;
+    block_argmin(bv, bi, s.scratch);   // contains __syncthreads: the zeroed counter is visible after it
+    if (bi == 0x7fffffff) return out;  // every error is Inf/NaN (non-finite input): same as no usable scale
+    out.degenerate = false;
+
+    // ---- candidates within the fp32 noise band of the minimum are re-scored in fp64 with true division
+    const double band = bv * (1.0 + kRescoreBand);
+#pragma unroll
+    for (int sl = 0; sl < CPT; ++sl) {
+        if (dacc[sl] <= band) {
+            const int pos = atomicAdd(&s.misc[0], 1);
+            if (pos < kListCap) s.list[pos] = sl * a.tg + t;
+        }
+    }
+    __syncthreads();
+    const int n_list = s.misc[0];
+    int best = bi;
+    if (n_list > 1 && n_list <= kListCap) {
+        double best_sse = INFINITY;
+        best = 0x7fffffff;
+        for (int l = 0; l < n_list; ++l) {
+            const int c = s.list[l];
+            const float ac = __fmul_rn((float)(c + 1), g.step);
+            double ss = 0.0;
+            long long zero = 0;
+            for (int i = tid; i < k; i += nthr) {
+                const float x = s.xs[i];
+                const double d = (double)x - (double)ac * (double)code_of(x, ac, flo, fhi);
+                ss += d * d;
+            }
+            block_sum2(ss, zero, s.scratch);
+            if (ss < best_sse || (ss == best_sse && c < best)) {
+                best_sse = ss;
+                best = c;
+            }
+        }
+    }
+
+    // ---- polish: alpha <- <x,q>/<q,q>, q = [x/alpha]_Zp, refine_iters times
+    float alpha = __fmul_rn((float)(best + 1), g.step);
+    for (int it = 0; it < a.refine_iters; ++it) {
+        double sxq = 0.0;
+        long long sqq = 0;
+        for (int i = tid; i < k; i += nthr) {
+            const float x = s.xs[i];
+            const int q = code_of(x, alpha, flo, fhi);
+            sqq += q * q;
+            sxq += (double)x * (double)q;
+        }
+        block_sum2(sxq, sqq, s.scratch);
+        if (sqq == 0) break;
+        const float a_new = (float)(sxq / (double)sqq);
+        if (!(a_new >= FLT_MIN) || !(a_new <= FLT_MAX)) break;
+        alpha = a_new;
+    }
+    out.alpha = alpha;
+    out.idx = best;
+    out.sse = 0.0;   // filled by emit_block
+    return out;
+}
+
+// Final codes at `alpha`, their squared error, and emission as int8 and/or nibbles.
+// row_base = flat index of the row's first element in the tensor; n_total = S*K.
+__device__ double emit_block(const RowSmem& s, int k, float alpha, float flo, float fhi,
+                             signed char* codes, unsigned char* packed, long long row_base,
+                             int* carry, bool more_rows_in_unit) {
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    double ss = 0.0;
+    const bool zero = !(alpha > 0.f);
+    const bool aligned = ((reinterpret_cast<unsigned long long>(codes) & 3ull) == 0) &&
+                         ((reinterpret_cast<unsigned long long>(packed) & 1ull) == 0);
+    if ((k & 3) == 0 && aligned) {
+        // aligned fast path: four codes per thread, 32-bit and 16-bit stores
+        const float4* xs4 = reinterpret_cast<const float4*>(s.xs);
+        for (int i4 = tid; i4 < (k >> 2); i4 += nthr) {
+            const float4 v = xs4[i4];
+            const float x[4] = {v.x, v.y, v.z, v.w};
+            int q[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                q[e] = zero ? 0 : code_of(x[e], alpha, flo, fhi);
+                const double d = (double)x[e] - (double)alpha * (double)q[e];
+                ss += d * d;
+            }
+            if (codes) {
+                const unsigned int w = (q[0] & 0xff) | ((q[1] & 0xff) << 8) | ((q[2] & 0xff) << 16) | ((unsigned)(q[3] & 0xff) << 24);
+                *reinterpret_cast<unsigned int*>(codes + row_base + 4ll * i4) = w;
+            }
+            if (packed) {
+                const unsigned short h = (unsigned short)((q[0] & 0xf) | ((q[1] & 0xf) << 4) | ((q[2] & 0xf) << 8) | ((q[3] & 0xf) << 12));
+                *reinterpret_cast<unsigned short*>(packed + ((row_base + 4ll * i4) >> 1)) = h;
+            }
+        }
+    } else {
+        // general path: one output byte (two flat-consecutive elements) per thread; a byte that
+        // straddles two rows is completed by the second row of the unit from the saved nibble
+        const int o = (int)(row_base & 1);
+        const int n_pairs = (k + o + 1) >> 1;
+        for (int p = tid; p < n_pairs; p += nthr) {
+            const int e0 = 2 * p - o, e1 = e0 + 1;
+            int q0 = 0, q1 = 0;
+            if (e0 >= 0) {
+                const float x = s.xs[e0];
+                q0 = zero ? 0 : code_of(x, alpha, flo, fhi);
+                const double d = (double)x - (double)alpha * (double)q0;
+                ss += d * d;
+                if (codes) codes[row_base + e0] = (signed char)q0;
+            } else {
+                q0 = *carry;
+            }
+            const bool has1 = e1 < k;
+            if (has1) {
+                const float x = s.xs[e1];
+                q1 = zero ? 0 : code_of(x, alpha, flo, fhi);
+                const double d = (double)x - (double)alpha * (double)q1;
+                ss += d * d;
+                if (codes) codes[row_base + e1] = (signed char)q1;
+            }
+            if (packed) {
+                if (has1 || !more_rows_in_unit) {
+                    packed[(row_base + e0) >> 1] = (unsigned char)((q0 & 0xf) | ((q1 & 0xf) << 4));
+                } else {
+                    *carry = q0;   // last element of the row: its byte is written by the next row
+                }
+            }
+        }
+    }
+    long long zero64 = 0;
+    block_sum2(ss, zero64, s.scratch);
+    return ss;
+}
+
+template <int CPT>
+__global__ void __launch_bounds__(512) rows_kernel(const RowArgs a) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    const int k = (int)a.K;
+    const int k4 = (k + 3) >> 2;
+    RowSmem s;
+    s.xs = reinterpret_cast<float*>(smem_raw);
+    s.x0 = s.xs + (a.keep_x0 ? 4 * k4 : 0);
+    s.xg = reinterpret_cast<double*>(s.x0 + 4 * k4);
+    s.scratch = s.xg + (size_t)(a.groups - 1) * CPT * a.tg;
+    s.list = reinterpret_cast<int*>(s.scratch + 64);
+    s.misc = s.list + kListCap;
+    const long long n_total = a.S * a.K;
+    const long long n_units = (a.S + a.rows_per_unit - 1) / a.rows_per_unit;
+    const long long packed_stride = (n_total + 1) >> 1;
+    unsigned int st = 0;
+
+    for (long long unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
+        for (int ru = 0; ru < a.rows_per_unit; ++ru) {
+            const long long row = unit * a.rows_per_unit + ru;
+            if (row >= a.S) break;
+            const bool more = (ru + 1 < a.rows_per_unit) && (row + 1 < a.S);
+            const long long row_base = row * a.K;
+            const float* src = a.w + row_base;
+            __syncthreads();   // previous row fully consumed
+            // ---- stage the row once from HBM (128-bit loads when the row start allows it)
+            bool bad = false;
+            if ((reinterpret_cast<unsigned long long>(src) & 15ull) == 0) {
+                const float4* src4 = reinterpret_cast<const float4*>(src);
+                for (int i4 = tid; i4 < (k >> 2); i4 += nthr) {
+                    const float4 v = __ldg(src4 + i4);
+                    reinterpret_cast<float4*>(s.xs)[i4] = v;
+                    bad |= !(fabsf(v.x) <= FLT_MAX) || !(fabsf(v.y) <= FLT_MAX) || !(fabsf(v.z) <= FLT_MAX) || !(fabsf(v.w) <= FLT_MAX);
+                }
+                for (int i = (k & ~3) + tid; i < 4 * k4; i += nthr) {
+                    const float v = i < k ? __ldg(src + i) : 0.f;
+                    s.xs[i] = v;
+                    bad |= !(fabsf(v) <= FLT_MAX);
+                }
+            } else {
+                for (int i = tid; i < 4 * k4; i += nthr) {
+                    const float v = i < k ? __ldg(src + i) : 0.f;
+                    s.xs[i] = v;
+                    bad |= !(fabsf(v) <= FLT_MAX);
+                }
+            }
+            if (bad) st |= 1u;
+            if (a.keep_x0) {
+                __syncthreads();
+                for (int i = tid; i < 4 * k4; i += nthr) s.x0[i] = s.xs[i];
+            }
+            __syncthreads();
+
+            // ---- Algorithm 1: sweeps over the tensors; one tensor and one sweep is plain phi
+            for (int sweep = 0; sweep < a.n_sweeps; ++sweep) {
+                for (int j = 0; j < a.n_tensors; ++j) {
+                    const float flo = (float)a.lo[j], fhi = (float)a.hi[j];
+                    if (a.keep_x0 && !(sweep == 0 && j == 0)) {
+                        // residual T - sum_{i != j} alpha_i q^i from the original row, increasing i
+                        for (int i = tid; i < k; i += nthr) {
+                            float v = s.x0[i];
+                            for (int i2 = 0; i2 < a.n_tensors; ++i2) {
+                                if (i2 == j || (sweep == 0 && i2 > j)) continue;
+                                const float ai = a.alpha[(long long)i2 * a.S + row];
+                                const float qi = (float)a.codes[(long long)i2 * n_total + row_base + i];
+                                v = fmaf(-ai, qi, v);
+                            }
+                            s.xs[i] = v;
+                        }
+                        __syncthreads();
+                    }
+                    PhiOut r = phi_block<CPT>(a, s, k, k4, flo, fhi);
+                    if (r.degenerate) st |= 2u;
+                    const double sse = emit_block(s, k, r.alpha, flo, fhi,
+                                                  a.codes ? a.codes + (long long)j * n_total : nullptr,
+                                                  a.packed ? a.packed + (long long)j * packed_stride : nullptr,
+                                                  row_base, &s.misc[1 + j], more);
+                    if (tid == 0) {
+                        a.alpha[(long long)j * a.S + row] = r.alpha;
+                        a.sse[(long long)j * a.S + row] = (float)sse;
+                        if (a.best_idx && j == 0) a.best_idx[row] = r.idx;
+                    }
+                    if (!a.keep_x0 && j + 1 < a.n_tensors) {
+                        // first sweep without a kept copy: the residual is updated in place
+                        for (int i = tid; i < k; i += nthr) {
+                            const float x = s.xs[i];
+                            const int q = r.alpha > 0.f ? code_of(x, r.alpha, flo, fhi) : 0;
+                            s.xs[i] = fmaf(-r.alpha, (float)q, x);
+                        }
+                    }
+                    __syncthreads();   // alpha / codes of tensor j visible to the block (global + shared)
+                }
+            }
+        }
+    }
+    if (st) atomicOr(a.status, st);   // any thread that saw a flag reports it
+}
+
+}  // namespace omse

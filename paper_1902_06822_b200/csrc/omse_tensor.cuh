@@ -1,0 +1,381 @@
+// Per-tensor MMSE scale (Section 3.7, first equation): one scale for a whole activation tensor.
+// The tensor does not fit on chip, so the search is a short pipeline of grid-wide kernels ordered
+// by the stream (no kernel waits on another block):
+//   absmax -> sweep (tiles through shared memory, partial error sums per block) -> finish (sum the
+//   partials in fixed order, argmin, near-minimal list) -> rescore (fp64, true division) ->
+//   refine x R (<x,q>, <q,q>) -> final (error at the final scale).
+// Grid-wide sums use "the last block to arrive reduces" (a ticket from atomicAdd, no waiting).
+#pragma once
+#include "omse_device.cuh"
+
+namespace omse {
+
+struct TensorState {          // lives in the context workspace
+    unsigned int mpos_bits, mneg_bits;   // max of positive / negative part as float bits (atomicMax)
+    unsigned int ticket;                 // arrivals for last-block reductions (reset by the last block)
+    int best_idx;
+    float alpha;
+    float step;
+    int n_list;
+    int list_overflow;
+    int list[kListCap];
+    int pad_;
+};
+
+struct TensorArgs {
+    const float* x;
+    long long n;
+    int n_cand;
+    float hi_frac;
+    int lo, hi;
+    int tg, groups;         // sweep block = groups*tg threads; candidate c = slot*tg + t
+    int tile4;              // float4s per tile
+    TensorState* st;
+    double* partials;       // sweep: [grid][n_cand]; passes: [grid][kListCap] doubles + [grid] int64
+    double* curve;          // [n_cand] summed error per candidate (workspace)
+    double* curve_out;      // user copy, nullable
+    float* alpha_out;
+    float* sse_out;
+    int* idx_out;
+    unsigned int* status;
+};
+
+__global__ void tensor_init_kernel(TensorState* st) {
+    if (threadIdx.x == 0) {
+        st->mpos_bits = 0u;
+        st->mneg_bits = 0u;
+        st->ticket = 0u;
+        st->best_idx = -1;
+        st->alpha = 0.f;
+        st->step = 0.f;
+        st->n_list = 0;
+        st->list_overflow = 0;
+    }
+}
+
+__global__ void __launch_bounds__(256) tensor_absmax_kernel(const float* __restrict__ x, long long n,
+                                                             TensorState* st, unsigned int* status) {
+    __shared__ double scratch[64];
+    float mpos = 0.f, mneg = 0.f;
+    bool bad = false;
+    const long long n4 = n >> 2;
+    const float4* x4 = reinterpret_cast<const float4*>(x);
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+        const float4 v = __ldg(x4 + i);
+        const float e[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (fabsf(e[j]) <= FLT_MAX) {
+                mpos = fmaxf(mpos, e[j]);
+                mneg = fmaxf(mneg, -e[j]);
+            } else {
+                bad = true;
+            }
+        }
+    }
+    for (long long i = (n4 << 2) + (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
+        const float v = x[i];
+        if (fabsf(v) <= FLT_MAX) {
+            mpos = fmaxf(mpos, v);
+            mneg = fmaxf(mneg, -v);
+        } else {
+            bad = true;
+        }
+    }
+    block_max2(mpos, mneg, scratch);
+    if (threadIdx.x == 0) {
+        atomicMax(&st->mpos_bits, __float_as_uint(mpos));   // non-negative floats order like their bits
+        atomicMax(&st->mneg_bits, __float_as_uint(mneg));
+    }
+    if (bad) atomicOr(status, 1u);
+}
+
+// Candidate sweep over tiles of the tensor; block b handles tiles b, b+grid, ...
+template <int CPT>
+__global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float4* tile = reinterpret_cast<float4*>(smem_raw);
+    double* xg = reinterpret_cast<double*>(tile + a.tile4);
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    const int grp = tid / a.tg, t = tid - grp * a.tg;
+    const float mpos = __uint_as_float(a.st->mpos_bits), mneg = __uint_as_float(a.st->mneg_bits);
+    const float m = fmaxf(mpos, mneg);
+    const float flo = (float)a.lo, fhi = (float)a.hi;
+    const GridSetup g = grid_setup(mpos, mneg, a.hi_frac, a.n_cand, flo, fhi);
+    const float a_last = __fmul_rn((float)a.n_cand, g.step);
+    if (!(m > 0.f) || !(a_last >= FLT_MIN)) return;   // degenerate tensor: finish kernel reports it
+
+    u64 inv2[CPT], na2[CPT];
+    double dacc[CPT];
+#pragma unroll
+    for (int sl = 0; sl < CPT; ++sl) {
+        const int c = sl * a.tg + t;
+        const float ac = __fmul_rn((float)(c + 1), g.step);
+        float inv = g.tiny ? __fdiv_rn(1.0f, ac) : __fdiv_rn(1.0f, (float)(c + 1)) * g.rstep;
+        if (!(ac >= FLT_MIN) || c >= a.n_cand) inv = 0.f;
+        inv2[sl] = pack2(inv, inv);
+        na2[sl] = pack2(-ac, -ac);
+        dacc[sl] = 0.0;
+    }
+    const int warp_t0 = t & ~31;
+    int ncl = (g.c_sat - warp_t0 + a.tg - 1) / a.tg;
+    ncl = max(0, min(CPT, ncl));
+
+    const long long n4_total = (a.n + 3) >> 2;
+    const long long n_tiles = (n4_total + a.tile4 - 1) / a.tile4;
+    const float4* x4 = reinterpret_cast<const float4*>(a.x);
+    for (long long tl = blockIdx.x; tl < n_tiles; tl += gridDim.x) {
+        const long long base4 = tl * a.tile4;
+        const int cnt4 = (int)min((long long)a.tile4, n4_total - base4);
+        __syncthreads();
+        for (int i = tid; i < cnt4; i += nthr) {
+            const long long e = (base4 + i) << 2;
+            float4 v;
+            if (e + 3 < a.n) {
+                v = __ldg(x4 + base4 + i);
+            } else {   // ragged end of the tensor: missing elements count as zeros (zero error)
+                v.x = e < a.n ? a.x[e] : 0.f;
+                v.y = e + 1 < a.n ? a.x[e + 1] : 0.f;
+                v.z = e + 2 < a.n ? a.x[e + 2] : 0.f;
+                v.w = 0.f;
+            }
+            tile[i] = v;
+        }
+        __syncthreads();
+        const int beg4 = (int)(((long long)cnt4 * grp) / a.groups);
+        const int end4 = (int)(((long long)cnt4 * (grp + 1)) / a.groups);
+        sweep_dispatch<CPT>(ncl, tile, beg4, end4, inv2, na2, dacc, kMagic + flo, kMagic + fhi);
+    }
+    if (a.groups > 1) {
+        __syncthreads();
+        if (grp > 0) {
+#pragma unroll
+            for (int sl = 0; sl < CPT; ++sl) xg[((grp - 1) * CPT + sl) * a.tg + t] = dacc[sl];
+        }
+        __syncthreads();
+        if (grp == 0) {
+            for (int gg = 1; gg < a.groups; ++gg)
+#pragma unroll
+                for (int sl = 0; sl < CPT; ++sl) dacc[sl] += xg[((gg - 1) * CPT + sl) * a.tg + t];
+        }
+    }
+    if (grp == 0) {
+#pragma unroll
+        for (int sl = 0; sl < CPT; ++sl) {
+            const int c = sl * a.tg + t;
+            if (c < a.n_cand) a.partials[(long long)blockIdx.x * a.n_cand + c] = dacc[sl];
+        }
+    }
+}
+
+// One block: sums the per-block partials in block order, takes the argmin and lists the candidates
+// inside the fp32 noise band of the minimum.
+__global__ void __launch_bounds__(1024) tensor_finish_kernel(const TensorArgs a, int n_blocks) {
+    __shared__ double scratch[64];
+    __shared__ int cnt;
+    TensorState* st = a.st;
+    const float mpos = __uint_as_float(st->mpos_bits), mneg = __uint_as_float(st->mneg_bits);
+    const float m = fmaxf(mpos, mneg);
+    const GridSetup g = grid_setup(mpos, mneg, a.hi_frac, a.n_cand, (float)a.lo, (float)a.hi);
+    const float a_last = __fmul_rn((float)a.n_cand, g.step);
+    const bool degenerate = !(m > 0.f) || !(a_last >= FLT_MIN);
+    double bv = INFINITY;
+    int bi = 0x7fffffff;
+    if (!degenerate) {
+        for (int c = threadIdx.x; c < a.n_cand; c += blockDim.x) {
+            double s = 0.0;
+            for (int b = 0; b < n_blocks; ++b) s += a.partials[(long long)b * a.n_cand + c];
+            const float ac = __fmul_rn((float)(c + 1), g.step);
+            if (!(ac >= FLT_MIN)) s = INFINITY;
+            a.curve[c] = s;
+            if (a.curve_out) a.curve_out[c] = s;
+            if (s < bv) {
+                bv = s;
+                bi = c;
+            }
+        }
+    }
+    if (threadIdx.x == 0) cnt = 0;
+    block_argmin(bv, bi, scratch);
+    if (degenerate || bi == 0x7fffffff) {
+        if (threadIdx.x == 0) {
+            st->best_idx = -1;
+            st->alpha = 0.f;
+            st->n_list = 0;
+            atomicOr(a.status, 2u);
+        }
+        if (degenerate && a.curve_out)
+            for (int c = threadIdx.x; c < a.n_cand; c += blockDim.x) a.curve_out[c] = INFINITY;
+        return;
+    }
+    const double band = bv * (1.0 + kRescoreBand);
+    for (int c = threadIdx.x; c < a.n_cand; c += blockDim.x) {
+        if (a.curve[c] <= band) {
+            const int pos = atomicAdd(&cnt, 1);
+            if (pos < kListCap) st->list[pos] = c;
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        st->step = g.step;
+        st->best_idx = bi;
+        st->alpha = __fmul_rn((float)(bi + 1), g.step);
+        st->n_list = (cnt > 1 && cnt <= kListCap) ? cnt : 0;   // 0: the fp32 winner stands
+    }
+}
+
+// Grid-wide pass over the tensor in fp64 with true division.
+//   MODE 0 (rescore): squared error at each listed candidate; the last block picks the best.
+//   MODE 1 (refine):  <x,q> and <q,q> at st->alpha; the last block sets alpha <- <x,q>/<q,q>.
+//   MODE 2 (final):   squared error at st->alpha; the last block writes the outputs.
+template <int MODE>
+__global__ void __launch_bounds__(256) tensor_pass_kernel(const TensorArgs a) {
+    __shared__ double scratch[64];
+    __shared__ bool is_last;
+    TensorState* st = a.st;
+    const float flo = (float)a.lo, fhi = (float)a.hi;
+    const int n_list = MODE == 0 ? st->n_list : 1;
+    if (MODE == 0 && n_list == 0) return;
+    const float alpha_now = st->alpha;
+    if (MODE == 1 && !(alpha_now > 0.f)) return;
+    double* part_d = a.partials;                                         // [grid][kListCap]
+    long long* part_q = reinterpret_cast<long long*>(a.partials + (size_t)gridDim.x * kListCap);  // [grid]
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    const long long tid0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long n4 = a.n >> 2;
+    const float4* x4 = reinterpret_cast<const float4*>(a.x);
+
+    for (int l0 = 0; l0 < n_list; l0 += 4) {
+        float al[4];
+        double acc[4] = {0.0, 0.0, 0.0, 0.0};
+        long long sqq = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (MODE == 0) {
+                const int c = (l0 + j < n_list) ? st->list[l0 + j] : st->list[l0];
+                al[j] = __fmul_rn((float)(c + 1), st->step);
+            } else {
+                al[j] = alpha_now;
+            }
+        }
+        auto element = [&](float x) {
+            if (MODE == 0) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const double d = (double)x - (double)al[j] * (double)code_of(x, al[j], flo, fhi);
+                    acc[j] += d * d;
+                }
+            } else if (MODE == 1) {
+                const int q = code_of(x, al[0], flo, fhi);
+                sqq += q * q;
+                acc[0] += (double)x * (double)q;
+            } else {
+                const int q = al[0] > 0.f ? code_of(x, al[0], flo, fhi) : 0;
+                const double d = (double)x - (double)al[0] * (double)q;
+                acc[0] += d * d;
+            }
+        };
+        for (long long i = tid0; i < n4; i += stride) {
+            const float4 v = __ldg(x4 + i);
+            element(v.x);
+            element(v.y);
+            element(v.z);
+            element(v.w);
+        }
+        for (long long i = (n4 << 2) + tid0; i < a.n; i += stride) element(a.x[i]);
+        const int nj = MODE == 0 ? 4 : 1;
+        for (int j = 0; j < nj; ++j) {
+            long long q = sqq;
+            block_sum2(acc[j], q, scratch);
+            if (threadIdx.x == 0) {
+                part_d[(size_t)blockIdx.x * kListCap + l0 + j] = acc[j];
+                if (MODE == 1) part_q[blockIdx.x] = q;
+            }
+        }
+    }
+    // ---- last block to arrive reduces the per-block partials in block order
+    __threadfence();
+    if (threadIdx.x == 0) {
+        const unsigned int tk = atomicAdd(&st->ticket, 1u);
+        is_last = (tk == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    const int nl = MODE == 0 ? ((n_list + 3) & ~3) : 1;
+    __shared__ double tot_d[kListCap];
+    __shared__ long long tot_q;
+    if (threadIdx.x < nl) {
+        double s = 0.0;
+        for (unsigned int b = 0; b < gridDim.x; ++b) s += __ldcg(&part_d[(size_t)b * kListCap + threadIdx.x]);
+        tot_d[threadIdx.x] = s;
+    }
+    if (MODE == 1 && threadIdx.x == 32) {
+        long long q = 0;
+        for (unsigned int b = 0; b < gridDim.x; ++b) q += __ldcg(&part_q[b]);
+        tot_q = q;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        st->ticket = 0u;
+        if (MODE == 0) {
+            double best_sse = INFINITY;
+            int best = 0x7fffffff;
+            for (int l = 0; l < n_list; ++l) {
+                const int c = st->list[l];
+                if (tot_d[l] < best_sse || (tot_d[l] == best_sse && c < best)) {
+                    best_sse = tot_d[l];
+                    best = c;
+                }
+            }
+            st->best_idx = best;
+            st->alpha = __fmul_rn((float)(best + 1), st->step);
+        } else if (MODE == 1) {
+            if (tot_q != 0) {
+                const float a_new = (float)(tot_d[0] / (double)tot_q);
+                if (a_new >= FLT_MIN && a_new <= FLT_MAX) st->alpha = a_new;
+            }
+        } else {
+            *a.alpha_out = st->alpha;
+            *a.sse_out = (float)tot_d[0];
+            if (a.idx_out) *a.idx_out = st->best_idx;
+        }
+    }
+}
+
+// INT4 emission: byte e/2 holds element e (even) in bits 0-3 and element e+1 in bits 4-7.
+__global__ void __launch_bounds__(256) pack_int4_kernel(const signed char* __restrict__ codes, long long n,
+                                                         unsigned char* __restrict__ packed) {
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    const long long tid0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const bool aligned = ((reinterpret_cast<unsigned long long>(codes) & 15ull) == 0) &&
+                         ((reinterpret_cast<unsigned long long>(packed) & 7ull) == 0);
+    const long long n16 = aligned ? (n >> 4) : 0;
+    for (long long i = tid0; i < n16; i += stride) {
+        const int4 v = __ldg(reinterpret_cast<const int4*>(codes) + i);
+        const unsigned int w[4] = {(unsigned)v.x, (unsigned)v.y, (unsigned)v.z, (unsigned)v.w};
+        unsigned int out[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            unsigned int r = 0;
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const unsigned int u = w[2 * h + j];   // four codes -> two bytes
+                const unsigned int b0 = (u & 0xf) | ((u >> 4) & 0xf0);
+                const unsigned int b1 = ((u >> 16) & 0xf) | ((u >> 20) & 0xf0);
+                r |= (b0 | (b1 << 8)) << (16 * j);
+            }
+            out[h] = r;
+        }
+        reinterpret_cast<uint2*>(packed)[i] = make_uint2(out[0], out[1]);
+    }
+    const long long nb = (n + 1) >> 1;
+    for (long long b = (n16 << 3) + tid0; b < nb; b += stride) {
+        const unsigned int lo = (unsigned char)codes[2 * b] & 0xf;
+        const unsigned int hi = (2 * b + 1 < n) ? ((unsigned char)codes[2 * b + 1] & 0xf) : 0u;
+        packed[b] = (unsigned char)(lo | (hi << 4));
+    }
+}
+
+}  // namespace omse

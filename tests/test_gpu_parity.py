@@ -1,0 +1,200 @@
+"""GPU parity: the CUDA library, called through its C interface, against the CPU oracle."""
+import numpy as np
+import pytest
+
+from oracle import omse_oracle as orc
+from paper_1902_06822_b200 import synth
+from parity import RTOL, check_rows
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def gpu():
+    import gpu_util
+    return gpu_util
+
+
+def _run_and_check(gpu, w, bits, signed, n_cand, refine, hi_frac=1.0, codes=True, packed=False, rows=None):
+    alpha, sse, idx, q, pk = gpu.quantize_weights(w, bits, signed, n_cand, hi_frac, refine, codes, packed)
+    stats = check_rows(w, alpha, sse, idx, q, pk, bits, signed, n_cand, hi_frac, refine, rows=rows)
+    assert stats["idx_diff"] <= max(1, stats["rows"] // 100), stats
+    assert stats["alpha_bitwise"] >= 0.99, stats
+    return stats
+
+
+# ---------------------------------------------------------------- configs[0]: one convolution layer
+def test_single_conv_layer_config(gpu):
+    w = synth.conv_layer(seed=1)
+    _run_and_check(gpu, w, 4, True, 256, 3, codes=True, packed=True)
+    _run_and_check(gpu, w, 4, True, 256, 0, codes=True, packed=False)
+
+
+# ---------------------------------------------------------------- shapes: several tiles, ragged tails
+@pytest.mark.parametrize("k", [1, 2, 3, 5, 27, 31, 32, 33, 64, 147, 255, 576, 1000, 4608])
+def test_kernel_lengths_with_odd_row_counts(gpu, k):
+    s = 37 if k < 2000 else 9
+    w = synth.student_t3(s * k, seed=50 + k, tensor_id=k).reshape(s, k)
+    _run_and_check(gpu, w, 4, True, 256, 3, codes=True, packed=True)
+
+
+@pytest.mark.parametrize("n_cand", [1, 16, 50, 64, 100, 128, 500, 1024, 2048, 4096])
+def test_candidate_counts(gpu, n_cand):
+    w = synth.laplace(21 * 300, 0.05, seed=60, tensor_id=n_cand).reshape(21, 300)
+    _run_and_check(gpu, w, 4, True, n_cand, 3, codes=True, packed=True)
+
+
+@pytest.mark.parametrize("bits,signed", [(2, True), (3, True), (4, True), (8, True), (2, False), (4, False), (8, False)])
+def test_bit_widths_and_signedness(gpu, bits, signed):
+    w = synth.student_t3(33 * 576, seed=70, tensor_id=bits).reshape(33, 576)
+    if not signed and bits != 4:
+        w = np.abs(w)          # unsigned grid on non-negative data; bits == 4 keeps the negatives
+    _run_and_check(gpu, w, bits, signed, 1024, 3, codes=True, packed=bits <= 4)
+
+
+def test_hi_frac_other_than_one_and_packed_only(gpu):
+    w = synth.laplace(40 * 147, 0.02, seed=80).reshape(40, 147)
+    _run_and_check(gpu, w, 4, True, 256, 2, hi_frac=1.0 / 7, codes=True, packed=True)
+    _run_and_check(gpu, w, 4, True, 256, 2, hi_frac=0.5, codes=False, packed=True)
+    _run_and_check(gpu, w, 3, True, 64, 1, codes=False, packed=False)
+
+
+def test_large_rows_span_element_groups(gpu):
+    w = synth.sweep_tensor(25088, seed=5, n_kernels=6)
+    _run_and_check(gpu, w, 4, True, 1024, 3, codes=True, packed=True)
+    w = synth.sweep_tensor(28672, seed=6, n_kernels=3)
+    _run_and_check(gpu, w, 2, True, 1024, 3, codes=True, packed=True)
+
+
+# ---------------------------------------------------------------- degenerate and invalid inputs
+def test_zero_rows_non_finite_values_and_status_word(gpu):
+    w = synth.laplace(8 * 64, 0.02, seed=90).reshape(8, 64).copy()
+    w[2] = 0.0
+    w[5, 3] = np.nan
+    w[6] = 1e-42          # every candidate below FLT_MIN
+    gpu.ctx().omse_last_device_status()
+    alpha, sse, idx, q, pk = gpu.quantize_weights(w, 4, True, 256, 1.0, 3, True, True)
+    st = gpu.ctx().omse_last_device_status()
+    assert st & 1 and st & 2
+    for r in (2, 6):
+        assert alpha[r] == 0.0 and idx[r] == -1 and not q.reshape(8, 64)[r].any()
+    assert sse[2] == 0.0
+    assert q.min() >= -8 and q.max() <= 7
+    good = [0, 1, 3, 4, 7]
+    check_rows(w, alpha, sse, idx, q, None, 4, True, 256, 1.0, 3, rows=good)
+    assert gpu.ctx().omse_last_device_status() == 0
+
+
+def test_invalid_arguments_are_rejected(gpu):
+    import torch
+    from paper_1902_06822_b200 import binding
+    c = gpu.ctx()
+    w = torch.zeros(64, device="cuda")
+    a = torch.zeros(8, device="cuda")
+    s = torch.zeros(8, device="cuda")
+    pk = torch.zeros(32, dtype=torch.uint8, device="cuda")
+    bad = [
+        dict(bits=1), dict(bits=9), dict(n_cand=0), dict(n_cand=4097), dict(hi_frac=0.0), dict(refine_iters=-1),
+        dict(kernel_len=0), dict(kernel_len=binding.MAX_KERNEL_LEN + 1), dict(n_kernels=-1), dict(bits=8, packed=pk),
+    ]
+    for kw in bad:
+        args = dict(w=w, n_kernels=8, kernel_len=8, bits=4, is_signed=True, n_cand=16, hi_frac=1.0, refine_iters=1,
+                    alpha=a, sse=s, packed=None)
+        args.update(kw)
+        with pytest.raises(binding.OmseError) as e:
+            c.omse_quantize_weights(**args)
+        assert e.value.code == binding.EINVAL, kw
+    with pytest.raises(binding.OmseError):
+        c.omse_residual_quantize(w, 8, 8, [4, 4], True, 16, 1.0, 1, 2, a, s, None, None)   # sweeps > 1 need codes
+    with pytest.raises(binding.OmseError):
+        c.omse_residual_quantize(w, 8, 8, [4] * 5, True, 16, 1.0, 1, 1, a, s, None, None)
+    c.omse_quantize_weights(w, 0, 8, 4, True, 16, 1.0, 1, a, s)     # empty input: nothing to do
+    torch.cuda.synchronize()
+
+
+# ---------------------------------------------------------------- INT4 emission
+@pytest.mark.parametrize("n", [0, 1, 2, 15, 16, 17, 4097, 1 << 20, (1 << 20) + 3])
+def test_pack_int4_matches_oracle(gpu, n):
+    import torch
+    rng = np.random.default_rng(n)
+    q = rng.integers(-8, 8, size=max(n, 1), dtype=np.int8)[:n]
+    d_q = torch.from_numpy(q).cuda() if n else torch.zeros(1, dtype=torch.int8, device="cuda")
+    d_p = torch.full(((n + 1) // 2 + 1,), 0xEE, dtype=torch.uint8, device="cuda")
+    gpu.ctx().omse_pack_int4(d_q, n, True, d_p)
+    torch.cuda.synchronize()
+    out = d_p.cpu().numpy()
+    assert out[-1] == 0xEE                                  # nothing written past the end
+    assert np.array_equal(out[:-1], orc.pack_int4(q))
+    if n > 16:                                              # unaligned views take the byte path
+        gpu.ctx().omse_pack_int4(d_q[1:], n - 1, True, d_p[1:])
+        torch.cuda.synchronize()
+        assert np.array_equal(d_p.cpu().numpy()[1:1 + n // 2], orc.pack_int4(q[1:]))
+
+
+# ---------------------------------------------------------------- Section 3.7: per-tensor scale
+def _check_activation(gpu, x, bits, signed, n_cand, refine):
+    alpha, sse, idx, curve = gpu.activation_scale(x, bits, signed, n_cand, 1.0, refine)
+    ref = orc.activation_scale(x, bits, signed, n_cand, 1.0, refine)
+    finite = np.isfinite(ref.sse_curve)
+    assert np.array_equal(finite, np.isfinite(curve))
+    np.testing.assert_allclose(curve[finite], ref.sse_curve[finite], rtol=2e-6)
+    if idx != ref.best_idx:
+        assert abs(ref.sse_curve[idx] - ref.sse_curve[ref.best_idx]) <= 1e-6 * ref.sse_curve[ref.best_idx]
+        ref = orc.phi(x, bits, signed, n_cand, 1.0, refine, start_idx=idx, want_codes=False)
+    assert alpha == pytest.approx(ref.alpha, rel=RTOL)
+    assert sse == pytest.approx(ref.sse, rel=RTOL)
+    return idx == ref.best_idx
+
+
+@pytest.mark.parametrize("n", [1, 3, 4, 1000, 4096, 4097, 300_001, 2_000_000])
+def test_activation_scale_sizes(gpu, n):
+    x = synth.relu_activations(n, seed=3, tensor_id=n % 97)
+    if n <= 4:
+        x = x + np.float32(0.25)
+    assert _check_activation(gpu, x, 4, False, 2048 if n > 1000 else 256, 3)
+
+
+@pytest.mark.parametrize("bits,signed,n_cand", [(4, True, 50), (8, False, 500), (2, False, 64), (3, True, 4096)])
+def test_activation_scale_grids(gpu, bits, signed, n_cand):
+    x = synth.student_t3(250_000, seed=33, tensor_id=bits)
+    if not signed:
+        x = np.abs(x)
+    _check_activation(gpu, x, bits, signed, n_cand, 2)
+
+
+def test_activation_scale_degenerate(gpu):
+    gpu.ctx().omse_last_device_status()
+    alpha, sse, idx, curve = gpu.activation_scale(np.zeros(5000, np.float32), 4, False, 128, 1.0, 3)
+    assert (alpha, sse, idx) == (0.0, 0.0, -1) and gpu.ctx().omse_last_device_status() & 2
+
+
+# ---------------------------------------------------------------- Sections 3.5 / 3.7: residual, Algorithm 1
+def _residual_step_by_step(gpu, t, bits, n_cand, refine, packed=False):
+    alpha, sse, q, pk = gpu.residual_quantize(t, bits, True, n_cand, 1.0, refine, 1, True, packed)
+    S, K = t.shape
+    r = t.copy()
+    for j, b in enumerate(bits):
+        st = check_rows(r, alpha[j], sse[j], None, q[j], pk[j] if packed else None, b, True, n_cand, 1.0, refine)
+        assert st["alpha_bitwise"] >= 0.99
+        # next residual exactly as defined: one binary32 rounding of r - alpha*q per element
+        r = (r.astype(np.float64) - alpha[j][:, None].astype(np.float64) * q[j].reshape(S, K)).astype(np.float32)
+    assert np.all(sse[1] <= sse[0])
+    return alpha, sse, q
+
+
+def test_residual_two_tensors_small(gpu):
+    t = synth.laplace_with_outliers(30 * 500, 0.005, seed=4, outlier_prob=0.01).reshape(30, 500)
+    _residual_step_by_step(gpu, t, (4, 4), 256, 3, packed=True)
+    t = synth.student_t3(15 * 147, seed=41).reshape(15, 147)
+    _residual_step_by_step(gpu, t, (4, 2, 3), 128, 2, packed=True)
+
+
+def test_algorithm_1_two_sweeps_matches_oracle(gpu):
+    t = synth.student_t3(12 * 300, seed=21).reshape(12, 300)
+    alpha, sse, q, _ = gpu.residual_quantize(t, (3, 3), True, 128, 1.0, 2, n_sweeps=2)
+    ref = orc.residual_rows(t, (3, 3), True, 128, 1.0, 2, n_sweeps=2)
+    np.testing.assert_allclose(alpha, ref.alpha, rtol=RTOL)
+    np.testing.assert_allclose(sse, ref.sse, rtol=RTOL)
+    same = np.all(alpha == ref.alpha, axis=0)
+    assert same.mean() >= 0.9
+    assert np.array_equal(q.reshape(2, 12, 300)[:, same], ref.codes[:, same])

@@ -2,8 +2,8 @@
 """Throughput of the MMSE quantization search on the ResNet-50-shaped weight set.
 
 One step = the whole hot path over one batch of synthetic input: every one of the 54 weight
-tensors goes through omse_quantize_weights (stage, max, 1024-candidate sweep, argmin, 3 polish
-steps, codes, INT4 packing).  Prints ONE JSON line (rank 0).
+tensors goes through omse_quantize_weights_batched (stage, max, 1024-candidate sweep, argmin,
+3 polish steps, codes, INT4 packing; one launch for the set).  Prints ONE JSON line (rank 0).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
@@ -159,16 +159,18 @@ def run_ours(args, rank, world):
     host_out = [(a.cpu().pin_memory(), e.cpu().pin_memory(), p.cpu().pin_memory()) for a, e, p in outs]
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # > 126 MB L2
 
+    descs = [dict(w=dw, n_kernels=w.shape[0], kernel_len=w.shape[1], alpha=a, sse=e, packed=p)
+             for (name, w), dw, (a, e, p) in zip(weights, d_w, outs)]
+
     def step():
-        for (name, w), dw, (a, e, p) in zip(weights, d_w, outs):
-            s, k = w.shape
-            ctx.omse_quantize_weights(dw, s, k, BITS, True, N_CAND, HI_FRAC, REFINE, a, e, None, None, p)
+        # all 54 tensors in one launch: kernels of every layer are handed out longest first
+        ctx.omse_quantize_weights_batched(descs, BITS, True, N_CAND, HI_FRAC, REFINE)
 
     def step_e2e():
-        for (name, w), hin, dw, (a, e, p), (ha, he, hp) in zip(weights, host_in, d_w, outs, host_out):
-            s, k = w.shape
+        for hin, dw in zip(host_in, d_w):
             dw.copy_(hin, non_blocking=True)
-            ctx.omse_quantize_weights(dw, s, k, BITS, True, N_CAND, HI_FRAC, REFINE, a, e, None, None, p)
+        ctx.omse_quantize_weights_batched(descs, BITS, True, N_CAND, HI_FRAC, REFINE)
+        for (a, e, p), (ha, he, hp) in zip(outs, host_out):
             ha.copy_(a, non_blocking=True)
             he.copy_(e, non_blocking=True)
             hp.copy_(p, non_blocking=True)
@@ -223,7 +225,7 @@ def run_ours(args, rank, world):
             "clocks": clocks,
             "e2e": {"value": world * n_total / (ms_e2e * 1e-3 / args.steps), "unit": "elements/s",
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-            "gpu_launches": 54 * args.steps,
+            "gpu_launches": args.steps,
             "roofline": {"bound": "alu", "achieved": achieved / 1e12, "peak": peak / 1e12,
                          "unit": "T FP32-instr/s", "frac": achieved / peak, "traffic": None,
                          "kernel": "rows_kernel<8>", "peak_source": f"148 SMs x 128 lanes x {sm_max_mhz:.0f} MHz ({peak_src} max clock)",

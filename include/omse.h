@@ -53,6 +53,7 @@ typedef enum {
 #define OMSE_MAX_KERNEL_LEN 28672  /* kernel_len of the kernel-wise entry points (one row on chip) */
 #define OMSE_MAX_KERNEL_LEN_MULTISWEEP 25600 /* with n_sweeps > 1 (row and residual both on chip)       */
 #define OMSE_MAX_TENSORS 4         /* n_tensors of omse_residual_quantize                           */
+#define OMSE_MAX_BATCH 1024        /* weight tensors per omse_quantize_weights_batched call         */
 
 /* The line-search grid of Section 3.4 ("a given grid"): n_cand scales spaced linearly in
  * (0, hi_frac*max|x|], candidate c (0-based) being fl(fl(c+1) * fl(fl(hi_frac*max|x|)/fl(n_cand)))
@@ -96,6 +97,27 @@ size_t omse_workspace_bytes(const omse_ctx* ctx);
 int omse_quantize_weights(omse_ctx* ctx, const float* d_w, int64_t n_kernels, int64_t kernel_len,
                           int bits, int is_signed, const omse_grid* grid, float* d_alpha,
                           float* d_sse, int32_t* d_best_idx, int8_t* d_codes, uint8_t* d_packed);
+
+/*
+ * The same operation on a set of weight tensors (the layers W_1..W_L of a network, Section 3.1) in
+ * ONE launch: kernels of all tensors are handed out to the thread blocks longest first, so the GPU
+ * stays full across layer boundaries.  `tensors` is a HOST array of n_tensors descriptors (read
+ * before the call returns); each descriptor's fields have the meaning and nullability of the
+ * arguments of omse_quantize_weights.  bits / is_signed / grid apply to every tensor.
+ * 0 <= n_tensors <= OMSE_MAX_BATCH; tensors with n_kernels == 0 are skipped.
+ */
+typedef struct {
+    const float* d_w;
+    int64_t n_kernels, kernel_len;
+    float* d_alpha;
+    float* d_sse;
+    int32_t* d_best_idx;
+    int8_t* d_codes;
+    uint8_t* d_packed;
+} omse_weight_tensor;
+
+int omse_quantize_weights_batched(omse_ctx* ctx, const omse_weight_tensor* tensors, int n_tensors,
+                                  int bits, int is_signed, const omse_grid* grid);
 
 /*
  * Per-tensor MMSE scale for an activation tensor (Section 3.7, first equation): one scale for

@@ -20,6 +20,7 @@ MAX_CANDIDATES, MAX_KERNEL_LEN, MAX_KERNEL_LEN_MULTISWEEP, MAX_TENSORS = 4096, 2
 
 EXPORTS = [
     "omse_create", "omse_destroy", "omse_set_stream", "omse_workspace_bytes", "omse_quantize_weights",
+    "omse_quantize_weights_batched",
     "omse_activation_scale", "omse_residual_quantize", "omse_pack_int4", "omse_last_device_status",
     "omse_status_string",
 ]
@@ -27,6 +28,11 @@ EXPORTS = [
 
 class OmseGrid(C.Structure):
     _fields_ = [("n_cand", C.c_int32), ("hi_frac", C.c_float), ("refine_iters", C.c_int32)]
+
+
+class OmseWeightTensor(C.Structure):
+    _fields_ = [("d_w", C.c_void_p), ("n_kernels", C.c_int64), ("kernel_len", C.c_int64), ("d_alpha", C.c_void_p),
+                ("d_sse", C.c_void_p), ("d_best_idx", C.c_void_p), ("d_codes", C.c_void_p), ("d_packed", C.c_void_p)]
 
 
 class OmseError(RuntimeError):
@@ -53,6 +59,7 @@ def load_library() -> C.CDLL:
     lib.omse_workspace_bytes.argtypes = [vp]
     lib.omse_workspace_bytes.restype = C.c_size_t
     lib.omse_quantize_weights.argtypes = [vp, vp, i64, i64, i32, i32, C.POINTER(OmseGrid), vp, vp, vp, vp, vp]
+    lib.omse_quantize_weights_batched.argtypes = [vp, C.POINTER(OmseWeightTensor), i32, i32, i32, C.POINTER(OmseGrid)]
     lib.omse_activation_scale.argtypes = [vp, vp, i64, i32, i32, C.POINTER(OmseGrid), vp, vp, vp, vp]
     lib.omse_residual_quantize.argtypes = [vp, vp, i64, i64, C.POINTER(C.c_int), i32, C.POINTER(OmseGrid), i32, i32,
                                            vp, vp, vp, vp]
@@ -60,9 +67,6 @@ def load_library() -> C.CDLL:
     lib.omse_last_device_status.argtypes = [vp, C.POINTER(C.c_uint32)]
     lib.omse_status_string.argtypes = [i32]
     lib.omse_status_string.restype = C.c_char_p
-    for name in EXPORTS:
-        if getattr(lib, name).restype is None:
-            pass
     _lib = lib
     return lib
 
@@ -126,6 +130,23 @@ class Context:
             _ptr(codes, torch.int8), _ptr(packed, torch.uint8))
         if rc != OK:
             raise OmseError(rc, "omse_quantize_weights")
+
+    def omse_quantize_weights_batched(self, tensors, bits, is_signed, n_cand, hi_frac, refine_iters):
+        """tensors: sequence of dicts with keys w, n_kernels, kernel_len, alpha, sse and optionally
+        best_idx, codes, packed (CUDA tensors), one per weight tensor; all quantized in one launch."""
+        g = OmseGrid(n_cand, hi_frac, refine_iters)
+        arr = (OmseWeightTensor * len(tensors))()
+        for d, t in zip(arr, tensors):
+            d.d_w = _ptr(t["w"], torch.float32)
+            d.n_kernels, d.kernel_len = t["n_kernels"], t["kernel_len"]
+            d.d_alpha = _ptr(t["alpha"], torch.float32)
+            d.d_sse = _ptr(t["sse"], torch.float32)
+            d.d_best_idx = _ptr(t.get("best_idx"), torch.int32)
+            d.d_codes = _ptr(t.get("codes"), torch.int8)
+            d.d_packed = _ptr(t.get("packed"), torch.uint8)
+        rc = load_library().omse_quantize_weights_batched(self._h, arr, len(tensors), bits, int(is_signed), C.byref(g))
+        if rc != OK:
+            raise OmseError(rc, "omse_quantize_weights_batched")
 
     def omse_activation_scale(self, x, n, bits, is_signed, n_cand, hi_frac, refine_iters, alpha, sse,
                               best_idx=None, sse_curve=None):

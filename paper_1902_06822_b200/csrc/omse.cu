@@ -3,9 +3,25 @@
 // host arithmetic on tensor data and no CPU fallback.
 #include "../../include/omse.h"
 
+#include <algorithm>
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <vector>
+
+#ifndef OMSE_ROWS_BIG_K
+#define OMSE_ROWS_BIG_K 8192        /* rows at least this long use the larger block */
+#endif
+#ifndef OMSE_ROWS_THREADS_BIG
+#define OMSE_ROWS_THREADS_BIG 512
+#endif
+#ifndef OMSE_ROWS_THREADS_MID
+#define OMSE_ROWS_THREADS_MID 128
+#endif
+
+#ifndef OMSE_SMALL_K
+#define OMSE_SMALL_K 640            /* rows up to this length are batched per work unit */
+#endif
 
 #include "omse_rows.cuh"
 #include "omse_tensor.cuh"
@@ -13,11 +29,12 @@
 namespace {
 
 constexpr size_t kPartialBytes = 16u << 20;   // per-block partial sums of the per-tensor search
-constexpr int kMaxSmem = 232448;              // 227 KB opt-in limit per block on sm_100
+constexpr int kMaxSmem = 231424;              // dynamic shared memory per block: the 227 KB opt-in limit of sm_100 less 1 KB for static use
 
 struct Workspace {
     unsigned int status;
     unsigned int pad_[3];
+    unsigned long long ticket[2];   // work-unit dispenser of the row kernels (self-resetting)
     omse::TensorState tstate;
     double curve[OMSE_MAX_CANDIDATES];
 };
@@ -30,6 +47,7 @@ struct omse_ctx {
     int n_sm;
     Workspace* ws;       // device
     double* partials;    // device, kPartialBytes
+    omse::RowTensor* d_tensors;   // device, OMSE_MAX_BATCH descriptors of a batched launch
 };
 
 namespace {
@@ -63,18 +81,19 @@ int launch_rows_t(omse_ctx* ctx, omse::RowArgs& a, size_t smem) {
     int occ = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, omse::rows_kernel<CPT>, threads, smem) != cudaSuccess || occ < 1)
         return OMSE_ECUDA;
-    const long long n_units = (a.S + a.rows_per_unit - 1) / a.rows_per_unit;
     long long grid = (long long)ctx->n_sm * occ;
-    if (grid > n_units) grid = n_units;
+    if (grid > a.n_units) grid = a.n_units;
     omse::rows_kernel<CPT><<<(unsigned)grid, threads, smem, ctx->stream>>>(a);
     return cudaGetLastError() == cudaSuccess ? OMSE_OK : OMSE_ECUDA;
 }
 
-int launch_rows(omse_ctx* ctx, omse::RowArgs& a) {
+// Launch shape for rows of at most max_k elements: threads per block, element groups, shared memory.
+int launch_rows(omse_ctx* ctx, omse::RowArgs& a, long long max_k, size_t smem_small = 0) {
     const int cpt = cpt_for(a.n_cand);
     a.tg = (((a.n_cand + cpt - 1) / cpt) + 31) & ~31;
-    const int k4 = (int)((a.K + 3) >> 2);
-    int target = a.K >= 8192 ? 512 : a.K >= 512 ? 256 : 128;
+    const int k4 = (int)((max_k + 3) >> 2);
+    a.max_k4 = k4;
+    int target = max_k >= OMSE_ROWS_BIG_K ? OMSE_ROWS_THREADS_BIG : OMSE_ROWS_THREADS_MID;
     int groups = target / a.tg;
     if (groups > k4 / 8) groups = k4 / 8;
     if (groups < 1) groups = 1;
@@ -83,8 +102,11 @@ int launch_rows(omse_ctx* ctx, omse::RowArgs& a) {
         return (size_t)(a.keep_x0 ? 2 : 1) * k4 * 16 + (size_t)(gr - 1) * cpt * a.tg * 8 + 64 * 8 + omse::kListCap * 4 + 8 * 4;
     };
     while (a.groups > 1 && smem_for(a.groups) > (size_t)kMaxSmem) a.groups >>= 1;
-    const size_t smem = smem_for(a.groups);
+    size_t smem = smem_for(a.groups);
     if (smem > (size_t)kMaxSmem) return OMSE_EINVAL;
+    if (smem_small > smem) smem = smem_small;
+    a.ticket = ctx->ws->ticket;
+    a.status = &ctx->ws->status;
     switch (cpt) {
         case 1: return launch_rows_t<1>(ctx, a, smem);
         case 2: return launch_rows_t<2>(ctx, a, smem);
@@ -92,6 +114,34 @@ int launch_rows(omse_ctx* ctx, omse::RowArgs& a) {
         default: return launch_rows_t<8>(ctx, a, smem);
     }
 }
+
+void fill_tensor(omse::RowTensor& t, const float* w, int64_t S, int64_t K, float* alpha, float* sse, int32_t* idx,
+                 int8_t* codes, uint8_t* packed) {
+    t.w = w;
+    t.S = S;
+    t.K = K;
+    t.alpha = alpha;
+    t.sse = sse;
+    t.best_idx = idx;
+    t.codes = reinterpret_cast<signed char*>(codes);
+    t.packed = packed;
+    t.unit_begin = 0;
+    t.rows_per_unit = (packed && (K & 1)) ? 2 : 1;
+    t.small = 0;
+}
+
+// Threads of one element group and whether a launch over rows of at most max_k elements runs a
+// single group per block (the short-row path needs that).
+int group_threads(int n_cand) {
+    const int cpt = cpt_for(n_cand);
+    return (((n_cand + cpt - 1) / cpt) + 31) & ~31;
+}
+bool single_group(int n_cand, long long max_k) {
+    const int target = max_k >= OMSE_ROWS_BIG_K ? OMSE_ROWS_THREADS_BIG : OMSE_ROWS_THREADS_MID;
+    return target / group_threads(n_cand) <= 1;
+}
+
+bool misaligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3) != 0; }
 
 template <int CPT>
 int launch_tensor_sweep_t(omse_ctx* ctx, omse::TensorArgs& a, size_t smem, int* n_blocks) {
@@ -143,12 +193,15 @@ int omse_create(omse_ctx** out, int device, void* cuda_stream) {
     c->stream = static_cast<cudaStream_t>(cuda_stream);
     c->ws = nullptr;
     c->partials = nullptr;
+    c->d_tensors = nullptr;
     if (cudaDeviceGetAttribute(&c->n_sm, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
         delete c;
         return OMSE_ECUDA;
     }
-    if (cudaMalloc(&c->ws, sizeof(Workspace)) != cudaSuccess || cudaMalloc(&c->partials, kPartialBytes) != cudaSuccess) {
+    if (cudaMalloc(&c->ws, sizeof(Workspace)) != cudaSuccess || cudaMalloc(&c->partials, kPartialBytes) != cudaSuccess ||
+        cudaMalloc(&c->d_tensors, sizeof(omse::RowTensor) * OMSE_MAX_BATCH) != cudaSuccess) {
         cudaFree(c->ws);
+        cudaFree(c->partials);
         delete c;
         cudaGetLastError();
         return OMSE_ENOMEM;
@@ -156,6 +209,7 @@ int omse_create(omse_ctx** out, int device, void* cuda_stream) {
     if (cudaMemsetAsync(c->ws, 0, sizeof(Workspace), c->stream) != cudaSuccess) {
         cudaFree(c->ws);
         cudaFree(c->partials);
+        cudaFree(c->d_tensors);
         delete c;
         return OMSE_ECUDA;
     }
@@ -169,6 +223,7 @@ int omse_destroy(omse_ctx* ctx) {
     cudaStreamSynchronize(ctx->stream);
     cudaFree(ctx->ws);
     cudaFree(ctx->partials);
+    cudaFree(ctx->d_tensors);
     delete ctx;
     return OMSE_OK;
 }
@@ -179,7 +234,9 @@ int omse_set_stream(omse_ctx* ctx, void* cuda_stream) {
     return OMSE_OK;
 }
 
-size_t omse_workspace_bytes(const omse_ctx* ctx) { return ctx ? sizeof(Workspace) + kPartialBytes : 0; }
+size_t omse_workspace_bytes(const omse_ctx* ctx) {
+    return ctx ? sizeof(Workspace) + kPartialBytes + sizeof(omse::RowTensor) * OMSE_MAX_BATCH : 0;
+}
 
 int omse_last_device_status(omse_ctx* ctx, uint32_t* host_out) {
     if (!ctx || !host_out) return OMSE_EINVAL;
@@ -193,36 +250,92 @@ int omse_last_device_status(omse_ctx* ctx, uint32_t* host_out) {
 int omse_quantize_weights(omse_ctx* ctx, const float* d_w, int64_t n_kernels, int64_t kernel_len, int bits,
                           int is_signed, const omse_grid* grid, float* d_alpha, float* d_sse,
                           int32_t* d_best_idx, int8_t* d_codes, uint8_t* d_packed) {
-    if (!ctx || !grid_ok(grid) || bits < 2 || bits > 8 || n_kernels < 0 || kernel_len < 1 ||
-        kernel_len > OMSE_MAX_KERNEL_LEN || n_kernels > (int64_t)1 << 40)
+    omse_weight_tensor t;
+    t.d_w = d_w;
+    t.n_kernels = n_kernels;
+    t.kernel_len = kernel_len;
+    t.d_alpha = d_alpha;
+    t.d_sse = d_sse;
+    t.d_best_idx = d_best_idx;
+    t.d_codes = d_codes;
+    t.d_packed = d_packed;
+    return omse_quantize_weights_batched(ctx, &t, 1, bits, is_signed, grid);
+}
+
+int omse_quantize_weights_batched(omse_ctx* ctx, const omse_weight_tensor* tensors, int n_tensors, int bits,
+                                  int is_signed, const omse_grid* grid) {
+    if (!ctx || !grid_ok(grid) || bits < 2 || bits > 8 || n_tensors < 0 || n_tensors > OMSE_MAX_BATCH ||
+        (n_tensors > 0 && !tensors))
         return OMSE_EINVAL;
-    if (d_packed && bits > 4) return OMSE_EINVAL;
-    if (n_kernels == 0) return OMSE_OK;
-    if (!d_w || !d_alpha || !d_sse) return OMSE_EINVAL;
-    if ((reinterpret_cast<uintptr_t>(d_w) & 3) || (reinterpret_cast<uintptr_t>(d_alpha) & 3) ||
-        (reinterpret_cast<uintptr_t>(d_sse) & 3) || (reinterpret_cast<uintptr_t>(d_best_idx) & 3))
-        return OMSE_EINVAL;
+    std::vector<omse::RowTensor> list;
+    list.reserve((size_t)n_tensors);
+    long long max_k = 0;
+    for (int i = 0; i < n_tensors; ++i) {
+        const omse_weight_tensor& u = tensors[i];
+        if (u.n_kernels < 0 || u.kernel_len < 1 || u.kernel_len > OMSE_MAX_KERNEL_LEN || u.n_kernels > (int64_t)1 << 40)
+            return OMSE_EINVAL;
+        if (u.d_packed && bits > 4) return OMSE_EINVAL;
+        if (u.n_kernels == 0) continue;
+        if (!u.d_w || !u.d_alpha || !u.d_sse) return OMSE_EINVAL;
+        if (misaligned4(u.d_w) || misaligned4(u.d_alpha) || misaligned4(u.d_sse) || misaligned4(u.d_best_idx))
+            return OMSE_EINVAL;
+        omse::RowTensor t;
+        fill_tensor(t, u.d_w, u.n_kernels, u.kernel_len, u.d_alpha, u.d_sse, u.d_best_idx, u.d_codes, u.d_packed);
+        list.push_back(t);
+        if (u.kernel_len > max_k) max_k = u.kernel_len;
+    }
+    if (list.empty()) return OMSE_OK;
     if (cudaSetDevice(ctx->device) != cudaSuccess) return OMSE_ECUDA;
+    // Short rows are batched per work unit when the block is a single element group and the launch
+    // still has a few work units per SM afterwards (otherwise one row per block fills the GPU better).
+    size_t smem_small = 0;
+    if (single_group(grid->n_cand, max_k)) {
+        const int cpt = cpt_for(grid->n_cand);
+        const int ncs = cpt * group_threads(grid->n_cand);
+        long long units_if_small = 0;
+        for (const auto& t : list) {
+            const int b = t.K > OMSE_SMALL_K ? t.rows_per_unit : (t.K <= 128 ? 8 : 4);
+            units_if_small += (t.S + b - 1) / b;
+        }
+        if (units_if_small >= 4ll * ctx->n_sm) {
+            for (auto& t : list) {
+                if (t.K > OMSE_SMALL_K) continue;
+                t.small = 1;
+                t.rows_per_unit = t.K <= 128 ? 8 : 4;
+                const size_t kpad = (size_t)((t.K + 3) & ~3ll);
+                const size_t need = (size_t)t.rows_per_unit * (kpad * 4 + (size_t)ncs * 4 + 8);
+                if (need > smem_small) smem_small = need;
+            }
+        }
+    }
+    // longest rows first: the dispenser then hands out work in decreasing size and the tail is short
+    std::stable_sort(list.begin(), list.end(), [](const omse::RowTensor& x, const omse::RowTensor& y) { return x.K > y.K; });
+    long long units = 0;
+    for (auto& t : list) {
+        t.unit_begin = units;
+        units += (t.S + t.rows_per_unit - 1) / t.rows_per_unit;
+    }
     omse::RowArgs a;
     memset(&a, 0, sizeof(a));
-    a.w = d_w;
-    a.S = n_kernels;
-    a.K = kernel_len;
+    a.n_launch_tensors = (int)list.size();
+    a.n_units = units;
+    if (list.size() == 1) {
+        a.tensors = nullptr;
+        a.one = list[0];
+    } else {
+        if (cudaMemcpyAsync(ctx->d_tensors, list.data(), sizeof(omse::RowTensor) * list.size(), cudaMemcpyHostToDevice,
+                            ctx->stream) != cudaSuccess)
+            return OMSE_ECUDA;
+        a.tensors = ctx->d_tensors;
+    }
     a.n_cand = grid->n_cand;
     a.hi_frac = grid->hi_frac;
     a.refine_iters = grid->refine_iters;
     a.n_tensors = 1;
     a.n_sweeps = 1;
     bounds(bits, is_signed, &a.lo[0], &a.hi[0]);
-    a.alpha = d_alpha;
-    a.sse = d_sse;
-    a.best_idx = d_best_idx;
-    a.codes = reinterpret_cast<signed char*>(d_codes);
-    a.packed = d_packed;
-    a.status = &ctx->ws->status;
-    a.rows_per_unit = (d_packed && (kernel_len & 1)) ? 2 : 1;
     a.keep_x0 = 0;
-    return launch_rows(ctx, a);
+    return launch_rows(ctx, a, max_k, smem_small);
 }
 
 int omse_residual_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, int64_t kernel_len, const int* bits,
@@ -239,30 +352,22 @@ int omse_residual_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, i
     if (n_sweeps > 1 && (!d_codes || kernel_len > OMSE_MAX_KERNEL_LEN_MULTISWEEP)) return OMSE_EINVAL;
     if (n_kernels == 0) return OMSE_OK;
     if (!d_t || !d_alpha || !d_sse) return OMSE_EINVAL;
-    if ((reinterpret_cast<uintptr_t>(d_t) & 3) || (reinterpret_cast<uintptr_t>(d_alpha) & 3) ||
-        (reinterpret_cast<uintptr_t>(d_sse) & 3))
-        return OMSE_EINVAL;
+    if (misaligned4(d_t) || misaligned4(d_alpha) || misaligned4(d_sse)) return OMSE_EINVAL;
     if (cudaSetDevice(ctx->device) != cudaSuccess) return OMSE_ECUDA;
     omse::RowArgs a;
     memset(&a, 0, sizeof(a));
-    a.w = d_t;
-    a.S = n_kernels;
-    a.K = kernel_len;
+    fill_tensor(a.one, d_t, n_kernels, kernel_len, d_alpha, d_sse, nullptr, d_codes, d_packed);
+    a.tensors = nullptr;
+    a.n_launch_tensors = 1;
+    a.n_units = (n_kernels + a.one.rows_per_unit - 1) / a.one.rows_per_unit;
     a.n_cand = grid->n_cand;
     a.hi_frac = grid->hi_frac;
     a.refine_iters = grid->refine_iters;
     a.n_tensors = n_tensors;
     a.n_sweeps = n_sweeps;
     for (int j = 0; j < n_tensors; ++j) bounds(bits[j], is_signed, &a.lo[j], &a.hi[j]);
-    a.alpha = d_alpha;
-    a.sse = d_sse;
-    a.best_idx = nullptr;
-    a.codes = reinterpret_cast<signed char*>(d_codes);
-    a.packed = d_packed;
-    a.status = &ctx->ws->status;
-    a.rows_per_unit = (d_packed && (kernel_len & 1)) ? 2 : 1;
     a.keep_x0 = n_sweeps > 1 ? 1 : 0;
-    return launch_rows(ctx, a);
+    return launch_rows(ctx, a, kernel_len);
 }
 
 int omse_activation_scale(omse_ctx* ctx, const float* d_x, int64_t n, int bits, int is_signed, const omse_grid* grid,

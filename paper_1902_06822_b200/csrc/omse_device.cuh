@@ -19,7 +19,14 @@ namespace omse {
 typedef unsigned long long u64;
 
 constexpr float kMagic = 12582912.0f;   // 1.5 * 2^23
-constexpr int kFlushEvery4 = 32;        // float4 loads between folds of the fp32 partial sums into fp64
+#ifndef OMSE_FLUSH4
+#define OMSE_FLUSH4 32
+#endif
+#ifndef OMSE_UNROLL
+#define OMSE_UNROLL 2
+#endif
+constexpr int kUnroll = OMSE_UNROLL;      // float4 loads per unrolled step of the sweep loop
+constexpr int kFlushEvery4 = OMSE_FLUSH4;   // float4 loads between folds of the fp32 partial sums into fp64
 constexpr int kListCap = 32;            // most near-minimal candidates re-scored in fp64
 constexpr double kRescoreBand = 4e-6;   // candidates within this relative band of the fp32 minimum are re-scored
 
@@ -68,7 +75,7 @@ __device__ __forceinline__ void sweep_range(const float4* __restrict__ xs4, int 
     int i = beg4;
     while (i < end4) {
         const int stop = min(end4, i + kFlushEvery4);
-#pragma unroll 2
+#pragma unroll(kUnroll)
         for (; i < stop; ++i) {
             const float4 v = xs4[i];
             const u64 xa = pack2(v.x, v.y), xb = pack2(v.z, v.w);

@@ -4,27 +4,50 @@
 #pragma once
 #include "omse_device.cuh"
 
+#ifndef OMSE_ROWS_MAX_THREADS
+#define OMSE_ROWS_MAX_THREADS 512
+#endif
+
 namespace omse {
 
-struct RowArgs {
-    const float* w;        // [S][K]
+// One weight tensor of a launch (Section 3.1: W_l = {W_lk}, row k is kernel W_lk flattened).
+struct RowTensor {
+    const float* w;          // [S][K]
     long long S, K;
+    float* alpha;            // [n_tensors][S]
+    float* sse;              // [n_tensors][S]
+    int* best_idx;           // [S] (single quantized tensor only), nullable
+    signed char* codes;      // [n_tensors][N], nullable
+    unsigned char* packed;   // [n_tensors][ceil(N/2)], nullable
+    long long unit_begin;    // index of this tensor's first work unit in the launch-wide numbering
+    int rows_per_unit;       // long rows: 2 when nibble packing needs an even element count per unit (odd K), else 1;
+                             // short rows: the batch size B (even)
+    int small;               // 1: short-row path (batch of rows per unit, a warp finishes each row)
+};
+
+struct RowArgs {
+    const RowTensor* tensors;   // device array, ordered by decreasing K (longest rows are handed out first)
+    RowTensor one;              // the tensor itself when n_tensors_in_launch == 1 (tensors == nullptr)
+    int n_launch_tensors;
+    long long n_units;          // work units in the launch
+    unsigned long long* ticket; // [2] next unit to hand out, blocks finished; both return to 0 at kernel end
     int n_cand;
     float hi_frac;
     int refine_iters;
-    int n_tensors, n_sweeps;
-    int lo[4], hi[4];      // grid bounds per tensor (Section 3.1)
-    float* alpha;          // [n_tensors][S]
-    float* sse;            // [n_tensors][S]
-    int* best_idx;         // [S] (single tensor only), nullable
-    signed char* codes;    // [n_tensors][N], nullable
-    unsigned char* packed; // [n_tensors][ceil(N/2)], nullable
+    int n_tensors, n_sweeps;    // Algorithm 1: quantized tensors per row, sweeps
+    int lo[4], hi[4];           // grid bounds per quantized tensor (Section 3.1)
     unsigned int* status;
-    int groups;            // element groups per block
-    int tg;                // threads per group (multiple of 32); candidate c = slot*tg + t
-    int rows_per_unit;     // 2 when nibble packing needs an even element count per unit (odd K)
-    int keep_x0;           // n_sweeps > 1: keep the original row next to the residual
+    int groups;                 // element groups per block
+    int tg;                     // threads per group (multiple of 32); candidate c = slot*tg + t
+    int keep_x0;                // n_sweeps > 1: keep the original row next to the residual
+    int max_k4;                 // float4s of the longest row in the launch (shared-memory carve-up)
 };
+
+}  // namespace omse
+
+#include "omse_rows_small.cuh"
+
+namespace omse {
 
 struct PhiOut {
     float alpha;
@@ -45,7 +68,8 @@ struct RowSmem {
 
 // The quantization mapping phi of Section 3.4 on the row held in s.xs (k elements, k4 float4s).
 template <int CPT>
-__device__ PhiOut phi_block(const RowArgs& a, const RowSmem& s, int k, int k4, float flo, float fhi) {
+__device__ PhiOut phi_block(const RowArgs& a, const RowSmem& s, int k, int k4, float flo, float fhi,
+                             const float (&rcp)[CPT]) {
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int grp = tid / a.tg, t = tid - grp * a.tg;
     const float4* xs4 = reinterpret_cast<const float4*>(s.xs);
@@ -77,7 +101,7 @@ __device__ PhiOut phi_block(const RowArgs& a, const RowSmem& s, int k, int k4, f
     for (int sl = 0; sl < CPT; ++sl) {
         const int c = sl * a.tg + t;
         const float ac = __fmul_rn((float)(c + 1), g.step);
-        float inv = g.tiny ? __fdiv_rn(1.0f, ac) : __fdiv_rn(1.0f, (float)(c + 1)) * g.rstep;
+        float inv = g.tiny ? __fdiv_rn(1.0f, ac) : rcp[sl] * g.rstep;
         if (!(ac >= FLT_MIN) || c >= a.n_cand) inv = 0.f;  // unusable: evaluated harmlessly, discarded below
         inv2[sl] = pack2(inv, inv);
         na2[sl] = pack2(-ac, -ac);
@@ -252,31 +276,55 @@ __device__ double emit_block(const RowSmem& s, int k, float alpha, float flo, fl
 }
 
 template <int CPT>
-__global__ void __launch_bounds__(512) rows_kernel(const RowArgs a) {
+__global__ void __launch_bounds__(OMSE_ROWS_MAX_THREADS) rows_kernel(const RowArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ unsigned long long s_unit;
     const int tid = threadIdx.x, nthr = blockDim.x;
-    const int k = (int)a.K;
-    const int k4 = (k + 3) >> 2;
     RowSmem s;
     s.xs = reinterpret_cast<float*>(smem_raw);
-    s.x0 = s.xs + (a.keep_x0 ? 4 * k4 : 0);
-    s.xg = reinterpret_cast<double*>(s.x0 + 4 * k4);
+    s.x0 = s.xs + (a.keep_x0 ? 4 * a.max_k4 : 0);
+    s.xg = reinterpret_cast<double*>(s.x0 + 4 * a.max_k4);
     s.scratch = s.xg + (size_t)(a.groups - 1) * CPT * a.tg;
     s.list = reinterpret_cast<int*>(s.scratch + 64);
     s.misc = s.list + kListCap;
-    const long long n_total = a.S * a.K;
-    const long long n_units = (a.S + a.rows_per_unit - 1) / a.rows_per_unit;
-    const long long packed_stride = (n_total + 1) >> 1;
     unsigned int st = 0;
 
-    for (long long unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
-        for (int ru = 0; ru < a.rows_per_unit; ++ru) {
-            const long long row = unit * a.rows_per_unit + ru;
-            if (row >= a.S) break;
-            const bool more = (ru + 1 < a.rows_per_unit) && (row + 1 < a.S);
-            const long long row_base = row * a.K;
-            const float* src = a.w + row_base;
-            __syncthreads();   // previous row fully consumed
+    // 1/(c+1) for this thread's candidates: 1/alpha_c = (1/(c+1)) * (1/step) to within 2 ulp
+    float rcp[CPT];
+#pragma unroll
+    for (int sl = 0; sl < CPT; ++sl) rcp[sl] = __fdiv_rn(1.0f, (float)(sl * a.tg + (tid % a.tg) + 1));
+
+    for (;;) {
+        __syncthreads();   // previous unit fully consumed (shared row, s_unit)
+        if (tid == 0) s_unit = atomicAdd(a.ticket, 1ull);
+        __syncthreads();
+        const long long unit = (long long)s_unit;
+        if (unit >= a.n_units) break;
+        // ---- which tensor this unit belongs to (tensors are few: linear scan from the end)
+        const RowTensor* tp = &a.one;
+        if (a.tensors) {
+            int ti = a.n_launch_tensors - 1;
+            while (ti > 0 && a.tensors[ti].unit_begin > unit) --ti;
+            tp = a.tensors + ti;
+        }
+        const RowTensor& T = *tp;
+        if (T.small) {
+            small_unit<CPT>(a, T, unit - T.unit_begin, smem_raw, rcp, st);
+            continue;
+        }
+        const int k = (int)T.K;
+        const int k4 = (k + 3) >> 2;
+        const long long n_total = T.S * T.K;
+        const long long packed_stride = (n_total + 1) >> 1;
+        const long long unit_local = unit - T.unit_begin;
+
+        for (int ru = 0; ru < T.rows_per_unit; ++ru) {
+            const long long row = unit_local * T.rows_per_unit + ru;
+            if (row >= T.S) break;
+            const bool more = (ru + 1 < T.rows_per_unit) && (row + 1 < T.S);
+            const long long row_base = row * T.K;
+            const float* src = T.w + row_base;
+            if (ru > 0) __syncthreads();   // previous row of the unit fully consumed
             // ---- stage the row once from HBM (128-bit loads when the row start allows it)
             bool bad = false;
             if ((reinterpret_cast<unsigned long long>(src) & 15ull) == 0) {
@@ -315,24 +363,24 @@ __global__ void __launch_bounds__(512) rows_kernel(const RowArgs a) {
                             float v = s.x0[i];
                             for (int i2 = 0; i2 < a.n_tensors; ++i2) {
                                 if (i2 == j || (sweep == 0 && i2 > j)) continue;
-                                const float ai = a.alpha[(long long)i2 * a.S + row];
-                                const float qi = (float)a.codes[(long long)i2 * n_total + row_base + i];
+                                const float ai = T.alpha[(long long)i2 * T.S + row];
+                                const float qi = (float)T.codes[(long long)i2 * n_total + row_base + i];
                                 v = fmaf(-ai, qi, v);
                             }
                             s.xs[i] = v;
                         }
                         __syncthreads();
                     }
-                    PhiOut r = phi_block<CPT>(a, s, k, k4, flo, fhi);
+                    PhiOut r = phi_block<CPT>(a, s, k, k4, flo, fhi, rcp);
                     if (r.degenerate) st |= 2u;
                     const double sse = emit_block(s, k, r.alpha, flo, fhi,
-                                                  a.codes ? a.codes + (long long)j * n_total : nullptr,
-                                                  a.packed ? a.packed + (long long)j * packed_stride : nullptr,
+                                                  T.codes ? T.codes + (long long)j * n_total : nullptr,
+                                                  T.packed ? T.packed + (long long)j * packed_stride : nullptr,
                                                   row_base, &s.misc[1 + j], more);
                     if (tid == 0) {
-                        a.alpha[(long long)j * a.S + row] = r.alpha;
-                        a.sse[(long long)j * a.S + row] = (float)sse;
-                        if (a.best_idx && j == 0) a.best_idx[row] = r.idx;
+                        T.alpha[(long long)j * T.S + row] = r.alpha;
+                        T.sse[(long long)j * T.S + row] = (float)sse;
+                        if (T.best_idx && j == 0) T.best_idx[row] = r.idx;
                     }
                     if (!a.keep_x0 && j + 1 < a.n_tensors) {
                         // first sweep without a kept copy: the residual is updated in place
@@ -348,6 +396,16 @@ __global__ void __launch_bounds__(512) rows_kernel(const RowArgs a) {
         }
     }
     if (st) atomicOr(a.status, st);   // any thread that saw a flag reports it
+    // ---- the last block to leave re-arms the ticket pair for the next launch (no block waits)
+    if (tid == 0) {
+        __threadfence();
+        const unsigned long long done = atomicAdd(a.ticket + 1, 1ull);
+        if (done == (unsigned long long)gridDim.x - 1ull) {
+            a.ticket[0] = 0ull;
+            a.ticket[1] = 0ull;
+            __threadfence();
+        }
+    }
 }
 
 }  // namespace omse

@@ -1,0 +1,289 @@
+// Short kernels (rows of a few dozen to a few hundred weights): the per-row fixed costs of the
+// block-cooperative path (barriers, reductions, global round trips) would dominate, so a work unit
+// here is a batch of B consecutive rows: staged together, swept one after the other by the whole
+// block (error curve of each row kept in shared memory), then finished by one warp per row with
+// shuffle reductions only.  Results are identical in meaning to the long-row path: same candidate
+// arithmetic, same fp64 re-scoring of near-minimal candidates, same polish and emission.
+#pragma once
+#include "omse_device.cuh"
+
+namespace omse {
+
+__device__ __forceinline__ double warp_allsum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;   // a + b == b + a: every lane ends with the same bits
+}
+__device__ __forceinline__ int warp_allsum(int v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// One row, one warp: argmin of the stored curve, re-score, polish, final codes, outputs.
+// xr: the row in shared memory (k elements), cv: its error curve (n_cand floats).
+// prev_x_last / prev_alpha: last element and final scale of the previous row when this row starts
+// at an odd flat index (its first nibble shares a byte with that element); more: the next row will
+// complete this row's last byte.
+__device__ __forceinline__ float small_row_epilogue(const RowArgs& a, const RowTensor& T, const float* xr,
+                                                    const float* cv, int k, float mpos, float mneg, long long row,
+                                                    float prev_x_last, float prev_alpha, bool more,
+                                                    unsigned int& st) {
+    const int lane = threadIdx.x & 31;
+    const float flo = (float)a.lo[0], fhi = (float)a.hi[0];
+    const GridSetup g = grid_setup(mpos, mneg, a.hi_frac, a.n_cand, flo, fhi);
+    const float m = fmaxf(mpos, mneg);
+    const float a_last = __fmul_rn((float)a.n_cand, g.step);
+    float alpha = 0.f;
+    int best = -1;
+    bool degenerate = !(m > 0.f) || !(a_last >= FLT_MIN);
+    if (!degenerate) {
+        float bv = INFINITY;
+        int bi = 0x7fffffff;
+        for (int c = lane; c < a.n_cand; c += 32) {
+            const float v = cv[c];
+            if (v < bv) {
+                bv = v;
+                bi = c;
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (ov < bv || (ov == bv && oi < bi)) {
+                bv = ov;
+                bi = oi;
+            }
+        }
+        if (bi == 0x7fffffff) {
+            degenerate = true;   // every error Inf/NaN: non-finite input
+        } else {
+            best = bi;
+            const float band = (float)((double)bv * (1.0 + kRescoreBand));
+            int cnt = 0;
+            for (int c = lane; c < a.n_cand; c += 32) cnt += (cv[c] <= band) ? 1 : 0;
+            cnt = warp_allsum(cnt);
+            if (cnt > 1 && cnt <= kListCap) {
+                double best_sse = INFINITY;
+                best = 0x7fffffff;
+                for (int c0 = 0; c0 < a.n_cand; c0 += 32) {
+                    const float v = (c0 + lane < a.n_cand) ? cv[c0 + lane] : INFINITY;
+                    unsigned int mask = __ballot_sync(0xffffffffu, v <= band);
+                    while (mask) {
+                        const int c = c0 + __ffs(mask) - 1;
+                        mask &= mask - 1;
+                        const float ac = __fmul_rn((float)(c + 1), g.step);
+                        double ss = 0.0;
+                        for (int i = lane; i < k; i += 32) {
+                            const float x = xr[i];
+                            const double d = (double)x - (double)ac * (double)code_of(x, ac, flo, fhi);
+                            ss += d * d;
+                        }
+                        ss = warp_allsum(ss);
+                        if (ss < best_sse || (ss == best_sse && c < best)) {
+                            best_sse = ss;
+                            best = c;
+                        }
+                    }
+                }
+            }
+            alpha = __fmul_rn((float)(best + 1), g.step);
+            for (int it = 0; it < a.refine_iters; ++it) {
+                double sxq = 0.0;
+                int sqq = 0;
+                for (int i = lane; i < k; i += 32) {
+                    const float x = xr[i];
+                    const int q = code_of(x, alpha, flo, fhi);
+                    sqq += q * q;
+                    sxq += (double)x * (double)q;
+                }
+                sxq = warp_allsum(sxq);
+                sqq = warp_allsum(sqq);
+                if (sqq == 0) break;
+                const float a_new = (float)(sxq / (double)sqq);
+                if (!(a_new >= FLT_MIN) || !(a_new <= FLT_MAX)) break;
+                alpha = a_new;
+            }
+        }
+    }
+    if (degenerate) {
+        st |= 2u;
+        alpha = 0.f;
+        best = -1;
+    }
+
+    // ---- final codes, squared error, emission
+    const long long row_base = row * T.K;
+    const bool zero = !(alpha > 0.f);
+    double ss = 0.0;
+    const bool aligned = ((reinterpret_cast<unsigned long long>(T.codes) & 3ull) == 0) &&
+                         ((reinterpret_cast<unsigned long long>(T.packed) & 1ull) == 0);
+    if ((k & 3) == 0 && aligned) {
+        const float4* xr4 = reinterpret_cast<const float4*>(xr);
+        for (int i4 = lane; i4 < (k >> 2); i4 += 32) {
+            const float4 v = xr4[i4];
+            const float x[4] = {v.x, v.y, v.z, v.w};
+            int q[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                q[e] = zero ? 0 : code_of(x[e], alpha, flo, fhi);
+                const double d = (double)x[e] - (double)alpha * (double)q[e];
+                ss += d * d;
+            }
+            if (T.codes) {
+                const unsigned int w = (q[0] & 0xff) | ((q[1] & 0xff) << 8) | ((q[2] & 0xff) << 16) | ((unsigned)(q[3] & 0xff) << 24);
+                *reinterpret_cast<unsigned int*>(T.codes + row_base + 4ll * i4) = w;
+            }
+            if (T.packed) {
+                const unsigned short h = (unsigned short)((q[0] & 0xf) | ((q[1] & 0xf) << 4) | ((q[2] & 0xf) << 8) | ((q[3] & 0xf) << 12));
+                *reinterpret_cast<unsigned short*>(T.packed + ((row_base + 4ll * i4) >> 1)) = h;
+            }
+        }
+    } else {
+        const int o = (int)(row_base & 1);
+        const int n_pairs = (k + o + 1) >> 1;
+        for (int p = lane; p < n_pairs; p += 32) {
+            const int e0 = 2 * p - o, e1 = e0 + 1;
+            int q0 = 0, q1 = 0;
+            if (e0 >= 0) {
+                const float x = xr[e0];
+                q0 = zero ? 0 : code_of(x, alpha, flo, fhi);
+                const double d = (double)x - (double)alpha * (double)q0;
+                ss += d * d;
+                if (T.codes) T.codes[row_base + e0] = (signed char)q0;
+            } else {
+                q0 = prev_alpha > 0.f ? code_of(prev_x_last, prev_alpha, flo, fhi) : 0;
+            }
+            const bool has1 = e1 < k;
+            if (has1) {
+                const float x = xr[e1];
+                q1 = zero ? 0 : code_of(x, alpha, flo, fhi);
+                const double d = (double)x - (double)alpha * (double)q1;
+                ss += d * d;
+                if (T.codes) T.codes[row_base + e1] = (signed char)q1;
+            }
+            if (T.packed && (has1 || !more))
+                T.packed[(row_base + e0) >> 1] = (unsigned char)((q0 & 0xf) | ((q1 & 0xf) << 4));
+        }
+    }
+    ss = warp_allsum(ss);
+    if (lane == 0) {
+        T.alpha[row] = alpha;
+        T.sse[row] = (float)ss;
+        if (T.best_idx) T.best_idx[row] = best;
+    }
+    return alpha;
+}
+
+// One work unit of the short-row path: rows [unit_local*B, +B) of tensor T.  Requires a single
+// element group (blockDim.x == a.tg) and a single quantized tensor per row.
+template <int CPT>
+__device__ void small_unit(const RowArgs& a, const RowTensor& T, long long unit_local, unsigned char* smem_raw,
+                           const float (&rcp)[CPT], unsigned int& st) {
+    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
+    const int k = (int)T.K, kpad = (k + 3) & ~3, k4 = kpad >> 2;
+    const int B = T.rows_per_unit;
+    const long long row0 = unit_local * B;
+    const int nrows = (int)min((long long)B, T.S - row0);
+    const int ncs = CPT * a.tg;
+    float* xs = reinterpret_cast<float*>(smem_raw);
+    float* curve = xs + B * kpad;
+    float* rmax = curve + B * ncs;
+    const float flo = (float)a.lo[0], fhi = (float)a.hi[0];
+
+    // ---- stage the rows (contiguous in HBM) into rows of kpad floats, zero padded
+    const float* src = T.w + row0 * T.K;
+    const int n_el = nrows * k;
+    bool bad = false;
+    if ((k & 3) == 0 && (reinterpret_cast<unsigned long long>(src) & 15ull) == 0) {
+        const float4* src4 = reinterpret_cast<const float4*>(src);
+        for (int i4 = tid; i4 < (n_el >> 2); i4 += nthr) {
+            const float4 v = __ldg(src4 + i4);
+            reinterpret_cast<float4*>(xs)[i4] = v;
+            bad |= !(fabsf(v.x) <= FLT_MAX) || !(fabsf(v.y) <= FLT_MAX) || !(fabsf(v.z) <= FLT_MAX) || !(fabsf(v.w) <= FLT_MAX);
+        }
+    } else {
+        for (int i = tid; i < n_el; i += nthr) {
+            const int r = i / k, c = i - r * k;
+            const float v = __ldg(src + i);
+            xs[r * kpad + c] = v;
+            bad |= !(fabsf(v) <= FLT_MAX);
+        }
+        const int npad = kpad - k;
+        for (int i = tid; i < nrows * npad; i += nthr) {
+            const int r = i / npad, c = k + (i - r * npad);
+            xs[r * kpad + c] = 0.f;
+        }
+    }
+    if (bad) st |= 1u;
+    __syncthreads();
+
+    // ---- max of the positive and negative part of every row: a warp per row
+    for (int r = warp; r < nrows; r += nwarp) {
+        float mp = 0.f, mn = 0.f;
+        for (int i = lane; i < k; i += 32) {
+            const float v = xs[r * kpad + i];
+            if (fabsf(v) <= FLT_MAX) {
+                mp = fmaxf(mp, v);
+                mn = fmaxf(mn, -v);
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            mp = fmaxf(mp, __shfl_xor_sync(0xffffffffu, mp, o));
+            mn = fmaxf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+        }
+        if (lane == 0) {
+            rmax[2 * r] = mp;
+            rmax[2 * r + 1] = mn;
+        }
+    }
+    __syncthreads();
+
+    // ---- candidate sweep, row after row, by the whole block; error curves to shared memory
+    for (int r = 0; r < nrows; ++r) {
+        const float mpos = rmax[2 * r], mneg = rmax[2 * r + 1];
+        const GridSetup g = grid_setup(mpos, mneg, a.hi_frac, a.n_cand, flo, fhi);
+        const float a_last = __fmul_rn((float)a.n_cand, g.step);
+        if (!(fmaxf(mpos, mneg) > 0.f) || !(a_last >= FLT_MIN)) continue;   // the epilogue reports it
+        u64 inv2[CPT], na2[CPT];
+        double dacc[CPT];
+        bool ok[CPT];
+#pragma unroll
+        for (int sl = 0; sl < CPT; ++sl) {
+            const int c = sl * a.tg + tid;
+            const float ac = __fmul_rn((float)(c + 1), g.step);
+            float inv = g.tiny ? __fdiv_rn(1.0f, ac) : rcp[sl] * g.rstep;
+            ok[sl] = (ac >= FLT_MIN) && c < a.n_cand;
+            if (!ok[sl]) inv = 0.f;
+            inv2[sl] = pack2(inv, inv);
+            na2[sl] = pack2(-ac, -ac);
+            dacc[sl] = 0.0;
+        }
+        int ncl = (g.c_sat - (tid & ~31) + a.tg - 1) / a.tg;
+        ncl = max(0, min(CPT, ncl));
+        sweep_dispatch<CPT>(ncl, reinterpret_cast<const float4*>(xs) + r * k4, 0, k4, inv2, na2, dacc,
+                            kMagic + flo, kMagic + fhi);
+#pragma unroll
+        for (int sl = 0; sl < CPT; ++sl) curve[r * ncs + sl * a.tg + tid] = ok[sl] ? (float)dacc[sl] : INFINITY;
+    }
+    __syncthreads();
+
+    // ---- a warp finishes each row; two consecutive rows stay in one warp when a packed byte can
+    //      straddle them (odd row length)
+    const int rpt = (T.packed && (k & 1)) ? 2 : 1;
+    for (int task = warp; task * rpt < nrows; task += nwarp) {
+        float prev_alpha = 0.f;
+        for (int rr = 0; rr < rpt; ++rr) {
+            const int r = task * rpt + rr;
+            if (r >= nrows) break;
+            const bool more = (rr + 1 < rpt) && (r + 1 < nrows);
+            const float prev_x_last = r > 0 ? xs[(r - 1) * kpad + k - 1] : 0.f;
+            prev_alpha = small_row_epilogue(a, T, xs + r * kpad, curve + r * ncs, k, rmax[2 * r], rmax[2 * r + 1],
+                                            row0 + r, prev_x_last, prev_alpha, more, st);
+        }
+    }
+}
+
+}  // namespace omse

@@ -31,15 +31,28 @@ def _sample_rows(w, frac, seed):
 
 
 def test_resnet50_weight_set_every_row(gpu):
-    """configs[1]: all 54 tensors, signed 4-bit, 1024 candidates, packed INT4 out; every row checked."""
+    """configs[1]: all 54 tensors in one batched launch (as the benchmark does), signed 4-bit,
+    1024 candidates, packed INT4 out; every row checked."""
+    import torch
+    weights = synth.resnet50_weights(seed=2)
+    descs = []
+    for name, w in weights:
+        s, k = w.shape
+        descs.append(dict(w=torch.from_numpy(w).cuda(), n_kernels=s, kernel_len=k,
+                          alpha=torch.full((s,), -1.0, device="cuda"), sse=torch.full((s,), -1.0, device="cuda"),
+                          best_idx=torch.full((s,), -7, dtype=torch.int32, device="cuda"),
+                          packed=torch.full(((s * k + 1) // 2,), 0xAB, dtype=torch.uint8, device="cuda")))
+    gpu.ctx().omse_quantize_weights_batched(descs, 4, True, 1024, 1.0, 3)
+    torch.cuda.synchronize()
     total_rows, diff = 0, 0
-    for name, w in synth.resnet50_weights(seed=2):
-        alpha, sse, idx, q, pk = gpu.quantize_weights(w, 4, True, 1024, 1.0, 3, want_codes=False, want_packed=True)
-        st = check_rows(w, alpha, sse, idx, None, pk, 4, True, 1024, 1.0, 3)
+    for (name, w), d in zip(weights, descs):
+        st = check_rows(w, d["alpha"].cpu().numpy(), d["sse"].cpu().numpy(), d["best_idx"].cpu().numpy(), None,
+                        d["packed"].cpu().numpy(), 4, True, 1024, 1.0, 3)
         total_rows += st["rows"]
         diff += st["idx_diff"]
         assert st["alpha_bitwise"] >= 0.99, (name, st)
     assert total_rows == 27560 and diff <= 27
+    assert gpu.ctx().omse_last_device_status() == 0
 
 
 @pytest.mark.parametrize("k,bits", [(27, 4), (25088, 2)])

@@ -198,3 +198,37 @@ def test_algorithm_1_two_sweeps_matches_oracle(gpu):
     same = np.all(alpha == ref.alpha, axis=0)
     assert same.mean() >= 0.9
     assert np.array_equal(q.reshape(2, 12, 300)[:, same], ref.codes[:, same])
+
+
+# ---------------------------------------------------------------- several tensors in one launch
+def test_batched_launch_matches_per_tensor_results(gpu):
+    import torch
+    shapes = [(7, 147), (33, 64), (5, 4608), (0, 32), (64, 576), (19, 27), (3, 1000)]
+    hosts, descs = [], []
+    for i, (s, k) in enumerate(shapes):
+        w = synth.laplace(max(s * k, 1), 0.05, seed=300, tensor_id=i)[:s * k].reshape(s, k)
+        hosts.append(w)
+        descs.append(dict(w=torch.from_numpy(np.ascontiguousarray(w)).cuda() if s else torch.zeros(1, device="cuda"),
+                          n_kernels=s, kernel_len=k,
+                          alpha=torch.full((max(s, 1),), -1.0, device="cuda"),
+                          sse=torch.full((max(s, 1),), -1.0, device="cuda"),
+                          best_idx=torch.full((max(s, 1),), -7, dtype=torch.int32, device="cuda"),
+                          codes=torch.full((max(s * k, 1),), 99, dtype=torch.int8, device="cuda"),
+                          packed=torch.full(((s * k + 1) // 2 + 1,), 0xAB, dtype=torch.uint8, device="cuda")))
+    gpu.ctx().omse_quantize_weights_batched(descs, 4, True, 1024, 1.0, 3)
+    torch.cuda.synchronize()
+    for w, d in zip(hosts, descs):
+        s, k = w.shape
+        if s == 0:
+            continue
+        pk = d["packed"].cpu().numpy()
+        assert pk[-1] == 0xAB
+        check_rows(w, d["alpha"].cpu().numpy(), d["sse"].cpu().numpy(), d["best_idx"].cpu().numpy(),
+                   d["codes"].cpu().numpy(), pk[:-1], 4, True, 1024, 1.0, 3)
+        one = gpu.quantize_weights(w, 4, True, 1024, 1.0, 3, True, True)   # same call, tensor by tensor
+        assert np.array_equal(one[0], d["alpha"].cpu().numpy()) and np.array_equal(one[3], d["codes"].cpu().numpy())
+    # the dispenser is back at zero: a second launch on the same context gives the same answer
+    before = descs[2]["alpha"].clone()
+    gpu.ctx().omse_quantize_weights_batched(descs, 4, True, 1024, 1.0, 3)
+    torch.cuda.synchronize()
+    assert torch.equal(before, descs[2]["alpha"])

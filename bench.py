@@ -28,6 +28,9 @@ sys.path.insert(0, ROOT)
 
 N_CAND, BITS, REFINE, HI_FRAC = 1024, 4, 3, 1.0
 INSTR_PER_EVAL = 6            # reference FP32 sequence per (element, candidate): 3 fma + 2 min/max + 1 add
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the timed kernel, from the ncu capture summarised
+# in profiles/rows_kernel_resnet50_weight_set.md; set to None whenever the kernel changes after the capture
+NCU_TRAFFIC_BYTES = None
 N_SM, LANES_PER_SM = 148, 128
 WORKLOAD = "resnet50_weight_set_54_tensors_25.5M_params_signed4bit_kernelwise_1024cand_3refine_packed"
 
@@ -91,6 +94,25 @@ class ClockSampler:
         return out
 
 
+def max_over_ranks(ms_local: float, dist, device) -> float:
+    """Slowest rank's time (every multi-GPU number is the max over ranks); identity without a process group."""
+    if dist is None:
+        return ms_local
+    import torch
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(n_per_rank: int, world: int, ms_total: float, steps: int) -> float:
+    """Elements per second over all ranks: each rank quantizes its own copy of the set (weak scaling)."""
+    return world * n_per_rank / (ms_total * 1e-3 / steps)
+
+
+def rank_seed(rank: int) -> int:
+    return 2 + 1000 * rank
+
+
 def _cpu_sample(weights):
     """Every fourth kernel of every tensor: the bounded sample the oracle is timed on."""
     return [np.ascontiguousarray(w[::4]) for _, w in weights]
@@ -144,7 +166,7 @@ def run_ours(args, rank, world):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
-    weights = synth.resnet50_weights(seed=2 + 1000 * rank)
+    weights = synth.resnet50_weights(seed=rank_seed(rank))
     n_total = sum(w.size for _, w in weights)
     ctx = binding.Context(local)
     stream = torch.cuda.current_stream(dev)
@@ -190,12 +212,7 @@ def run_ours(args, rank, world):
             fn()
             s1.record(stream)
         barrier()
-        ms = sum(s0.elapsed_time(s1) for s0, s1 in ev)
-        if dist is not None:
-            t = torch.tensor([ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(sum(s0.elapsed_time(s1) for s0, s1 in ev), dist, dev)
 
     sampler = ClockSampler(local) if rank == 0 else None
     for _ in range(max(args.warmup, 3)):
@@ -210,7 +227,7 @@ def run_ours(args, rank, world):
     if rank == 0:
         sm_max_mhz, peak_src = _peaks()
         per_step_s = ms * 1e-3 / args.steps
-        value = world * n_total / per_step_s
+        value = whole_job_value(n_total, world, ms, args.steps)
         peak = N_SM * LANES_PER_SM * sm_max_mhz * 1e6                     # FP32 lane-instructions per second
         achieved = INSTR_PER_EVAL * N_CAND * n_total / per_step_s          # algorithmic instructions per second
         h2d = sum(h.numel() * 4 for h in host_in)
@@ -223,11 +240,11 @@ def run_ours(args, rank, world):
                        "refine_iters": REFINE, "l2": "flushed between timed steps (256 MB write)",
                        "device_status": status},
             "clocks": clocks,
-            "e2e": {"value": world * n_total / (ms_e2e * 1e-3 / args.steps), "unit": "elements/s",
+            "e2e": {"value": whole_job_value(n_total, world, ms_e2e, args.steps), "unit": "elements/s",
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": args.steps,
             "roofline": {"bound": "alu", "achieved": achieved / 1e12, "peak": peak / 1e12,
-                         "unit": "T FP32-instr/s", "frac": achieved / peak, "traffic": None,
+                         "unit": "T FP32-instr/s", "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES,
                          "kernel": "rows_kernel<8>", "peak_source": f"148 SMs x 128 lanes x {sm_max_mhz:.0f} MHz ({peak_src} max clock)",
                          "instr_per_eval": INSTR_PER_EVAL},
         }

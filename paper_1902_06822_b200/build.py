@@ -33,7 +33,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not needs_build():
         return LIB_PATH
     nvcc = shutil.which("nvcc") or "/usr/local/cuda/bin/nvcc"
-    cus = [p for p in sources() if p.endswith(".cu")]
+    cus = [p for p in sources() if p.endswith(".cu") and not p.endswith("_bench.cu")]
     cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", LIB_PATH] + cus
     subprocess.run(cmd, check=True)
     return LIB_PATH

@@ -41,7 +41,8 @@ typedef enum {
     OMSE_OK = 0,
     OMSE_EINVAL = -1, /* NULL pointer, size or parameter out of range                 */
     OMSE_ECUDA = -2,  /* a CUDA runtime call or a kernel launch failed                */
-    OMSE_ENOMEM = -3  /* the context workspace could not be allocated                 */
+    OMSE_ENOMEM = -3, /* the context workspace could not be allocated                 */
+    OMSE_ELIMIT = -4  /* a size exceeds the fixed scratch of omse_activation_scale_static */
 } omse_status;
 
 /* bits of the device status word */
@@ -158,6 +159,37 @@ int omse_residual_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, i
  */
 int omse_pack_int4(omse_ctx* ctx, const int8_t* d_codes, int64_t n, int is_signed,
                    uint8_t* d_packed);
+
+/*
+ * omse_activation_scale without any allocation.  (The paper has no counterpart: this is a property
+ * of the library, not of the method.)
+ *
+ * Who needs it: code that may not call cudaMalloc when it wants a scale - a plugin running inside a
+ * host application whose memory pool already owns all device memory, a real-time or safety-certified
+ * loop that forbids allocation after start-up, a caller holding a lock under which the allocator
+ * could deadlock.  Such code cannot even create an omse_ctx, because omse_create allocates the
+ * workspace.  This entry point takes no context: the scratch of the search (search state, summed
+ * error curve, per-block partial sums) is a fixed array inside the library, OMSE_STATIC_SCRATCH_BYTES
+ * per GPU, present on every GPU that loads the library until the process exits.  The call itself
+ * performs no cudaMalloc / cudaFree and calls no allocating routine; inputs and outputs are still
+ * the caller's device buffers.
+ *
+ * Arguments are those of omse_activation_scale, with `device` / `cuda_stream` instead of the context
+ * and d_status (device, nullable): receives the OMSE_DEV_* bits of THIS call when its work completes.
+ * Limits: grid->n_cand <= OMSE_STATIC_MAX_CANDIDATES, otherwise OMSE_ELIMIT is returned and nothing
+ * is enqueued; device < 64.
+ * First call on a device: looks up the array's device address (cudaGetSymbolAddress) and the SM
+ * count and caches them; make that first call outside any stream capture.
+ * Sharing: all calls on a device use the same array.  Each call re-initialises what must start
+ * at zero, so calls that follow one another on one stream are independent; calls that can overlap
+ * on the GPU (different streams, different threads) race on the array and give wrong results.
+ * Results equal omse_activation_scale's up to the grouping of partial sums (same tolerances).
+ */
+#define OMSE_STATIC_MAX_CANDIDATES 2048
+#define OMSE_STATIC_SCRATCH_BYTES (4u * 1024u * 1024u + 32u * 1024u)
+int omse_activation_scale_static(int device, void* cuda_stream, const float* d_x, int64_t n, int bits,
+                                 int is_signed, const omse_grid* grid, float* d_alpha, float* d_sse,
+                                 int32_t* d_best_idx, double* d_sse_curve, uint32_t* d_status);
 
 /* Synchronises the stream, copies the device status word (OMSE_DEV_* bits OR-ed over all calls
  * since the last read) to *host_out and clears it. */

@@ -14,15 +14,16 @@ import torch
 
 from . import build as _build
 
-OK, EINVAL, ECUDA, ENOMEM = 0, -1, -2, -3
+OK, EINVAL, ECUDA, ENOMEM, ELIMIT = 0, -1, -2, -3, -4
 DEV_NONFINITE, DEV_DEGENERATE = 1, 2
 MAX_CANDIDATES, MAX_KERNEL_LEN, MAX_KERNEL_LEN_MULTISWEEP, MAX_TENSORS = 4096, 28672, 25600, 4
+STATIC_MAX_CANDIDATES = 2048
 
 EXPORTS = [
     "omse_create", "omse_destroy", "omse_set_stream", "omse_workspace_bytes", "omse_quantize_weights",
     "omse_quantize_weights_batched",
     "omse_activation_scale", "omse_residual_quantize", "omse_pack_int4", "omse_last_device_status",
-    "omse_status_string",
+    "omse_status_string", "omse_activation_scale_static",
 ]
 
 
@@ -64,6 +65,7 @@ def load_library() -> C.CDLL:
     lib.omse_residual_quantize.argtypes = [vp, vp, i64, i64, C.POINTER(C.c_int), i32, C.POINTER(OmseGrid), i32, i32,
                                            vp, vp, vp, vp]
     lib.omse_pack_int4.argtypes = [vp, vp, i64, i32, vp]
+    lib.omse_activation_scale_static.argtypes = [i32, vp, vp, i64, i32, i32, C.POINTER(OmseGrid), vp, vp, vp, vp, vp]
     lib.omse_last_device_status.argtypes = [vp, C.POINTER(C.c_uint32)]
     lib.omse_status_string.argtypes = [i32]
     lib.omse_status_string.restype = C.c_char_p
@@ -83,6 +85,27 @@ def _ptr(t: torch.Tensor | None, dtype: torch.dtype | None = None):
     if dtype is not None and t.dtype != dtype:
         raise ValueError(f"expected dtype {dtype}, got {t.dtype}")
     return C.c_void_p(t.data_ptr())
+
+
+def omse_activation_scale_static(x, n, bits, is_signed, n_cand, hi_frac, refine_iters, alpha, sse, best_idx=None,
+                                 sse_curve=None, status=None, stream=None):
+    """Per-tensor scale search that allocates nothing and needs no Context.
+
+    For callers that must not allocate device memory (they cannot build a Context either, since that
+    allocates the workspace): the scratch is a fixed array inside the library.  Runs on x's device and
+    on `stream` (default: torch's current stream).  At most STATIC_MAX_CANDIDATES candidates; calls that
+    may overlap on the GPU must not be issued, they share the scratch.  status: optional uint32-sized
+    CUDA tensor (dtype int32) receiving this call's device status bits.
+    """
+    dev = x.device if n > 0 else alpha.device
+    st = stream if stream is not None else torch.cuda.current_stream(dev)
+    g = OmseGrid(n_cand, hi_frac, refine_iters)
+    rc = load_library().omse_activation_scale_static(
+        dev.index or 0, C.c_void_p(st.cuda_stream), _ptr(x, torch.float32), n, bits, int(is_signed), C.byref(g),
+        _ptr(alpha, torch.float32), _ptr(sse, torch.float32), _ptr(best_idx, torch.int32),
+        _ptr(sse_curve, torch.float64), _ptr(status, torch.int32))
+    if rc != OK:
+        raise OmseError(rc, "omse_activation_scale_static")
 
 
 class Context:

@@ -6,6 +6,7 @@
 #include <algorithm>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -177,6 +178,7 @@ const char* omse_status_string(int status) {
         case OMSE_EINVAL: return "invalid argument";
         case OMSE_ECUDA: return "CUDA runtime or launch failure";
         case OMSE_ENOMEM: return "out of device memory";
+        case OMSE_ELIMIT: return "size beyond the fixed scratch of the allocation-free entry point";
         default: return "unknown status";
     }
 }
@@ -438,3 +440,145 @@ int omse_pack_int4(omse_ctx* ctx, const int8_t* d_codes, int64_t n, int is_signe
 }
 
 }  // extern "C"
+
+// -------------------------------------------------------------------------------------------------
+// Allocation-free per-tensor search (omse_activation_scale_static).  The scratch that
+// omse_activation_scale takes from the context workspace lives here in a fixed device array; every
+// GPU that loads the library holds OMSE_STATIC_SCRATCH_BYTES of it until the process exits.
+// -------------------------------------------------------------------------------------------------
+namespace {
+
+constexpr size_t kStaticPartialDoubles = 1u << 19;   // 4 MiB of per-block partial sums
+
+struct StaticScratch {
+    unsigned int status;
+    unsigned int pad_[3];
+    omse::TensorState tstate;
+    double curve[OMSE_STATIC_MAX_CANDIDATES];
+    double partials[kStaticPartialDoubles];
+};
+static_assert(sizeof(StaticScratch) <= OMSE_STATIC_SCRATCH_BYTES, "static scratch larger than documented");
+
+// In host code this name is only a handle for cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) unsigned char g_static_scratch[OMSE_STATIC_SCRATCH_BYTES];
+
+struct StaticDevice {
+    StaticScratch* ptr;   // device address of g_static_scratch on this device
+    int n_sm;
+    bool ready;
+};
+StaticDevice g_static_dev[64];
+std::mutex g_static_mutex;
+
+// Everything that must start from zero: the array keeps the previous call's contents.
+__global__ void static_begin_kernel(StaticScratch* s) {
+    if (threadIdx.x == 0) {
+        s->status = 0u;
+        s->tstate.mpos_bits = 0u;
+        s->tstate.mneg_bits = 0u;
+        s->tstate.ticket = 0u;
+        s->tstate.best_idx = -1;
+        s->tstate.alpha = 0.f;
+        s->tstate.step = 0.f;
+        s->tstate.n_list = 0;
+        s->tstate.list_overflow = 0;
+    }
+}
+
+__global__ void static_end_kernel(const StaticScratch* s, unsigned int* d_status) {
+    if (threadIdx.x == 0 && d_status) *d_status = s->status;
+}
+
+template <int CPT>
+int launch_static_sweep_t(int n_sm, cudaStream_t stream, omse::TensorArgs& a, size_t smem, int* n_blocks) {
+    const int threads = a.groups * a.tg;
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, omse::tensor_sweep_kernel<CPT>, threads, smem) != cudaSuccess || occ < 1)
+        return OMSE_ECUDA;
+    const long long n4 = (a.n + 3) >> 2;
+    const long long n_tiles = (n4 + a.tile4 - 1) / a.tile4;
+    long long grid = (long long)n_sm * occ;
+    const long long cap = (long long)(kStaticPartialDoubles / (size_t)a.n_cand);
+    if (grid > cap) grid = cap;
+    if (grid > n_tiles) grid = n_tiles;
+    if (grid < 1) grid = 1;
+    *n_blocks = (int)grid;
+    omse::tensor_sweep_kernel<CPT><<<(unsigned)grid, threads, smem, stream>>>(a);
+    return cudaGetLastError() == cudaSuccess ? OMSE_OK : OMSE_ECUDA;
+}
+
+}  // namespace
+
+extern "C" int omse_activation_scale_static(int device, void* cuda_stream, const float* d_x, int64_t n, int bits,
+                                            int is_signed, const omse_grid* grid, float* d_alpha, float* d_sse,
+                                            int32_t* d_best_idx, double* d_sse_curve, uint32_t* d_status) {
+    if (!grid_ok(grid) || bits < 2 || bits > 8 || n < 0 || !d_alpha || !d_sse || device < 0 || device >= 64)
+        return OMSE_EINVAL;
+    if (grid->n_cand > OMSE_STATIC_MAX_CANDIDATES) return OMSE_ELIMIT;
+    if (n > 0 && !d_x) return OMSE_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(d_x) & 15) || (reinterpret_cast<uintptr_t>(d_alpha) & 3) ||
+        (reinterpret_cast<uintptr_t>(d_sse) & 3) || (reinterpret_cast<uintptr_t>(d_best_idx) & 3) ||
+        (reinterpret_cast<uintptr_t>(d_sse_curve) & 7) || (reinterpret_cast<uintptr_t>(d_status) & 3))
+        return OMSE_EINVAL;
+    if (cudaSetDevice(device) != cudaSuccess) return OMSE_ECUDA;
+    StaticDevice& sd = g_static_dev[device];
+    {
+        // once per device, with that device current: the device address of the array
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!sd.ready) {
+            void* p = nullptr;
+            if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return OMSE_ECUDA;
+            if (cudaDeviceGetAttribute(&sd.n_sm, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) return OMSE_ECUDA;
+            sd.ptr = static_cast<StaticScratch*>(p);
+            sd.ready = true;
+        }
+    }
+    StaticScratch* sc = sd.ptr;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    omse::TensorArgs a;
+    memset(&a, 0, sizeof(a));
+    a.x = d_x;
+    a.n = n;
+    a.n_cand = grid->n_cand;
+    a.hi_frac = grid->hi_frac;
+    bounds(bits, is_signed, &a.lo, &a.hi);
+    const int cpt = cpt_for(a.n_cand);
+    a.tg = (((a.n_cand + cpt - 1) / cpt) + 31) & ~31;
+    a.groups = 256 / a.tg < 1 ? 1 : 256 / a.tg;
+    a.tile4 = 1024;
+    a.st = &sc->tstate;
+    a.partials = sc->partials;
+    a.curve = sc->curve;
+    a.curve_out = d_sse_curve;
+    a.alpha_out = d_alpha;
+    a.sse_out = d_sse;
+    a.idx_out = d_best_idx;
+    a.status = &sc->status;
+
+    static_begin_kernel<<<1, 32, 0, s>>>(sc);
+    long long pass_grid = (n + 1023) / 1024;
+    if (pass_grid > (long long)sd.n_sm * 8) pass_grid = (long long)sd.n_sm * 8;
+    const long long pass_cap = (long long)(kStaticPartialDoubles / (omse::kListCap + 1));
+    if (pass_grid > pass_cap) pass_grid = pass_cap;
+    if (pass_grid < 1) pass_grid = 1;
+    int n_blocks = 1;
+    if (n > 0) {
+        omse::tensor_absmax_kernel<<<(unsigned)pass_grid, 256, 0, s>>>(d_x, n, a.st, a.status);
+        const size_t smem = (size_t)a.tile4 * 16 + (size_t)(a.groups - 1) * cpt * a.tg * 8;   // < 48 KB: no opt-in needed
+        int rc;
+        switch (cpt) {
+            case 1: rc = launch_static_sweep_t<1>(sd.n_sm, s, a, smem, &n_blocks); break;
+            case 2: rc = launch_static_sweep_t<2>(sd.n_sm, s, a, smem, &n_blocks); break;
+            case 4: rc = launch_static_sweep_t<4>(sd.n_sm, s, a, smem, &n_blocks); break;
+            default: rc = launch_static_sweep_t<8>(sd.n_sm, s, a, smem, &n_blocks); break;
+        }
+        if (rc != OMSE_OK) return rc;
+    }
+    omse::tensor_finish_kernel<<<1, 1024, 0, s>>>(a, n_blocks);
+    omse::tensor_pass_kernel<0><<<(unsigned)pass_grid, 256, 0, s>>>(a);
+    for (int it = 0; it < grid->refine_iters; ++it) omse::tensor_pass_kernel<1><<<(unsigned)pass_grid, 256, 0, s>>>(a);
+    omse::tensor_pass_kernel<2><<<(unsigned)pass_grid, 256, 0, s>>>(a);
+    static_end_kernel<<<1, 32, 0, s>>>(sc, d_status);
+    return cudaGetLastError() == cudaSuccess ? OMSE_OK : OMSE_ECUDA;
+}
+

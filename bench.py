@@ -7,6 +7,9 @@ tensors goes through omse_quantize_weights_batched (stage, max, 1024-candidate s
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
+--workload selects one of the other configurations (c1, c3, c4, c5:K:bits) for measurement and
+profiling; the default c2 is the one the metric is quoted on.
+
 With N > 1 (launched under torch.distributed.run) every rank quantizes its own copy of the
 weight set (different seed): kernels of different tensors are independent, so there is no
 data-path collective; only the timing is reduced (max over ranks).
@@ -113,42 +116,192 @@ def rank_seed(rank: int) -> int:
     return 2 + 1000 * rank
 
 
-def _cpu_sample(weights):
-    """Every fourth kernel of every tensor: the bounded sample the oracle is timed on."""
-    return [np.ascontiguousarray(w[::4]) for _, w in weights]
-
-
-def _time_oracle(sample):
+# --------------------------------------------------------------------------------------------------
+# Workloads.  "c2" (the ResNet-50-shaped weight set) is the one the metric is quoted on and the
+# default; the others are the remaining configurations, selectable for measurement and profiling.
+# Every workload gives: device-resident step, end-to-end step (host buffers), byte counts, and a
+# bounded sample for the oracle.
+# --------------------------------------------------------------------------------------------------
+def _time_oracle_rows(samples, bits, n_cand, packed=True):
     from oracle import omse_oracle as orc
     orc.build()
     t0 = time.perf_counter()
-    for w in sample:
-        r = orc.quantize_rows(w, BITS, True, N_CAND, HI_FRAC, REFINE)
-        orc.pack_int4(r.codes)
+    for w in samples:
+        r = orc.quantize_rows(w, bits, True, n_cand, HI_FRAC, REFINE)
+        if packed:
+            orc.pack_int4(r.codes)
     dt = time.perf_counter() - t0
-    n = sum(w.size for w in sample)
+    n = sum(w.size for w in samples)
     return n / dt, dt, n, orc.max_threads()
 
 
+class Workload:
+    name = ""
+    n_cand = N_CAND
+    evals_per_element = 1        # quantized tensors searched per element
+    kernel = "rows_kernel<8>"
+    launches_per_step = 1
+
+    def host_arrays(self):       # list of numpy inputs
+        raise NotImplementedError
+
+
+class WeightSet(Workload):
+    """One or more weight tensors through the batched kernel-wise call."""
+
+    def __init__(self, name, tensors, bits, n_cand, packed, sample_stride, sample_desc):
+        self.name, self.tensors, self.bits, self.n_cand, self.packed = name, tensors, bits, n_cand, packed
+        self.sample_stride, self.sample_desc = sample_stride, sample_desc
+
+    def host_arrays(self):
+        return self.tensors
+
+    def setup(self, ctx, torch, dev):
+        self.host_in = [torch.from_numpy(w).pin_memory() for w in self.tensors]
+        self.d_w = [h.to(dev) for h in self.host_in]
+        self.outs = []
+        for w in self.tensors:
+            s, k = w.shape
+            code = (torch.empty((s * k + 1) // 2, dtype=torch.uint8, device=dev) if self.packed
+                    else torch.empty(s * k, dtype=torch.int8, device=dev))
+            self.outs.append((torch.empty(s, device=dev), torch.empty(s, device=dev), code))
+        self.host_out = [tuple(t.cpu().pin_memory() for t in o) for o in self.outs]
+        key = "packed" if self.packed else "codes"
+        descs = [dict(w=dw, n_kernels=w.shape[0], kernel_len=w.shape[1], alpha=a, sse=e, **{key: c})
+                 for w, dw, (a, e, c) in zip(self.tensors, self.d_w, self.outs)]
+        self.n_total = sum(w.size for w in self.tensors)
+        self.h2d = 4 * self.n_total
+        self.d2h = sum(a.numel() * 4 + e.numel() * 4 + c.numel() for a, e, c in self.outs)
+
+        def step():   # every tensor in one launch: kernels of all layers are handed out longest first
+            ctx.omse_quantize_weights_batched(descs, self.bits, True, self.n_cand, HI_FRAC, REFINE)
+        self.step = step
+
+    def step_e2e(self):
+        for hin, dw in zip(self.host_in, self.d_w):
+            dw.copy_(hin, non_blocking=True)
+        self.step()
+        for o, ho in zip(self.outs, self.host_out):
+            for t, h in zip(o, ho):
+                h.copy_(t, non_blocking=True)
+
+    def cpu(self):
+        samples = [np.ascontiguousarray(w[::self.sample_stride]) for w in self.tensors]
+        v, dt, n, cores = _time_oracle_rows(samples, self.bits, self.n_cand, self.packed)
+        return v, cores, f"{self.sample_desc} ({n} elements, {dt:.1f} s)", n
+
+
+class Activation(Workload):
+    kernel = "tensor_sweep_kernel<8>"
+    launches_per_step = 9        # init, absmax, sweep, finish, re-score, 3 polish, final
+
+    def __init__(self, name, x, n_cand):
+        self.name, self.x, self.n_cand = name, x, n_cand
+
+    def setup(self, ctx, torch, dev):
+        self.host_in = torch.from_numpy(self.x).pin_memory()
+        self.d_x = self.host_in.to(dev)
+        self.out = (torch.empty(1, device=dev), torch.empty(1, device=dev))
+        self.host_out = tuple(t.cpu().pin_memory() for t in self.out)
+        self.n_total = self.x.size
+        self.h2d, self.d2h = 4 * self.n_total, 8
+
+        def step():
+            ctx.omse_activation_scale(self.d_x, self.n_total, BITS, False, self.n_cand, HI_FRAC, REFINE, *self.out)
+        self.step = step
+
+    def step_e2e(self):
+        self.d_x.copy_(self.host_in, non_blocking=True)
+        self.step()
+        for t, h in zip(self.out, self.host_out):
+            h.copy_(t, non_blocking=True)
+
+    def cpu(self):
+        from oracle import omse_oracle as orc
+        sub = np.ascontiguousarray(self.x[: 1 << 21])       # the per-tensor search on the first 2M elements
+        t0 = time.perf_counter()
+        orc.activation_scale(sub, BITS, False, self.n_cand, HI_FRAC, REFINE)
+        dt = time.perf_counter() - t0
+        return (sub.size / dt, orc.max_threads(),
+                f"first {sub.size} elements of the tensor, all {self.n_cand} candidates ({dt:.1f} s)", sub.size)
+
+
+class Residual(Workload):
+    evals_per_element = 2
+
+    def __init__(self, name, t, n_cand):
+        self.name, self.t, self.n_cand = name, t, n_cand
+
+    def setup(self, ctx, torch, dev):
+        s, k = self.t.shape
+        self.host_in = torch.from_numpy(self.t).pin_memory()
+        self.d_t = self.host_in.to(dev)
+        self.out = (torch.empty(2, s, device=dev), torch.empty(2, s, device=dev),
+                    torch.empty(2, (s * k + 1) // 2, dtype=torch.uint8, device=dev))
+        self.host_out = tuple(t.cpu().pin_memory() for t in self.out)
+        self.n_total = s * k
+        self.h2d, self.d2h = 4 * self.n_total, sum(t.numel() * t.element_size() for t in self.out)
+
+        def step():
+            ctx.omse_residual_quantize(self.d_t, s, k, [BITS, BITS], True, self.n_cand, HI_FRAC, REFINE, 1,
+                                       self.out[0], self.out[1], None, self.out[2])
+        self.step = step
+
+    def step_e2e(self):
+        self.d_t.copy_(self.host_in, non_blocking=True)
+        self.step()
+        for t, h in zip(self.out, self.host_out):
+            h.copy_(t, non_blocking=True)
+
+    def cpu(self):
+        from oracle import omse_oracle as orc
+        sub = np.ascontiguousarray(self.t[::64])
+        t0 = time.perf_counter()
+        orc.residual_rows(sub, (BITS, BITS), True, self.n_cand, HI_FRAC, REFINE, 1)
+        dt = time.perf_counter() - t0
+        return sub.size / dt, orc.max_threads(), f"every 64th kernel ({sub.size} elements, {dt:.1f} s)", sub.size
+
+
+def make_workload(spec: str, rank: int):
+    from paper_1902_06822_b200 import synth
+    if spec == "c2":
+        ws = [w for _, w in synth.resnet50_weights(seed=rank_seed(rank))]
+        return WeightSet(WORKLOAD, ws, BITS, N_CAND, True, 4, "every 4th kernel of each of the 54 tensors")
+    if spec == "c1":
+        return WeightSet("single_conv_layer_64x576_signed4bit_256cand_3refine_int8", [synth.conv_layer(1 + rank)],
+                         BITS, 256, False, 1, "all 64 kernels")
+    if spec == "c3":
+        return Activation("activation_64x256x56x56_unsigned4bit_per_tensor_2048cand_3refine",
+                          synth.activation_tensor(seed=3 + 1000 * rank), 2048)
+    if spec == "c4":
+        return Residual("vgg16_fc6_4096x25088_residual_two_tensors_signed4bit_1024cand_3refine_packed",
+                        synth.fc6_weights(seed=4 + 1000 * rank), N_CAND)
+    if spec.startswith("c5"):          # c5:K:bits
+        _, k, bits = spec.split(":")
+        k, bits = int(k), int(bits)
+        w = synth.sweep_tensor(k, seed=5 + 1000 * rank)
+        stride = max(1, w.shape[0] // max(1, (6_000_000 // k)))
+        return WeightSet(f"sweep_64M_student_t_K{k}_signed{bits}bit_1024cand_3refine", [w], bits, N_CAND, bits <= 4,
+                         stride, f"every {stride}th kernel")
+    raise SystemExit(f"unknown workload {spec}")
+
+
 def run_reference(args, rank):
-    """The oracle, as it stands, on the host cores; each step is the bounded sample."""
+    """The oracle, as it stands, on the host cores; each step is the workload's bounded sample."""
     if rank != 0:
         return
-    from paper_1902_06822_b200 import synth
-    sample = _cpu_sample(synth.resnet50_weights(seed=2))
-    for _ in range(min(args.warmup, 1)):
-        _time_oracle(sample[:4])
+    wl = make_workload(args.workload, 0)
     total_t, n = 0.0, 0
     for _ in range(args.steps):
-        _, dt, n, cores = _time_oracle(sample)
-        total_t += dt
+        t0 = time.perf_counter()
+        _, cores, desc, n = wl.cpu()
+        total_t += time.perf_counter() - t0
     value = n * args.steps / total_t
-    desc = f"every 4th kernel of each of the 54 tensors ({n} elements per step)"
     print(json.dumps({
         "impl": "reference", "metric": "elements quantized/sec (4-bit MMSE search)", "value": value,
         "unit": "elements/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": 1e3 * total_t / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f64", "data": "synthetic", "config": {"workload": WORKLOAD, "sample": desc},
+        "dtype": "f64", "data": "synthetic", "config": {"workload": wl.name, "sample": desc},
         "cpu_baseline": {"value": value, "unit": "elements/s", "cores": cores, "kind": "oracle", "sample": desc},
         "e2e": {"value": value, "unit": "elements/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
@@ -156,7 +309,7 @@ def run_reference(args, rank):
 
 def run_ours(args, rank, world):
     import torch
-    from paper_1902_06822_b200 import binding, build, synth
+    from paper_1902_06822_b200 import binding, build
     build.build()
     local = int(os.environ.get("LOCAL_RANK", 0))
     torch.cuda.set_device(local)
@@ -166,36 +319,12 @@ def run_ours(args, rank, world):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
-    weights = synth.resnet50_weights(seed=rank_seed(rank))
-    n_total = sum(w.size for _, w in weights)
+    wl = make_workload(args.workload, rank)
     ctx = binding.Context(local)
     stream = torch.cuda.current_stream(dev)
-
-    host_in = [torch.from_numpy(w).pin_memory() for _, w in weights]
-    d_w = [h.to(dev) for h in host_in]
-    outs = []
-    for _, w in weights:
-        s, k = w.shape
-        outs.append((torch.empty(s, dtype=torch.float32, device=dev), torch.empty(s, dtype=torch.float32, device=dev),
-                     torch.empty((s * k + 1) // 2, dtype=torch.uint8, device=dev)))
-    host_out = [(a.cpu().pin_memory(), e.cpu().pin_memory(), p.cpu().pin_memory()) for a, e, p in outs]
+    wl.setup(ctx, torch, dev)
+    n_total = wl.n_total
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # > 126 MB L2
-
-    descs = [dict(w=dw, n_kernels=w.shape[0], kernel_len=w.shape[1], alpha=a, sse=e, packed=p)
-             for (name, w), dw, (a, e, p) in zip(weights, d_w, outs)]
-
-    def step():
-        # all 54 tensors in one launch: kernels of every layer are handed out longest first
-        ctx.omse_quantize_weights_batched(descs, BITS, True, N_CAND, HI_FRAC, REFINE)
-
-    def step_e2e():
-        for hin, dw in zip(host_in, d_w):
-            dw.copy_(hin, non_blocking=True)
-        ctx.omse_quantize_weights_batched(descs, BITS, True, N_CAND, HI_FRAC, REFINE)
-        for (a, e, p), (ha, he, hp) in zip(outs, host_out):
-            ha.copy_(a, non_blocking=True)
-            he.copy_(e, non_blocking=True)
-            hp.copy_(p, non_blocking=True)
 
     def barrier():
         torch.cuda.synchronize()
@@ -216,12 +345,12 @@ def run_ours(args, rank, world):
 
     sampler = ClockSampler(local) if rank == 0 else None
     for _ in range(max(args.warmup, 3)):
-        step()
+        wl.step()
     torch.cuda.synchronize()
-    ms = timed(step, args.steps)
+    ms = timed(wl.step, args.steps)
     clocks = sampler.stop() if sampler else None
-    step_e2e()
-    ms_e2e = timed(step_e2e, args.steps)
+    wl.step_e2e()
+    ms_e2e = timed(wl.step_e2e, args.steps)
     status = ctx.omse_last_device_status()
 
     if rank == 0:
@@ -229,29 +358,28 @@ def run_ours(args, rank, world):
         per_step_s = ms * 1e-3 / args.steps
         value = whole_job_value(n_total, world, ms, args.steps)
         peak = N_SM * LANES_PER_SM * sm_max_mhz * 1e6                     # FP32 lane-instructions per second
-        achieved = INSTR_PER_EVAL * N_CAND * n_total / per_step_s          # algorithmic instructions per second
-        h2d = sum(h.numel() * 4 for h in host_in)
-        d2h = sum(a.numel() * 4 + e.numel() * 4 + p.numel() for a, e, p in outs)
+        evals = wl.n_cand * wl.evals_per_element * n_total                 # (element, candidate) evaluations per step
+        achieved = INSTR_PER_EVAL * evals / per_step_s                     # algorithmic instructions per second
         out = {
             "metric": "elements quantized/sec (4-bit MMSE search)", "value": value, "unit": "elements/s",
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "elements_per_gpu": n_total, "n_cand": N_CAND, "bits": BITS,
+            "config": {"workload": wl.name, "elements_per_gpu": n_total, "n_cand": wl.n_cand,
                        "refine_iters": REFINE, "l2": "flushed between timed steps (256 MB write)",
                        "device_status": status},
             "clocks": clocks,
             "e2e": {"value": whole_job_value(n_total, world, ms_e2e, args.steps), "unit": "elements/s",
-                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-            "gpu_launches": args.steps,
+                    "h2d_bytes_per_step": wl.h2d, "d2h_bytes_per_step": wl.d2h},
+            "gpu_launches": wl.launches_per_step * args.steps,
             "roofline": {"bound": "alu", "achieved": achieved / 1e12, "peak": peak / 1e12,
-                         "unit": "T FP32-instr/s", "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES,
-                         "kernel": "rows_kernel<8>", "peak_source": f"148 SMs x 128 lanes x {sm_max_mhz:.0f} MHz ({peak_src} max clock)",
-                         "instr_per_eval": INSTR_PER_EVAL},
+                         "unit": "T FP32-instr/s", "frac": achieved / peak,
+                         "traffic": NCU_TRAFFIC_BYTES if args.workload == "c2" else None,
+                         "kernel": wl.kernel, "peak_source": f"148 SMs x 128 lanes x {sm_max_mhz:.0f} MHz ({peak_src} max clock)",
+                         "instr_per_eval": INSTR_PER_EVAL, "evaluations_per_s": evals / per_step_s},
         }
         if world == 1 and not args.no_cpu_baseline:
-            v, dt, n, cores = _time_oracle(_cpu_sample(weights))
-            out["cpu_baseline"] = {"value": v, "unit": "elements/s", "cores": cores, "kind": "oracle",
-                                   "sample": f"every 4th kernel of each of the 54 tensors ({n} elements, {dt:.1f} s)"}
+            v, cores, desc, _ = wl.cpu()
+            out["cpu_baseline"] = {"value": v, "unit": "elements/s", "cores": cores, "kind": "oracle", "sample": desc}
         print(json.dumps(out))
     if dist is not None:
         dist.destroy_process_group()
@@ -264,6 +392,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="c2",
+                    help="c2 (default: the ResNet-50 weight set the metric is quoted on), c1, c3, c4, c5:K:bits")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))

@@ -92,12 +92,17 @@ __global__ void __launch_bounds__(256) tensor_absmax_kernel(const float* __restr
 }
 
 // Candidate sweep over tiles of the tensor; block b handles tiles b, b+grid, ...
+// Elements with |x| <= 0.4999*step get code 0 from every candidate (x/alpha_c <= x/alpha_0 < 1/2), so
+// their contribution x^2 is the same for all candidates: they are dropped while the tile is staged
+// (deterministic block scan, order preserved) and their sum of squares is added once per block.
+// Exact zeros (40 % of a post-ReLU tensor) are the main beneficiaries.
 template <int CPT>
 __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    float4* tile = reinterpret_cast<float4*>(smem_raw);
-    double* xg = reinterpret_cast<double*>(tile + a.tile4);
-    const int tid = threadIdx.x, nthr = blockDim.x;
+    __shared__ int warp_tot[16];
+    float* tile = reinterpret_cast<float*>(smem_raw);
+    double* xg = reinterpret_cast<double*>(tile + 4 * a.tile4);
+    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
     const int grp = tid / a.tg, t = tid - grp * a.tg;
     const float mpos = __uint_as_float(a.st->mpos_bits), mneg = __uint_as_float(a.st->mneg_bits);
     const float m = fmaxf(mpos, mneg);
@@ -105,6 +110,7 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
     const GridSetup g = grid_setup(mpos, mneg, a.hi_frac, a.n_cand, flo, fhi);
     const float a_last = __fmul_rn((float)a.n_cand, g.step);
     if (!(m > 0.f) || !(a_last >= FLT_MIN)) return;   // degenerate tensor: finish kernel reports it
+    const float drop_below = 0.4999f * g.step;
 
     u64 inv2[CPT], na2[CPT];
     double dacc[CPT];
@@ -125,27 +131,62 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
     const long long n4_total = (a.n + 3) >> 2;
     const long long n_tiles = (n4_total + a.tile4 - 1) / a.tile4;
     const float4* x4 = reinterpret_cast<const float4*>(a.x);
+    const int per_thread4 = a.tile4 / nthr;          // consecutive float4s staged by one thread
+    double dropped = 0.0;
     for (long long tl = blockIdx.x; tl < n_tiles; tl += gridDim.x) {
         const long long base4 = tl * a.tile4;
         const int cnt4 = (int)min((long long)a.tile4, n4_total - base4);
-        __syncthreads();
-        for (int i = tid; i < cnt4; i += nthr) {
-            const long long e = (base4 + i) << 2;
-            float4 v;
-            if (e + 3 < a.n) {
-                v = __ldg(x4 + base4 + i);
-            } else {   // ragged end of the tensor: missing elements count as zeros (zero error)
-                v.x = e < a.n ? a.x[e] : 0.f;
-                v.y = e + 1 < a.n ? a.x[e + 1] : 0.f;
-                v.z = e + 2 < a.n ? a.x[e + 2] : 0.f;
-                v.w = 0.f;
+        // ---- load this thread's span, count what it keeps
+        float keep[16];
+        int n_keep = 0;
+        for (int j = 0; j < per_thread4; ++j) {
+            const int i = tid * per_thread4 + j;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (i < cnt4) {
+                const long long e = (base4 + i) << 2;
+                if (e + 3 < a.n) {
+                    v = __ldg(x4 + base4 + i);
+                } else {   // ragged end of the tensor: missing elements count as zeros
+                    v.x = e < a.n ? a.x[e] : 0.f;
+                    v.y = e + 1 < a.n ? a.x[e + 1] : 0.f;
+                    v.z = e + 2 < a.n ? a.x[e + 2] : 0.f;
+                }
             }
-            tile[i] = v;
+            const float e4[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if (fabsf(e4[q]) > drop_below) {
+                    keep[n_keep++] = e4[q];
+                } else {
+                    dropped += (double)e4[q] * (double)e4[q];
+                }
+            }
         }
+        // ---- exclusive scan of the counts over the block (lanes by shuffle, warps in order)
+        int incl = n_keep;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int up = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += up;
+        }
+        __syncthreads();   // previous tile fully swept; warp_tot free
+        if (lane == 31) warp_tot[warp] = incl;
         __syncthreads();
-        const int beg4 = (int)(((long long)cnt4 * grp) / a.groups);
-        const int end4 = (int)(((long long)cnt4 * (grp + 1)) / a.groups);
-        sweep_dispatch<CPT>(ncl, tile, beg4, end4, inv2, na2, dacc, kMagic + flo, kMagic + fhi);
+        int offset = incl - n_keep, total = 0;
+        for (int w = 0; w < nwarp; ++w) {
+            const int wt = warp_tot[w];
+            if (w < warp) offset += wt;
+            total += wt;
+        }
+        for (int j = 0; j < n_keep; ++j) tile[offset + j] = keep[j];
+        const int padded = (total + 3) & ~3;
+        if (tid < padded - total) tile[total + tid] = 0.f;
+        __syncthreads();
+        const int kept4 = padded >> 2;
+        const int beg4 = (int)(((long long)kept4 * grp) / a.groups);
+        const int end4 = (int)(((long long)kept4 * (grp + 1)) / a.groups);
+        sweep_dispatch<CPT>(ncl, reinterpret_cast<const float4*>(tile), beg4, end4, inv2, na2, dacc, kMagic + flo,
+                            kMagic + fhi);
     }
     if (a.groups > 1) {
         __syncthreads();
@@ -160,11 +201,15 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
                 for (int sl = 0; sl < CPT; ++sl) dacc[sl] += xg[((gg - 1) * CPT + sl) * a.tg + t];
         }
     }
+    // ---- sum of squares of the dropped elements of this block (fixed order), added to every candidate
+    __shared__ double dscratch[64];
+    long long zero = 0;
+    block_sum2(dropped, zero, dscratch);
     if (grp == 0) {
 #pragma unroll
         for (int sl = 0; sl < CPT; ++sl) {
             const int c = sl * a.tg + t;
-            if (c < a.n_cand) a.partials[(long long)blockIdx.x * a.n_cand + c] = dacc[sl];
+            if (c < a.n_cand) a.partials[(long long)blockIdx.x * a.n_cand + c] = dacc[sl] + dropped;
         }
     }
 }

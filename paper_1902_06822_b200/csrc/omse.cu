@@ -53,7 +53,13 @@ struct omse_ctx {
 
 namespace {
 
-int cpt_for(int n_cand) { return n_cand <= 32 ? 1 : n_cand <= 64 ? 2 : n_cand <= 128 ? 4 : 8; }
+#ifndef OMSE_MAX_CPT
+#define OMSE_MAX_CPT 8
+#endif
+int cpt_for(int n_cand) {
+    const int c = n_cand <= 32 ? 1 : n_cand <= 64 ? 2 : n_cand <= 128 ? 4 : 8;
+    return c > OMSE_MAX_CPT ? OMSE_MAX_CPT : c;
+}
 
 bool grid_ok(const omse_grid* g) {
     return g && g->n_cand >= 1 && g->n_cand <= OMSE_MAX_CANDIDATES && g->hi_frac > 0.f &&
@@ -305,7 +311,7 @@ int omse_quantize_weights_batched(omse_ctx* ctx, const omse_weight_tensor* tenso
                 t.small = 1;
                 t.rows_per_unit = t.K <= 128 ? 8 : 4;
                 const size_t kpad = (size_t)((t.K + 3) & ~3ll);
-                const size_t need = (size_t)t.rows_per_unit * (kpad * 4 + (size_t)ncs * 4 + 8);
+                const size_t need = (size_t)t.rows_per_unit * (kpad * 4 + (size_t)ncs * 4 + 16);
                 if (need > smem_small) smem_small = need;
             }
         }

@@ -20,32 +20,100 @@ __device__ __forceinline__ int warp_allsum(int v) {
     return v;
 }
 
+// Per-row quantities every thread needs, computed once by the warp that takes the row's maxima.
+struct SmallRowParams {
+    float step;     // candidate step
+    float rstep;    // ~1/step
+    int c_sat;      // candidates below this index may saturate
+    int flags;      // bit 0: step so small that reciprocals need a division; bit 1: no usable scale
+};
+
+// Candidate sweep of a row of at most 4*kFlushEvery4 elements: one fp32 block, no fp64 fold.
+template <int CPT, int NCL>
+__device__ __forceinline__ void sweep_short(const float4* __restrict__ xs4, int n4, const u64 (&inv2)[CPT],
+                                            const u64 (&na2)[CPT], float (&out)[CPT], float clo, float chi) {
+    const u64 M2 = pack2(kMagic, kMagic);
+    const u64 NM2 = pack2(-kMagic, -kMagic);
+    u64 acc2[CPT];
+#pragma unroll
+    for (int s = 0; s < CPT; ++s) acc2[s] = 0ull;
+#pragma unroll 1
+    for (int i = 0; i < n4; ++i) {
+        const float4 v = xs4[i];
+        const u64 xa = pack2(v.x, v.y), xb = pack2(v.z, v.w);
+#pragma unroll
+        for (int s = 0; s < CPT; ++s) {
+            u64 ta = fma2(xa, inv2[s], M2);
+            u64 tb = fma2(xb, inv2[s], M2);
+            if (s < NCL) {
+                float a0, a1, b0, b1;
+                unpack2(ta, a0, a1);
+                unpack2(tb, b0, b1);
+                a0 = fminf(fmaxf(a0, clo), chi);
+                a1 = fminf(fmaxf(a1, clo), chi);
+                b0 = fminf(fmaxf(b0, clo), chi);
+                b1 = fminf(fmaxf(b1, clo), chi);
+                ta = pack2(a0, a1);
+                tb = pack2(b0, b1);
+            }
+            const u64 qa = add2(ta, NM2);
+            const u64 qb = add2(tb, NM2);
+            const u64 ea = fma2(na2[s], qa, xa);
+            const u64 eb = fma2(na2[s], qb, xb);
+            acc2[s] = fma2(ea, ea, acc2[s]);
+            acc2[s] = fma2(eb, eb, acc2[s]);
+        }
+    }
+#pragma unroll
+    for (int s = 0; s < CPT; ++s) {
+        float p0, p1;
+        unpack2(acc2[s], p0, p1);
+        out[s] = p0 + p1;
+    }
+}
+
+template <int CPT>
+__device__ __forceinline__ void sweep_short_dispatch(int ncl, const float4* xs4, int n4, const u64 (&inv2)[CPT],
+                                                     const u64 (&na2)[CPT], float (&out)[CPT], float clo, float chi) {
+    if (ncl <= 0) {
+        sweep_short<CPT, 0>(xs4, n4, inv2, na2, out, clo, chi);
+    } else if (ncl == 1) {
+        sweep_short<CPT, 1>(xs4, n4, inv2, na2, out, clo, chi);
+    } else if (ncl == 2 && CPT > 2) {
+        sweep_short<CPT, (CPT > 2 ? 2 : CPT)>(xs4, n4, inv2, na2, out, clo, chi);
+    } else if (ncl <= CPT / 2 && CPT > 4) {
+        sweep_short<CPT, CPT / 2>(xs4, n4, inv2, na2, out, clo, chi);
+    } else {
+        sweep_short<CPT, CPT>(xs4, n4, inv2, na2, out, clo, chi);
+    }
+}
+
 // One row, one warp: argmin of the stored curve, re-score, polish, final codes, outputs.
 // xr: the row in shared memory (k elements), cv: its error curve (n_cand floats).
 // prev_x_last / prev_alpha: last element and final scale of the previous row when this row starts
 // at an odd flat index (its first nibble shares a byte with that element); more: the next row will
 // complete this row's last byte.
 __device__ __forceinline__ float small_row_epilogue(const RowArgs& a, const RowTensor& T, const float* xr,
-                                                    const float* cv, int k, float mpos, float mneg, long long row,
+                                                    const float* cv, int k, const SmallRowParams& rp, long long row,
                                                     float prev_x_last, float prev_alpha, bool more,
                                                     unsigned int& st) {
     const int lane = threadIdx.x & 31;
     const float flo = (float)a.lo[0], fhi = (float)a.hi[0];
-    const GridSetup g = grid_setup(mpos, mneg, a.hi_frac, a.n_cand, flo, fhi);
-    const float m = fmaxf(mpos, mneg);
-    const float a_last = __fmul_rn((float)a.n_cand, g.step);
+    struct { float step; } g = {rp.step};
     float alpha = 0.f;
     int best = -1;
-    bool degenerate = !(m > 0.f) || !(a_last >= FLT_MIN);
+    bool degenerate = (rp.flags & 2) != 0;
+    const int n4 = (a.n_cand + 3) >> 2;          // the curve is padded with +Inf up to a multiple of 4
     if (!degenerate) {
         float bv = INFINITY;
         int bi = 0x7fffffff;
-        for (int c = lane; c < a.n_cand; c += 32) {
-            const float v = cv[c];
-            if (v < bv) {
-                bv = v;
-                bi = c;
-            }
+        const float4* cv4 = reinterpret_cast<const float4*>(cv);
+        for (int j = lane; j < n4; j += 32) {    // ascending candidate index within a lane: strict < keeps the lowest
+            const float4 v = cv4[j];
+            if (v.x < bv) { bv = v.x; bi = 4 * j; }
+            if (v.y < bv) { bv = v.y; bi = 4 * j + 1; }
+            if (v.z < bv) { bv = v.z; bi = 4 * j + 2; }
+            if (v.w < bv) { bv = v.w; bi = 4 * j + 3; }
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
@@ -62,7 +130,10 @@ __device__ __forceinline__ float small_row_epilogue(const RowArgs& a, const RowT
             best = bi;
             const float band = (float)((double)bv * (1.0 + kRescoreBand));
             int cnt = 0;
-            for (int c = lane; c < a.n_cand; c += 32) cnt += (cv[c] <= band) ? 1 : 0;
+            for (int j = lane; j < n4; j += 32) {
+                const float4 v = cv4[j];
+                cnt += (v.x <= band) + (v.y <= band) + (v.z <= band) + (v.w <= band);
+            }
             cnt = warp_allsum(cnt);
             if (cnt > 1 && cnt <= kListCap) {
                 double best_sse = INFINITY;
@@ -189,7 +260,7 @@ __device__ void small_unit(const RowArgs& a, const RowTensor& T, long long unit_
     const int ncs = CPT * a.tg;
     float* xs = reinterpret_cast<float*>(smem_raw);
     float* curve = xs + B * kpad;
-    float* rmax = curve + B * ncs;
+    SmallRowParams* rowp = reinterpret_cast<SmallRowParams*>(curve + B * ncs);
     const float flo = (float)a.lo[0], fhi = (float)a.hi[0];
 
     // ---- stage the rows (contiguous in HBM) into rows of kpad floats, zero padded
@@ -219,7 +290,7 @@ __device__ void small_unit(const RowArgs& a, const RowTensor& T, long long unit_
     if (bad) st |= 1u;
     __syncthreads();
 
-    // ---- max of the positive and negative part of every row: a warp per row
+    // ---- max of the positive and negative part of every row, and the row's grid: a warp per row
     for (int r = warp; r < nrows; r += nwarp) {
         float mp = 0.f, mn = 0.f;
         for (int i = lane; i < k; i += 32) {
@@ -235,38 +306,59 @@ __device__ void small_unit(const RowArgs& a, const RowTensor& T, long long unit_
             mn = fmaxf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
         }
         if (lane == 0) {
-            rmax[2 * r] = mp;
-            rmax[2 * r + 1] = mn;
+            const GridSetup g = grid_setup(mp, mn, a.hi_frac, a.n_cand, flo, fhi);
+            const float a_last = __fmul_rn((float)a.n_cand, g.step);
+            SmallRowParams rp;
+            rp.step = g.step;
+            rp.rstep = g.rstep;
+            rp.c_sat = g.c_sat;
+            rp.flags = (g.tiny ? 1 : 0) | ((!(fmaxf(mp, mn) > 0.f) || !(a_last >= FLT_MIN)) ? 2 : 0);
+            rowp[r] = rp;
         }
     }
     __syncthreads();
 
     // ---- candidate sweep, row after row, by the whole block; error curves to shared memory
+    const bool short_rows = k4 <= kFlushEvery4;       // one fp32 block per candidate: no fp64 fold needed
+    bool in_range[CPT];
+#pragma unroll
+    for (int sl = 0; sl < CPT; ++sl) in_range[sl] = sl * a.tg + tid < a.n_cand;
     for (int r = 0; r < nrows; ++r) {
-        const float mpos = rmax[2 * r], mneg = rmax[2 * r + 1];
-        const GridSetup g = grid_setup(mpos, mneg, a.hi_frac, a.n_cand, flo, fhi);
-        const float a_last = __fmul_rn((float)a.n_cand, g.step);
-        if (!(fmaxf(mpos, mneg) > 0.f) || !(a_last >= FLT_MIN)) continue;   // the epilogue reports it
+        const SmallRowParams rp = rowp[r];
+        if (rp.flags & 2) continue;   // no usable scale: the epilogue reports it
         u64 inv2[CPT], na2[CPT];
-        double dacc[CPT];
         bool ok[CPT];
 #pragma unroll
         for (int sl = 0; sl < CPT; ++sl) {
-            const int c = sl * a.tg + tid;
-            const float ac = __fmul_rn((float)(c + 1), g.step);
-            float inv = g.tiny ? __fdiv_rn(1.0f, ac) : rcp[sl] * g.rstep;
-            ok[sl] = (ac >= FLT_MIN) && c < a.n_cand;
+            const float cf = (float)(sl * a.tg + tid + 1);
+            const float ac = __fmul_rn(cf, rp.step);
+            float inv = rcp[sl] * rp.rstep;
+            ok[sl] = in_range[sl];
+            if (rp.flags & 1) {       // denormal-range row: exact reciprocal, per-candidate validity
+                inv = __fdiv_rn(1.0f, ac);
+                ok[sl] = ok[sl] && (ac >= FLT_MIN);
+            }
             if (!ok[sl]) inv = 0.f;
             inv2[sl] = pack2(inv, inv);
             na2[sl] = pack2(-ac, -ac);
-            dacc[sl] = 0.0;
         }
-        int ncl = (g.c_sat - (tid & ~31) + a.tg - 1) / a.tg;
+        int ncl = (rp.c_sat - (tid & ~31) + a.tg - 1) / a.tg;
         ncl = max(0, min(CPT, ncl));
-        sweep_dispatch<CPT>(ncl, reinterpret_cast<const float4*>(xs) + r * k4, 0, k4, inv2, na2, dacc,
-                            kMagic + flo, kMagic + fhi);
+        const float4* xr4 = reinterpret_cast<const float4*>(xs) + r * k4;
+        float* cvr = curve + r * ncs;
+        if (short_rows) {
+            float out[CPT];
+            sweep_short_dispatch<CPT>(ncl, xr4, k4, inv2, na2, out, kMagic + flo, kMagic + fhi);
 #pragma unroll
-        for (int sl = 0; sl < CPT; ++sl) curve[r * ncs + sl * a.tg + tid] = ok[sl] ? (float)dacc[sl] : INFINITY;
+            for (int sl = 0; sl < CPT; ++sl) cvr[sl * a.tg + tid] = ok[sl] ? out[sl] : INFINITY;
+        } else {
+            double dacc[CPT];
+#pragma unroll
+            for (int sl = 0; sl < CPT; ++sl) dacc[sl] = 0.0;
+            sweep_dispatch<CPT>(ncl, xr4, 0, k4, inv2, na2, dacc, kMagic + flo, kMagic + fhi);
+#pragma unroll
+            for (int sl = 0; sl < CPT; ++sl) cvr[sl * a.tg + tid] = ok[sl] ? (float)dacc[sl] : INFINITY;
+        }
     }
     __syncthreads();
 
@@ -280,8 +372,8 @@ __device__ void small_unit(const RowArgs& a, const RowTensor& T, long long unit_
             if (r >= nrows) break;
             const bool more = (rr + 1 < rpt) && (r + 1 < nrows);
             const float prev_x_last = r > 0 ? xs[(r - 1) * kpad + k - 1] : 0.f;
-            prev_alpha = small_row_epilogue(a, T, xs + r * kpad, curve + r * ncs, k, rmax[2 * r], rmax[2 * r + 1],
-                                            row0 + r, prev_x_last, prev_alpha, more, st);
+            prev_alpha = small_row_epilogue(a, T, xs + r * kpad, curve + r * ncs, k, rowp[r], row0 + r, prev_x_last,
+                                            prev_alpha, more, st);
         }
     }
 }

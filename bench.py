@@ -34,6 +34,7 @@ INSTR_PER_EVAL = 6            # reference FP32 sequence per (element, candidate)
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the timed kernel, from the ncu capture summarised
 # in profiles/rows_kernel_resnet50_weight_set.md; set to None whenever the kernel changes after the capture
 NCU_TRAFFIC_BYTES = None
+E2E_CHUNKS = 6                # batched launches per end-to-end step (copies of later chunks overlap earlier searches)
 N_SM, LANES_PER_SM = 148, 128
 WORKLOAD = "resnet50_weight_set_54_tensors_25.5M_params_signed4bit_kernelwise_1024cand_3refine_packed"
 
@@ -177,13 +178,47 @@ class WeightSet(Workload):
             ctx.omse_quantize_weights_batched(descs, self.bits, True, self.n_cand, HI_FRAC, REFINE)
         self.step = step
 
+        # End-to-end: the host->device copies of later tensors run under the search of earlier ones.
+        # Tensors go longest rows first in E2E_CHUNKS chunks of equal bytes; each chunk is one batched launch.
+        order = sorted(range(len(descs)), key=lambda i: -self.tensors[i].shape[1])
+        n_chunks = min(E2E_CHUNKS, len(descs))
+        target, acc, self.chunks, cur = self.n_total / n_chunks, 0, [], []
+        for i in order:
+            cur.append(i)
+            acc += self.tensors[i].size
+            if acc >= target * (len(self.chunks) + 1) and len(self.chunks) < n_chunks - 1:
+                self.chunks.append(cur)
+                cur = []
+        if cur:
+            self.chunks.append(cur)
+        self.h2d_stream, self.d2h_stream = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+        self._torch, self._ctx, self._descs = torch, ctx, descs
+
     def step_e2e(self):
-        for hin, dw in zip(self.host_in, self.d_w):
-            dw.copy_(hin, non_blocking=True)
-        self.step()
-        for o, ho in zip(self.outs, self.host_out):
-            for t, h in zip(o, ho):
-                h.copy_(t, non_blocking=True)
+        torch, ctx = self._torch, self._ctx
+        main = torch.cuda.current_stream()
+        self.h2d_stream.wait_stream(main)          # inputs of the previous step are no longer in use
+        self.d2h_stream.wait_stream(main)
+        ready = []
+        with torch.cuda.stream(self.h2d_stream):
+            for ch in self.chunks:
+                for i in ch:
+                    self.d_w[i].copy_(self.host_in[i], non_blocking=True)
+                ev = torch.cuda.Event()
+                ev.record(self.h2d_stream)
+                ready.append(ev)
+        for ch, ev in zip(self.chunks, ready):
+            main.wait_event(ev)
+            ctx.omse_quantize_weights_batched([self._descs[i] for i in ch], self.bits, True, self.n_cand, HI_FRAC,
+                                              REFINE)
+            done = torch.cuda.Event()
+            done.record(main)
+            with torch.cuda.stream(self.d2h_stream):
+                self.d2h_stream.wait_event(done)
+                for i in ch:
+                    for t, h in zip(self.outs[i], self.host_out[i]):
+                        h.copy_(t, non_blocking=True)
+        main.wait_stream(self.d2h_stream)          # the step ends when its results are on the host
 
     def cpu(self):
         samples = [np.ascontiguousarray(w[::self.sample_stride]) for w in self.tensors]

@@ -20,6 +20,9 @@
 #define OMSE_ROWS_THREADS_MID 128
 #endif
 
+#ifndef OMSE_PRUNE
+#define OMSE_PRUNE 1
+#endif
 #ifndef OMSE_SMALL_K
 #define OMSE_SMALL_K 640            /* rows up to this length are batched per work unit */
 #endif
@@ -85,9 +88,19 @@ int launch_rows_t(omse_ctx* ctx, omse::RowArgs& a, size_t smem) {
         attr_set[ctx->device & 63] = true;
     }
     const int threads = a.groups * a.tg;
+    // blocks per SM for this launch shape (remembered: the query costs more than a small launch)
+    struct Shape { int device, threads; size_t smem; int occ; };
+    static Shape seen[16];
+    static int n_seen = 0;
     int occ = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, omse::rows_kernel<CPT>, threads, smem) != cudaSuccess || occ < 1)
-        return OMSE_ECUDA;
+    for (int i = 0; i < n_seen; ++i)
+        if (seen[i].device == ctx->device && seen[i].threads == threads && seen[i].smem == smem) occ = seen[i].occ;
+    if (occ == 0) {
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, omse::rows_kernel<CPT>, threads, smem) != cudaSuccess || occ < 1)
+            return OMSE_ECUDA;
+        seen[n_seen % 16] = Shape{ctx->device, threads, smem, occ};
+        if (n_seen < 16) ++n_seen;
+    }
     long long grid = (long long)ctx->n_sm * occ;
     if (grid > a.n_units) grid = a.n_units;
     omse::rows_kernel<CPT><<<(unsigned)grid, threads, smem, ctx->stream>>>(a);
@@ -105,9 +118,16 @@ int launch_rows(omse_ctx* ctx, omse::RowArgs& a, long long max_k, size_t smem_sm
     if (groups > k4 / 8) groups = k4 / 8;
     if (groups < 1) groups = 1;
     a.groups = groups;
+    // fixed part: reduction scratch, skipped sums, near-minimal list, class table, misc
+    const size_t fixed = (size_t)omse::kScratchDoubles * 8 + (size_t)cpt * 8 + omse::kListCap * 4 + 2 * (cpt + 1) * 4 + 8 * 4;
     auto smem_for = [&](int gr) {
-        return (size_t)(a.keep_x0 ? 2 : 1) * k4 * 16 + (size_t)(gr - 1) * cpt * a.tg * 8 + 64 * 8 + omse::kListCap * 4 + 8 * 4;
+        return (size_t)(a.keep_x0 ? 2 : 1) * k4 * 16 + (a.prune ? (size_t)k4 * 16 + (size_t)cpt * 16 : 0) +
+               (size_t)(gr - 1) * cpt * a.tg * 8 + fixed;
     };
+    // Regrouping by magnitude needs a second copy of the row on chip and 16-bit class counts; it is worth its
+    // fixed cost only for long rows or for launches with several rows per SM.
+    a.prune = (OMSE_PRUNE && max_k < 65536 && (max_k >= 1024 || a.n_units >= 4ll * ctx->n_sm)) ? 1 : 0;
+    if (a.prune && smem_for(1) > (size_t)kMaxSmem) a.prune = 0;
     while (a.groups > 1 && smem_for(a.groups) > (size_t)kMaxSmem) a.groups >>= 1;
     size_t smem = smem_for(a.groups);
     if (smem > (size_t)kMaxSmem) return OMSE_EINVAL;

@@ -58,20 +58,21 @@ __device__ __forceinline__ int code_of(float x, float alpha, float flo, float fh
 
 // ---------------------------------------------------------------------------------------------
 // Candidate sweep over float4 indices [beg4, end4) of a shared-memory span.  CPT candidates per
-// thread; the first NCL of them are evaluated with saturation, the rest without.
+// thread, of which only the first NACT are evaluated on this span (the others are known to code
+// every element of the span as zero); the first NCL of them are evaluated with saturation.
 // acc2 holds two fp32 partial sums per candidate (even / odd element of each pair); every
 // kFlushEvery4 loads they are folded into the fp64 accumulators so that the rounding noise of the
 // fp32 sums stays near 1e-7 relative whatever the span length.
 // ---------------------------------------------------------------------------------------------
-template <int CPT, int NCL>
+template <int CPT, int NACT, int NCL>
 __device__ __forceinline__ void sweep_range(const float4* __restrict__ xs4, int beg4, int end4,
                                             const u64 (&inv2)[CPT], const u64 (&na2)[CPT],
                                             double (&dacc)[CPT], float clo, float chi) {
     const u64 M2 = pack2(kMagic, kMagic);
     const u64 NM2 = pack2(-kMagic, -kMagic);
-    u64 acc2[CPT];
+    u64 acc2[NACT];
 #pragma unroll
-    for (int s = 0; s < CPT; ++s) acc2[s] = 0ull;
+    for (int s = 0; s < NACT; ++s) acc2[s] = 0ull;
     int i = beg4;
     while (i < end4) {
         const int stop = min(end4, i + kFlushEvery4);
@@ -80,7 +81,7 @@ __device__ __forceinline__ void sweep_range(const float4* __restrict__ xs4, int 
             const float4 v = xs4[i];
             const u64 xa = pack2(v.x, v.y), xb = pack2(v.z, v.w);
 #pragma unroll
-            for (int s = 0; s < CPT; ++s) {
+            for (int s = 0; s < NACT; ++s) {
                 u64 ta = fma2(xa, inv2[s], M2);
                 u64 tb = fma2(xb, inv2[s], M2);
                 if (s < NCL) {
@@ -103,7 +104,7 @@ __device__ __forceinline__ void sweep_range(const float4* __restrict__ xs4, int 
             }
         }
 #pragma unroll
-        for (int s = 0; s < CPT; ++s) {
+        for (int s = 0; s < NACT; ++s) {
             float p0, p1;
             unpack2(acc2[s], p0, p1);
             dacc[s] += (double)(p0 + p1);
@@ -112,22 +113,47 @@ __device__ __forceinline__ void sweep_range(const float4* __restrict__ xs4, int 
     }
 }
 
-// Dispatch on the (warp-uniform) number of leading candidates per thread that need saturation.
+// Dispatch on the (warp-uniform) number of leading candidates per thread that need saturation ...
+template <int CPT, int NACT>
+__device__ __forceinline__ void sweep_ncl(int ncl, const float4* xs4, int beg4, int end4, const u64 (&inv2)[CPT],
+                                          const u64 (&na2)[CPT], double (&dacc)[CPT], float clo, float chi) {
+    if (ncl <= 0) {
+        sweep_range<CPT, NACT, 0>(xs4, beg4, end4, inv2, na2, dacc, clo, chi);
+    } else if (ncl == 1) {
+        sweep_range<CPT, NACT, 1>(xs4, beg4, end4, inv2, na2, dacc, clo, chi);
+    } else if (ncl == 2 && NACT > 2) {
+        sweep_range<CPT, NACT, (NACT > 2 ? 2 : NACT)>(xs4, beg4, end4, inv2, na2, dacc, clo, chi);
+    } else if (ncl <= 4 && NACT > 4) {
+        sweep_range<CPT, NACT, (NACT > 4 ? 4 : NACT)>(xs4, beg4, end4, inv2, na2, dacc, clo, chi);
+    } else {
+        sweep_range<CPT, NACT, NACT>(xs4, beg4, end4, inv2, na2, dacc, clo, chi);
+    }
+}
+
+// ... and on the number of candidates per thread that are evaluated at all on this span.
+template <int CPT>
+__device__ __forceinline__ void sweep_dispatch(int nact, int ncl, const float4* xs4, int beg4, int end4,
+                                               const u64 (&inv2)[CPT], const u64 (&na2)[CPT],
+                                               double (&dacc)[CPT], float clo, float chi) {
+    if (beg4 >= end4 || nact <= 0) return;
+    if (ncl > nact) ncl = nact;
+    switch (nact) {
+        case 1: sweep_ncl<CPT, 1>(ncl, xs4, beg4, end4, inv2, na2, dacc, clo, chi); break;
+        case 2: if constexpr (CPT >= 2) sweep_ncl<CPT, 2>(ncl, xs4, beg4, end4, inv2, na2, dacc, clo, chi); break;
+        case 3: if constexpr (CPT >= 4) sweep_ncl<CPT, 3>(ncl, xs4, beg4, end4, inv2, na2, dacc, clo, chi); break;
+        case 4: if constexpr (CPT >= 4) sweep_ncl<CPT, 4>(ncl, xs4, beg4, end4, inv2, na2, dacc, clo, chi); break;
+        case 5: if constexpr (CPT >= 8) sweep_ncl<CPT, 5>(ncl, xs4, beg4, end4, inv2, na2, dacc, clo, chi); break;
+        case 6: if constexpr (CPT >= 8) sweep_ncl<CPT, 6>(ncl, xs4, beg4, end4, inv2, na2, dacc, clo, chi); break;
+        case 7: if constexpr (CPT >= 8) sweep_ncl<CPT, 7>(ncl, xs4, beg4, end4, inv2, na2, dacc, clo, chi); break;
+        default: sweep_ncl<CPT, CPT>(ncl, xs4, beg4, end4, inv2, na2, dacc, clo, chi); break;
+    }
+}
+
 template <int CPT>
 __device__ __forceinline__ void sweep_dispatch(int ncl, const float4* xs4, int beg4, int end4,
                                                const u64 (&inv2)[CPT], const u64 (&na2)[CPT],
                                                double (&dacc)[CPT], float clo, float chi) {
-    if (ncl <= 0) {
-        sweep_range<CPT, 0>(xs4, beg4, end4, inv2, na2, dacc, clo, chi);
-    } else if (ncl == 1) {
-        sweep_range<CPT, 1>(xs4, beg4, end4, inv2, na2, dacc, clo, chi);
-    } else if (ncl == 2 && CPT > 2) {
-        sweep_range<CPT, (CPT > 2 ? 2 : CPT)>(xs4, beg4, end4, inv2, na2, dacc, clo, chi);
-    } else if (ncl <= CPT / 2 && CPT > 4) {
-        sweep_range<CPT, CPT / 2>(xs4, beg4, end4, inv2, na2, dacc, clo, chi);
-    } else {
-        sweep_range<CPT, CPT>(xs4, beg4, end4, inv2, na2, dacc, clo, chi);
-    }
+    sweep_dispatch<CPT>(CPT, ncl, xs4, beg4, end4, inv2, na2, dacc, clo, chi);
 }
 
 // ---------------------------------------------------------------------------------------------

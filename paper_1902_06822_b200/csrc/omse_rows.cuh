@@ -41,6 +41,7 @@ struct RowArgs {
     int tg;                     // threads per group (multiple of 32); candidate c = slot*tg + t
     int keep_x0;                // n_sweeps > 1: keep the original row next to the residual
     int max_k4;                 // float4s of the longest row in the launch (shared-memory carve-up)
+    int prune;                  // 1: rows are regrouped by magnitude so that candidates skip elements they code as 0
 };
 
 }  // namespace omse
@@ -48,6 +49,8 @@ struct RowArgs {
 #include "omse_rows_small.cuh"
 
 namespace omse {
+
+constexpr int kScratchDoubles = 64 + 16 * 9;
 
 struct PhiOut {
     float alpha;
@@ -60,11 +63,134 @@ struct PhiOut {
 struct RowSmem {
     float* xs;        // [k4*4] current tensor (row or residual), zero padded to a multiple of 4
     float* x0;        // [k4*4] original row (only when keep_x0)
+    float* xb;        // [k4*4 + 4*CPT] the row regrouped by magnitude class (only when pruning)
     double* xg;       // [(groups-1)*CPT*tg] partial sums of the other element groups
-    double* scratch;  // [64] reductions
+    double* scratch;  // [kScratchDoubles] reductions
+    double* skip;     // [CPT] squared sum of the elements a candidate slot does not evaluate
+    int* seg;         // [2*(CPT+1)] first element and padded length of each magnitude class in xb
     int* list;        // [kListCap] near-minimal candidates
     int* misc;        // [8]: 0 list count; 1..4 nibble carried to the next row, per tensor
 };
+
+// ---------------------------------------------------------------------------------------------
+// Magnitude classes.  Candidate slot sl of every thread holds scales >= alpha_{sl*tg} = (sl*tg+1)*step.
+// An element with |x| <= 0.4999*alpha gets code 0 from that scale and from every larger one, and
+// then contributes exactly x^2 to their errors.  So the row is regrouped (stable counting sort, fixed
+// order) into classes nb = number of leading slots that still have to evaluate the element; the
+// sweep runs slots 0..nb-1 on class nb, and each slot adds the squared sum of the classes it skipped.
+// With the grid reaching up to max|x| most (element, candidate) pairs fall away: the large scales
+// only see the few large elements.
+// ---------------------------------------------------------------------------------------------
+template <int CPT>
+__device__ __forceinline__ int magnitude_class(float x, float inv_thr, float inv_tg) {
+    const float ax = fabsf(x);
+    if (!(ax <= FLT_MAX)) return CPT;          // non-finite: every slot sees it (and reports it)
+    const float r = ax * inv_thr;              // |x| / (0.4999*step)
+    if (r <= 1.0f) return 0;
+    const float f = (r - 1.0f) * inv_tg;       // slot sl needs x iff r > sl*tg + 1
+    return f >= (float)CPT ? CPT : (int)f + 1;
+}
+
+template <int CPT>
+__device__ void partition_row(const RowSmem& s, int k, const GridSetup& g, int tg) {
+    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
+    const float inv_thr = g.rstep * (1.0f / 0.4999f);
+    const float inv_tg = 1.0f / (float)tg;
+    const int span = (k + nthr - 1) / nthr;
+    const int beg = min(k, tid * span), end = min(k, beg + span);
+    // ---- pass 1: class counts of this thread's span (16-bit fields), squared sums per class
+    u64 c0 = 0ull, c1 = 0ull;                  // classes 1..4 and 5..8
+    double d[CPT + 1];
+#pragma unroll
+    for (int b = 0; b <= CPT; ++b) d[b] = 0.0;
+    for (int i = beg; i < end; ++i) {
+        const float x = s.xs[i];
+        const int nb = magnitude_class<CPT>(x, inv_thr, inv_tg);
+        const double xx = (double)x * (double)x;
+#pragma unroll
+        for (int b = 0; b <= CPT; ++b) d[b] += (nb == b) ? xx : 0.0;
+        if (nb >= 5) c1 += 1ull << (16 * (nb - 5));
+        else if (nb >= 1) c0 += 1ull << (16 * (nb - 1));
+    }
+    // ---- exclusive scan of the counts over the block (lanes by shuffle, warps in order)
+    u64 i0 = c0, i1 = c1;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const u64 u0 = __shfl_up_sync(0xffffffffu, i0, o);
+        const u64 u1 = __shfl_up_sync(0xffffffffu, i1, o);
+        if (lane >= o) {
+            i0 += u0;
+            i1 += u1;
+        }
+    }
+    u64* wt = reinterpret_cast<u64*>(s.scratch);          // [nwarp][2]
+    __syncthreads();
+    if (lane == 31) {
+        wt[2 * warp] = i0;
+        wt[2 * warp + 1] = i1;
+    }
+    __syncthreads();
+    u64 off0 = i0 - c0, off1 = i1 - c1, tot0 = 0ull, tot1 = 0ull;
+    for (int w = 0; w < nwarp; ++w) {
+        const u64 a0 = wt[2 * w], a1 = wt[2 * w + 1];
+        if (w < warp) {
+            off0 += a0;
+            off1 += a1;
+        }
+        tot0 += a0;
+        tot1 += a1;
+    }
+    // ---- class layout in xb: class CPT first, each class padded with zeros to a multiple of 4
+    int base[CPT + 1];
+    int pos = 0;
+#pragma unroll
+    for (int b = CPT; b >= 1; --b) {
+        const int cnt = (int)(((b >= 5 ? tot1 : tot0) >> (16 * ((b - 1) & 3))) & 0xffffull);
+        base[b] = pos;
+        const int padded = (cnt + 3) & ~3;
+        if (tid == 0) {
+            s.seg[2 * b] = pos;
+            s.seg[2 * b + 1] = padded;
+        }
+        if (tid < padded - cnt) s.xb[pos + cnt + tid] = 0.f;
+        pos += padded;
+    }
+    // ---- pass 2: scatter in the original order within each class
+    for (int i = beg; i < end; ++i) {
+        const float x = s.xs[i];
+        const int nb = magnitude_class<CPT>(x, inv_thr, inv_tg);
+        if (nb >= 1) {
+            const int sh = 16 * ((nb - 1) & 3);
+            int within;
+            if (nb >= 5) {
+                within = (int)((off1 >> sh) & 0xffffull);
+                off1 += 1ull << sh;
+            } else {
+                within = (int)((off0 >> sh) & 0xffffull);
+                off0 += 1ull << sh;
+            }
+            int bs = 0;
+#pragma unroll
+            for (int b = 1; b <= CPT; ++b) bs = (nb == b) ? base[b] : bs;
+            s.xb[bs + within] = x;
+        }
+    }
+    // ---- squared sums per class -> what each slot skips: classes 0..sl
+    double* ds = s.scratch + 64;                           // [nwarp][CPT+1]
+#pragma unroll
+    for (int b = 0; b <= CPT; ++b) {
+        const double v = warp_sum(d[b]);
+        if (lane == 0) ds[warp * (CPT + 1) + b] = v;
+    }
+    __syncthreads();
+    if (tid < CPT) {
+        double acc = 0.0;
+        for (int b = 0; b <= tid; ++b)
+            for (int w = 0; w < nwarp; ++w) acc += ds[w * (CPT + 1) + b];
+        s.skip[tid] = acc;
+    }
+    __syncthreads();
+}
 
 // The quantization mapping phi of Section 3.4 on the row held in s.xs (k elements, k4 float4s).
 template <int CPT>
@@ -111,10 +237,25 @@ __device__ PhiOut phi_block(const RowArgs& a, const RowSmem& s, int k, int k4, f
     int ncl = (g.c_sat - warp_t0 + a.tg - 1) / a.tg;
     ncl = max(0, min(CPT, ncl));
 
-    // ---- sweep: this group's contiguous share of the row, all candidates
-    const int beg4 = (int)(((long long)k4 * grp) / a.groups);
-    const int end4 = (int)(((long long)k4 * (grp + 1)) / a.groups);
-    sweep_dispatch<CPT>(ncl, xs4, beg4, end4, inv2, na2, dacc, kMagic + flo, kMagic + fhi);
+    // ---- sweep: this group's contiguous share of the row (of every magnitude class), all candidates
+    if (a.prune && !g.tiny) {
+        partition_row<CPT>(s, k, g, a.tg);
+        const float4* xb4 = reinterpret_cast<const float4*>(s.xb);
+        for (int b = CPT; b >= 1; --b) {
+            const int first4 = s.seg[2 * b] >> 2, len4 = s.seg[2 * b + 1] >> 2;
+            const int beg4 = first4 + (int)(((long long)len4 * grp) / a.groups);
+            const int end4 = first4 + (int)(((long long)len4 * (grp + 1)) / a.groups);
+            sweep_dispatch<CPT>(b, ncl, xb4, beg4, end4, inv2, na2, dacc, kMagic + flo, kMagic + fhi);
+        }
+        if (grp == 0) {
+#pragma unroll
+            for (int sl = 0; sl < CPT; ++sl) dacc[sl] += s.skip[sl];
+        }
+    } else {
+        const int beg4 = (int)(((long long)k4 * grp) / a.groups);
+        const int end4 = (int)(((long long)k4 * (grp + 1)) / a.groups);
+        sweep_dispatch<CPT>(ncl, xs4, beg4, end4, inv2, na2, dacc, kMagic + flo, kMagic + fhi);
+    }
 
     if (a.groups > 1) {
         if (grp > 0) {
@@ -283,10 +424,13 @@ __global__ void __launch_bounds__(OMSE_ROWS_MAX_THREADS) rows_kernel(const RowAr
     RowSmem s;
     s.xs = reinterpret_cast<float*>(smem_raw);
     s.x0 = s.xs + (a.keep_x0 ? 4 * a.max_k4 : 0);
-    s.xg = reinterpret_cast<double*>(s.x0 + 4 * a.max_k4);
+    s.xb = s.x0 + 4 * a.max_k4;
+    s.xg = reinterpret_cast<double*>(s.xb + (a.prune ? 4 * a.max_k4 + 4 * CPT : 0));
     s.scratch = s.xg + (size_t)(a.groups - 1) * CPT * a.tg;
-    s.list = reinterpret_cast<int*>(s.scratch + 64);
-    s.misc = s.list + kListCap;
+    s.skip = s.scratch + kScratchDoubles;
+    s.list = reinterpret_cast<int*>(s.skip + CPT);
+    s.seg = s.list + kListCap;
+    s.misc = s.seg + 2 * (CPT + 1);
     unsigned int st = 0;
 
     // 1/(c+1) for this thread's candidates: 1/alpha_c = (1/(c+1)) * (1/step) to within 2 ulp

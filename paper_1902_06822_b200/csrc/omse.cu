@@ -435,7 +435,7 @@ int omse_activation_scale(omse_ctx* ctx, const float* d_x, int64_t n, int bits, 
     int n_blocks = 1;
     if (n > 0) {
         omse::tensor_absmax_kernel<<<(unsigned)pass_grid, 256, 0, s>>>(d_x, n, a.st, a.status);
-        const size_t smem = (size_t)a.tile4 * 16 + (size_t)(a.groups - 1) * cpt * a.tg * 8;
+        const size_t smem = (size_t)a.tile4 * 16 + (size_t)cpt * 16 + (size_t)(a.groups - 1) * cpt * a.tg * 8;
         int rc;
         switch (cpt) {
             case 1: rc = launch_tensor_sweep_t<1>(ctx, a, smem, &n_blocks); break;
@@ -590,7 +590,7 @@ extern "C" int omse_activation_scale_static(int device, void* cuda_stream, const
     int n_blocks = 1;
     if (n > 0) {
         omse::tensor_absmax_kernel<<<(unsigned)pass_grid, 256, 0, s>>>(d_x, n, a.st, a.status);
-        const size_t smem = (size_t)a.tile4 * 16 + (size_t)(a.groups - 1) * cpt * a.tg * 8;   // < 48 KB: no opt-in needed
+        const size_t smem = (size_t)a.tile4 * 16 + (size_t)cpt * 16 + (size_t)(a.groups - 1) * cpt * a.tg * 8;   // < 48 KB: no opt-in needed
         int rc;
         switch (cpt) {
             case 1: rc = launch_static_sweep_t<1>(sd.n_sm, s, a, smem, &n_blocks); break;

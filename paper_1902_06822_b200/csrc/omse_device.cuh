@@ -249,6 +249,18 @@ __device__ __forceinline__ void block_argmin(double& v, int& idx, double* scratc
     idx = bi;
 }
 
+// Number of leading candidate slots (slot sl holds scales >= (sl*tg+1)*step) that must still evaluate x:
+// the others code it as 0.  inv_thr = 1/(0.4999*step), inv_tg = 1/tg.
+template <int CPT>
+__device__ __forceinline__ int magnitude_class(float x, float inv_thr, float inv_tg) {
+    const float ax = fabsf(x);
+    if (!(ax <= FLT_MAX)) return CPT;          // non-finite: every slot sees it (and reports it)
+    const float r = ax * inv_thr;              // |x| / (0.4999*step)
+    if (r <= 1.0f) return 0;
+    const float f = (r - 1.0f) * inv_tg;       // slot sl needs x iff r > sl*tg + 1
+    return f >= (float)CPT ? CPT : (int)f + 1;
+}
+
 // Per-candidate constants of one thread for the grid of Section 3.4 on a tensor with max|x| = m.
 // Candidate c has alpha_c = fl(fl(c+1)*step), step = fl(fl(hi_frac*m)/fl(C)), all binary32.
 // In the sweep x/alpha_c is replaced by x*inv_c with inv_c within 2 ulp of 1/alpha_c: a code can

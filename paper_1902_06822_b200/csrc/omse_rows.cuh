@@ -82,16 +82,6 @@ struct RowSmem {
 // only see the few large elements.
 // ---------------------------------------------------------------------------------------------
 template <int CPT>
-__device__ __forceinline__ int magnitude_class(float x, float inv_thr, float inv_tg) {
-    const float ax = fabsf(x);
-    if (!(ax <= FLT_MAX)) return CPT;          // non-finite: every slot sees it (and reports it)
-    const float r = ax * inv_thr;              // |x| / (0.4999*step)
-    if (r <= 1.0f) return 0;
-    const float f = (r - 1.0f) * inv_tg;       // slot sl needs x iff r > sl*tg + 1
-    return f >= (float)CPT ? CPT : (int)f + 1;
-}
-
-template <int CPT>
 __device__ void partition_row(const RowSmem& s, int k, const GridSetup& g, int tg) {
     const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
     const float inv_thr = g.rstep * (1.0f / 0.4999f);

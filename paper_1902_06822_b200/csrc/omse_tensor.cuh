@@ -92,16 +92,17 @@ __global__ void __launch_bounds__(256) tensor_absmax_kernel(const float* __restr
 }
 
 // Candidate sweep over tiles of the tensor; block b handles tiles b, b+grid, ...
-// Elements with |x| <= 0.4999*step get code 0 from every candidate (x/alpha_c <= x/alpha_0 < 1/2), so
-// their contribution x^2 is the same for all candidates: they are dropped while the tile is staged
-// (deterministic block scan, order preserved) and their sum of squares is added once per block.
-// Exact zeros (40 % of a post-ReLU tensor) are the main beneficiaries.
+// While a tile is staged its elements are regrouped by magnitude class (see magnitude_class): class nb
+// is evaluated by candidate slots 0..nb-1 only, class 0 (|x| <= 0.4999*step, in particular the exact
+// zeros of a post-ReLU tensor) by none; every slot adds the squared sum of the classes it skipped.
+// The regrouping is a deterministic block-wide counting sort, so results do not depend on scheduling.
 template <int CPT>
 __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    __shared__ int warp_tot[16];
-    float* tile = reinterpret_cast<float*>(smem_raw);
-    double* xg = reinterpret_cast<double*>(tile + 4 * a.tile4);
+    __shared__ u64 warp_tot[16][2];
+    __shared__ double dscratch[64];
+    float* tile = reinterpret_cast<float*>(smem_raw);                      // [4*tile4 + 4*CPT]
+    double* xg = reinterpret_cast<double*>(tile + 4 * a.tile4 + 4 * CPT);
     const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
     const int grp = tid / a.tg, t = tid - grp * a.tg;
     const float mpos = __uint_as_float(a.st->mpos_bits), mneg = __uint_as_float(a.st->mneg_bits);
@@ -110,7 +111,8 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
     const GridSetup g = grid_setup(mpos, mneg, a.hi_frac, a.n_cand, flo, fhi);
     const float a_last = __fmul_rn((float)a.n_cand, g.step);
     if (!(m > 0.f) || !(a_last >= FLT_MIN)) return;   // degenerate tensor: finish kernel reports it
-    const float drop_below = 0.4999f * g.step;
+    const float inv_thr = g.rstep * (1.0f / 0.4999f);
+    const float inv_tg = 1.0f / (float)a.tg;
 
     u64 inv2[CPT], na2[CPT];
     double dacc[CPT];
@@ -131,18 +133,21 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
     const long long n4_total = (a.n + 3) >> 2;
     const long long n_tiles = (n4_total + a.tile4 - 1) / a.tile4;
     const float4* x4 = reinterpret_cast<const float4*>(a.x);
-    const int per_thread4 = a.tile4 / nthr;          // consecutive float4s staged by one thread
-    double dropped = 0.0;
+    const int per_thread4 = a.tile4 / nthr;          // consecutive float4s staged by one thread (<= 4)
+    double skipped[CPT + 1];                         // squared sums per class over this block's tiles
+#pragma unroll
+    for (int b = 0; b <= CPT; ++b) skipped[b] = 0.0;
     for (long long tl = blockIdx.x; tl < n_tiles; tl += gridDim.x) {
         const long long base4 = tl * a.tile4;
         const int cnt4 = (int)min((long long)a.tile4, n4_total - base4);
-        // ---- load this thread's span, count what it keeps
-        float keep[16];
-        int n_keep = 0;
-        for (int j = 0; j < per_thread4; ++j) {
-            const int i = tid * per_thread4 + j;
+        // ---- load this thread's span, classify, count
+        float vals[16];
+        u64 cls = 0ull, c0 = 0ull, c1 = 0ull;        // 4-bit class per value; counts in 16-bit fields
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
             float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (i < cnt4) {
+            const int i = tid * per_thread4 + j;
+            if (j < per_thread4 && i < cnt4) {
                 const long long e = (base4 + i) << 2;
                 if (e + 3 < a.n) {
                     v = __ldg(x4 + base4 + i);
@@ -155,38 +160,85 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
             const float e4[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-                if (fabsf(e4[q]) > drop_below) {
-                    keep[n_keep++] = e4[q];
-                } else {
-                    dropped += (double)e4[q] * (double)e4[q];
-                }
+                const float x = e4[q];
+                int nb = magnitude_class<CPT>(x, inv_thr, inv_tg);
+                if (g.tiny && x != 0.f) nb = CPT;
+                vals[4 * j + q] = x;
+                cls |= (u64)nb << (4 * (4 * j + q));
+                const double xx = (double)x * (double)x;
+#pragma unroll
+                for (int b = 0; b <= CPT; ++b) skipped[b] += (nb == b) ? xx : 0.0;
+                if (nb >= 5) c1 += 1ull << (16 * (nb - 5));
+                else if (nb >= 1) c0 += 1ull << (16 * (nb - 1));
             }
         }
-        // ---- exclusive scan of the counts over the block (lanes by shuffle, warps in order)
-        int incl = n_keep;
+        // ---- exclusive scan of the class counts over the block (lanes by shuffle, warps in order)
+        u64 i0 = c0, i1 = c1;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
-            const int up = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += up;
+            const u64 u0 = __shfl_up_sync(0xffffffffu, i0, o);
+            const u64 u1 = __shfl_up_sync(0xffffffffu, i1, o);
+            if (lane >= o) {
+                i0 += u0;
+                i1 += u1;
+            }
         }
         __syncthreads();   // previous tile fully swept; warp_tot free
-        if (lane == 31) warp_tot[warp] = incl;
-        __syncthreads();
-        int offset = incl - n_keep, total = 0;
-        for (int w = 0; w < nwarp; ++w) {
-            const int wt = warp_tot[w];
-            if (w < warp) offset += wt;
-            total += wt;
+        if (lane == 31) {
+            warp_tot[warp][0] = i0;
+            warp_tot[warp][1] = i1;
         }
-        for (int j = 0; j < n_keep; ++j) tile[offset + j] = keep[j];
-        const int padded = (total + 3) & ~3;
-        if (tid < padded - total) tile[total + tid] = 0.f;
         __syncthreads();
-        const int kept4 = padded >> 2;
-        const int beg4 = (int)(((long long)kept4 * grp) / a.groups);
-        const int end4 = (int)(((long long)kept4 * (grp + 1)) / a.groups);
-        sweep_dispatch<CPT>(ncl, reinterpret_cast<const float4*>(tile), beg4, end4, inv2, na2, dacc, kMagic + flo,
-                            kMagic + fhi);
+        u64 off0 = i0 - c0, off1 = i1 - c1, tot0 = 0ull, tot1 = 0ull;
+        for (int w = 0; w < nwarp; ++w) {
+            const u64 a0 = warp_tot[w][0], a1 = warp_tot[w][1];
+            if (w < warp) {
+                off0 += a0;
+                off1 += a1;
+            }
+            tot0 += a0;
+            tot1 += a1;
+        }
+        // ---- class layout in the tile buffer: class CPT first, each padded with zeros to a multiple of 4
+        int base[CPT + 1], len4[CPT + 1];
+        int pos = 0;
+#pragma unroll
+        for (int b = CPT; b >= 1; --b) {
+            const int cnt = (int)(((b >= 5 ? tot1 : tot0) >> (16 * ((b - 1) & 3))) & 0xffffull);
+            base[b] = pos;
+            const int padded = (cnt + 3) & ~3;
+            len4[b] = padded >> 2;
+            if (tid < padded - cnt) tile[pos + cnt + tid] = 0.f;
+            pos += padded;
+        }
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+            const int nb = (int)((cls >> (4 * e)) & 0xfull);
+            if (nb >= 1) {
+                const int sh = 16 * ((nb - 1) & 3);
+                int within;
+                if (nb >= 5) {
+                    within = (int)((off1 >> sh) & 0xffffull);
+                    off1 += 1ull << sh;
+                } else {
+                    within = (int)((off0 >> sh) & 0xffffull);
+                    off0 += 1ull << sh;
+                }
+                int bs = 0;
+#pragma unroll
+                for (int b = 1; b <= CPT; ++b) bs = (nb == b) ? base[b] : bs;
+                tile[bs + within] = vals[e];
+            }
+        }
+        __syncthreads();
+        const float4* tile4p = reinterpret_cast<const float4*>(tile);
+#pragma unroll
+        for (int b = CPT; b >= 1; --b) {
+            const int first4 = base[b] >> 2;
+            const int beg4 = first4 + (int)(((long long)len4[b] * grp) / a.groups);
+            const int end4 = first4 + (int)(((long long)len4[b] * (grp + 1)) / a.groups);
+            sweep_dispatch<CPT>(b, ncl, tile4p, beg4, end4, inv2, na2, dacc, kMagic + flo, kMagic + fhi);
+        }
     }
     if (a.groups > 1) {
         __syncthreads();
@@ -201,15 +253,21 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
                 for (int sl = 0; sl < CPT; ++sl) dacc[sl] += xg[((gg - 1) * CPT + sl) * a.tg + t];
         }
     }
-    // ---- sum of squares of the dropped elements of this block (fixed order), added to every candidate
-    __shared__ double dscratch[64];
+    // ---- what each slot skipped in this block: classes 0..sl (block sums in fixed order)
     long long zero = 0;
-    block_sum2(dropped, zero, dscratch);
+    double run = 0.0;
+#pragma unroll
+    for (int b = 0; b < CPT; ++b) {
+        double v = skipped[b];
+        block_sum2(v, zero, dscratch);
+        run += v;
+        dacc[b] += run;          // slot b skips classes 0..b
+    }
     if (grp == 0) {
 #pragma unroll
         for (int sl = 0; sl < CPT; ++sl) {
             const int c = sl * a.tg + t;
-            if (c < a.n_cand) a.partials[(long long)blockIdx.x * a.n_cand + c] = dacc[sl] + dropped;
+            if (c < a.n_cand) a.partials[(long long)blockIdx.x * a.n_cand + c] = dacc[sl];
         }
     }
 }

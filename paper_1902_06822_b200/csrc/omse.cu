@@ -23,6 +23,9 @@
 #ifndef OMSE_PRUNE
 #define OMSE_PRUNE 1
 #endif
+#ifndef OMSE_SMALL_PRUNE_K
+#define OMSE_SMALL_PRUNE_K 192      /* short rows at least this long are regrouped by magnitude class */
+#endif
 #ifndef OMSE_SMALL_K
 #define OMSE_SMALL_K 640            /* rows up to this length are batched per work unit */
 #endif
@@ -328,10 +331,14 @@ int omse_quantize_weights_batched(omse_ctx* ctx, const omse_weight_tensor* tenso
         if (units_if_small >= 4ll * ctx->n_sm) {
             for (auto& t : list) {
                 if (t.K > OMSE_SMALL_K) continue;
-                t.small = 1;
+                const bool prune = OMSE_PRUNE && t.K >= OMSE_SMALL_PRUNE_K;
+                t.small = prune ? 3 : 1;
                 t.rows_per_unit = t.K <= 128 ? 8 : 4;
                 const size_t kpad = (size_t)((t.K + 3) & ~3ll);
-                const size_t need = (size_t)t.rows_per_unit * (kpad * 4 + (size_t)ncs * 4 + 16);
+                // per row: the row, its error curve, its grid; when regrouping also skipped sums, class table, regrouped row
+                const size_t need = (size_t)t.rows_per_unit *
+                    (kpad * 4 + (size_t)ncs * 4 + 16 +
+                     (prune ? (size_t)cpt * 8 + 2 * (cpt + 1) * 4 + (kpad + 4 * cpt) * 4 : 0));
                 if (need > smem_small) smem_small = need;
             }
         }

@@ -157,6 +157,79 @@ __device__ __forceinline__ void sweep_dispatch(int ncl, const float4* xs4, int b
 }
 
 // ---------------------------------------------------------------------------------------------
+// The same evaluation without the fp64 fold: the caller keeps the fp32 pair sums across several
+// spans (at most kFlushEvery4 loads between two folds) and folds them itself.  Used where a row is
+// swept as a handful of short spans (magnitude classes of a short row).
+// ---------------------------------------------------------------------------------------------
+template <int CPT, int NACT, int NCL>
+__device__ __forceinline__ void sweep_accum(const float4* __restrict__ xs4, int beg4, int end4,
+                                            const u64 (&inv2)[CPT], const u64 (&na2)[CPT], u64 (&acc2)[CPT],
+                                            float clo, float chi) {
+    const u64 M2 = pack2(kMagic, kMagic);
+    const u64 NM2 = pack2(-kMagic, -kMagic);
+#pragma unroll 1
+    for (int i = beg4; i < end4; ++i) {
+        const float4 v = xs4[i];
+        const u64 xa = pack2(v.x, v.y), xb = pack2(v.z, v.w);
+#pragma unroll
+        for (int s = 0; s < NACT; ++s) {
+            u64 ta = fma2(xa, inv2[s], M2);
+            u64 tb = fma2(xb, inv2[s], M2);
+            if (s < NCL) {
+                float a0, a1, b0, b1;
+                unpack2(ta, a0, a1);
+                unpack2(tb, b0, b1);
+                a0 = fminf(fmaxf(a0, clo), chi);
+                a1 = fminf(fmaxf(a1, clo), chi);
+                b0 = fminf(fmaxf(b0, clo), chi);
+                b1 = fminf(fmaxf(b1, clo), chi);
+                ta = pack2(a0, a1);
+                tb = pack2(b0, b1);
+            }
+            const u64 qa = add2(ta, NM2);
+            const u64 qb = add2(tb, NM2);
+            const u64 ea = fma2(na2[s], qa, xa);
+            const u64 eb = fma2(na2[s], qb, xb);
+            acc2[s] = fma2(ea, ea, acc2[s]);
+            acc2[s] = fma2(eb, eb, acc2[s]);
+        }
+    }
+}
+
+template <int CPT, int NACT>
+__device__ __forceinline__ void sweep_accum_ncl(int ncl, const float4* xs4, int beg4, int end4,
+                                                const u64 (&inv2)[CPT], const u64 (&na2)[CPT], u64 (&acc2)[CPT],
+                                                float clo, float chi) {
+    if (ncl <= 0) {
+        sweep_accum<CPT, NACT, 0>(xs4, beg4, end4, inv2, na2, acc2, clo, chi);
+    } else if (ncl == 1) {
+        sweep_accum<CPT, NACT, 1>(xs4, beg4, end4, inv2, na2, acc2, clo, chi);
+    } else if (ncl == 2 && NACT > 2) {
+        sweep_accum<CPT, NACT, (NACT > 2 ? 2 : NACT)>(xs4, beg4, end4, inv2, na2, acc2, clo, chi);
+    } else {
+        sweep_accum<CPT, NACT, NACT>(xs4, beg4, end4, inv2, na2, acc2, clo, chi);
+    }
+}
+
+template <int CPT>
+__device__ __forceinline__ void sweep_accum_dispatch(int nact, int ncl, const float4* xs4, int beg4, int end4,
+                                                     const u64 (&inv2)[CPT], const u64 (&na2)[CPT],
+                                                     u64 (&acc2)[CPT], float clo, float chi) {
+    if (beg4 >= end4 || nact <= 0) return;
+    if (ncl > nact) ncl = nact;
+    switch (nact) {
+        case 1: sweep_accum_ncl<CPT, 1>(ncl, xs4, beg4, end4, inv2, na2, acc2, clo, chi); break;
+        case 2: if constexpr (CPT >= 2) sweep_accum_ncl<CPT, 2>(ncl, xs4, beg4, end4, inv2, na2, acc2, clo, chi); break;
+        case 3: if constexpr (CPT >= 4) sweep_accum_ncl<CPT, 3>(ncl, xs4, beg4, end4, inv2, na2, acc2, clo, chi); break;
+        case 4: if constexpr (CPT >= 4) sweep_accum_ncl<CPT, 4>(ncl, xs4, beg4, end4, inv2, na2, acc2, clo, chi); break;
+        case 5: if constexpr (CPT >= 8) sweep_accum_ncl<CPT, 5>(ncl, xs4, beg4, end4, inv2, na2, acc2, clo, chi); break;
+        case 6: if constexpr (CPT >= 8) sweep_accum_ncl<CPT, 6>(ncl, xs4, beg4, end4, inv2, na2, acc2, clo, chi); break;
+        case 7: if constexpr (CPT >= 8) sweep_accum_ncl<CPT, 7>(ncl, xs4, beg4, end4, inv2, na2, acc2, clo, chi); break;
+        default: sweep_accum_ncl<CPT, CPT>(ncl, xs4, beg4, end4, inv2, na2, acc2, clo, chi); break;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 // Block-wide reductions (fixed order: lanes by shuffle tree, warps in index order) so that results
 // do not depend on scheduling.  `scratch` holds at least 2*32 doubles.  All threads get the result.
 // ---------------------------------------------------------------------------------------------

@@ -22,7 +22,8 @@ struct RowTensor {
     long long unit_begin;    // index of this tensor's first work unit in the launch-wide numbering
     int rows_per_unit;       // long rows: 2 when nibble packing needs an even element count per unit (odd K), else 1;
                              // short rows: the batch size B (even)
-    int small;               // 1: short-row path (batch of rows per unit, a warp finishes each row)
+    int small;               // bit 0: short-row path (batch of rows per unit, a warp finishes each row);
+                             // bit 1: that path regroups rows by magnitude class
 };
 
 struct RowArgs {

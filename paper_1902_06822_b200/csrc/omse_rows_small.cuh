@@ -258,9 +258,14 @@ __device__ void small_unit(const RowArgs& a, const RowTensor& T, long long unit_
     const long long row0 = unit_local * B;
     const int nrows = (int)min((long long)B, T.S - row0);
     const int ncs = CPT * a.tg;
+    const bool prune = (T.small & 2) != 0;       // rows regrouped by magnitude class before the sweep
+    const int kb = kpad + 4 * CPT;               // floats of a regrouped row (every class padded to 4)
     float* xs = reinterpret_cast<float*>(smem_raw);
     float* curve = xs + B * kpad;
     SmallRowParams* rowp = reinterpret_cast<SmallRowParams*>(curve + B * ncs);
+    double* skip = reinterpret_cast<double*>(rowp + B);            // [B][CPT]   (prune only)
+    int* seg = reinterpret_cast<int*>(skip + B * CPT);              // [B][2*(CPT+1)]
+    float* xb = reinterpret_cast<float*>(seg + B * 2 * (CPT + 1));  // [B][kb]
     const float flo = (float)a.lo[0], fhi = (float)a.hi[0];
 
     // ---- stage the rows (contiguous in HBM) into rows of kpad floats, zero padded
@@ -315,6 +320,81 @@ __device__ void small_unit(const RowArgs& a, const RowTensor& T, long long unit_
             rp.flags = (g.tiny ? 1 : 0) | ((!(fmaxf(mp, mn) > 0.f) || !(a_last >= FLT_MIN)) ? 2 : 0);
             rowp[r] = rp;
         }
+        if (prune) {
+            // ---- regroup the row by magnitude class: the same counting sort as the long-row path, by one warp
+            __syncwarp();
+            const SmallRowParams rp = rowp[r];
+            const bool plain = (rp.flags & 3) != 0;           // denormal-range or unusable row: one class, all slots
+            const float inv_thr = rp.rstep * (1.0f / 0.4999f), inv_tg = 1.0f / (float)a.tg;
+            const int span = (k + 31) >> 5;
+            const int beg = min(k, lane * span), end = min(k, beg + span);
+            const float* xr = xs + r * kpad;
+            u64 c0 = 0ull, c1 = 0ull;
+            double d[CPT + 1];
+#pragma unroll
+            for (int b = 0; b <= CPT; ++b) d[b] = 0.0;
+            for (int i = beg; i < end; ++i) {
+                const float x = xr[i];
+                const int nb = plain ? CPT : magnitude_class<CPT>(x, inv_thr, inv_tg);
+                const double xx = (double)x * (double)x;
+#pragma unroll
+                for (int b = 0; b <= CPT; ++b) d[b] += (nb == b) ? xx : 0.0;
+                if (nb >= 5) c1 += 1ull << (16 * (nb - 5));
+                else if (nb >= 1) c0 += 1ull << (16 * (nb - 1));
+            }
+            u64 i0 = c0, i1 = c1;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const u64 u0 = __shfl_up_sync(0xffffffffu, i0, o);
+                const u64 u1 = __shfl_up_sync(0xffffffffu, i1, o);
+                if (lane >= o) {
+                    i0 += u0;
+                    i1 += u1;
+                }
+            }
+            u64 off0 = i0 - c0, off1 = i1 - c1;
+            const u64 tot0 = __shfl_sync(0xffffffffu, i0, 31), tot1 = __shfl_sync(0xffffffffu, i1, 31);
+            int base[CPT + 1];
+            int pos = 0;
+            float* xbr = xb + r * kb;
+#pragma unroll
+            for (int b = CPT; b >= 1; --b) {
+                const int cnt = (int)(((b >= 5 ? tot1 : tot0) >> (16 * ((b - 1) & 3))) & 0xffffull);
+                base[b] = pos;
+                const int padded = (cnt + 3) & ~3;
+                if (lane == 0) {
+                    seg[(r * (CPT + 1) + b) * 2] = pos;
+                    seg[(r * (CPT + 1) + b) * 2 + 1] = padded;
+                }
+                if (lane < padded - cnt) xbr[pos + cnt + lane] = 0.f;
+                pos += padded;
+            }
+            for (int i = beg; i < end; ++i) {
+                const float x = xr[i];
+                const int nb = plain ? CPT : magnitude_class<CPT>(x, inv_thr, inv_tg);
+                if (nb >= 1) {
+                    const int sh = 16 * ((nb - 1) & 3);
+                    int within;
+                    if (nb >= 5) {
+                        within = (int)((off1 >> sh) & 0xffffull);
+                        off1 += 1ull << sh;
+                    } else {
+                        within = (int)((off0 >> sh) & 0xffffull);
+                        off0 += 1ull << sh;
+                    }
+                    int bs = 0;
+#pragma unroll
+                    for (int b = 1; b <= CPT; ++b) bs = (nb == b) ? base[b] : bs;
+                    xbr[bs + within] = x;
+                }
+            }
+            double run = 0.0;                                   // slot sl skips classes 0..sl
+#pragma unroll
+            for (int b = 0; b < CPT; ++b) {
+                run += warp_allsum(d[b]);
+                if (lane == 0) skip[r * CPT + b] = run;
+            }
+        }
     }
     __syncthreads();
 
@@ -346,7 +426,46 @@ __device__ void small_unit(const RowArgs& a, const RowTensor& T, long long unit_
         ncl = max(0, min(CPT, ncl));
         const float4* xr4 = reinterpret_cast<const float4*>(xs) + r * k4;
         float* cvr = curve + r * ncs;
-        if (short_rows) {
+        if (prune) {
+            // class nb is evaluated by slots 0..nb-1; fp32 pair sums are kept across classes and folded
+            // into fp64 every kFlushEvery4 loads
+            const float4* xb4 = reinterpret_cast<const float4*>(xb + r * kb);
+            u64 acc2[CPT];
+            double dacc[CPT];
+#pragma unroll
+            for (int sl = 0; sl < CPT; ++sl) {
+                acc2[sl] = 0ull;
+                dacc[sl] = 0.0;
+            }
+            int pending = 0;
+            for (int b = CPT; b >= 1; --b) {
+                int i = seg[(r * (CPT + 1) + b) * 2] >> 2;
+                const int stop = i + (seg[(r * (CPT + 1) + b) * 2 + 1] >> 2);
+                while (i < stop) {
+                    const int n = min(stop - i, kFlushEvery4 - pending);
+                    sweep_accum_dispatch<CPT>(b, ncl, xb4, i, i + n, inv2, na2, acc2, kMagic + flo, kMagic + fhi);
+                    i += n;
+                    pending += n;
+                    if (pending == kFlushEvery4) {
+#pragma unroll
+                        for (int sl = 0; sl < CPT; ++sl) {
+                            float p0, p1;
+                            unpack2(acc2[sl], p0, p1);
+                            dacc[sl] += (double)(p0 + p1);
+                            acc2[sl] = 0ull;
+                        }
+                        pending = 0;
+                    }
+                }
+            }
+#pragma unroll
+            for (int sl = 0; sl < CPT; ++sl) {
+                float p0, p1;
+                unpack2(acc2[sl], p0, p1);
+                const double v = dacc[sl] + (double)(p0 + p1) + skip[r * CPT + sl];
+                cvr[sl * a.tg + tid] = ok[sl] ? (float)v : INFINITY;
+            }
+        } else if (short_rows) {
             float out[CPT];
             sweep_short_dispatch<CPT>(ncl, xr4, k4, inv2, na2, out, kMagic + flo, kMagic + fhi);
 #pragma unroll

@@ -123,8 +123,6 @@ __device__ __forceinline__ void sweep_ncl(int ncl, const float4* xs4, int beg4, 
         sweep_range<CPT, NACT, 1>(xs4, beg4, end4, inv2, na2, dacc, clo, chi);
     } else if (ncl == 2 && NACT > 2) {
         sweep_range<CPT, NACT, (NACT > 2 ? 2 : NACT)>(xs4, beg4, end4, inv2, na2, dacc, clo, chi);
-    } else if (ncl <= 4 && NACT > 4) {
-        sweep_range<CPT, NACT, (NACT > 4 ? 4 : NACT)>(xs4, beg4, end4, inv2, na2, dacc, clo, chi);
     } else {
         sweep_range<CPT, NACT, NACT>(xs4, beg4, end4, inv2, na2, dacc, clo, chi);
     }
@@ -142,9 +140,7 @@ __device__ __forceinline__ void sweep_dispatch(int nact, int ncl, const float4* 
         case 2: if constexpr (CPT >= 2) sweep_ncl<CPT, 2>(ncl, xs4, beg4, end4, inv2, na2, dacc, clo, chi); break;
         case 3: if constexpr (CPT >= 4) sweep_ncl<CPT, 3>(ncl, xs4, beg4, end4, inv2, na2, dacc, clo, chi); break;
         case 4: if constexpr (CPT >= 4) sweep_ncl<CPT, 4>(ncl, xs4, beg4, end4, inv2, na2, dacc, clo, chi); break;
-        case 5: if constexpr (CPT >= 8) sweep_ncl<CPT, 5>(ncl, xs4, beg4, end4, inv2, na2, dacc, clo, chi); break;
         case 6: if constexpr (CPT >= 8) sweep_ncl<CPT, 6>(ncl, xs4, beg4, end4, inv2, na2, dacc, clo, chi); break;
-        case 7: if constexpr (CPT >= 8) sweep_ncl<CPT, 7>(ncl, xs4, beg4, end4, inv2, na2, dacc, clo, chi); break;
         default: sweep_ncl<CPT, CPT>(ncl, xs4, beg4, end4, inv2, na2, dacc, clo, chi); break;
     }
 }
@@ -222,9 +218,7 @@ __device__ __forceinline__ void sweep_accum_dispatch(int nact, int ncl, const fl
         case 2: if constexpr (CPT >= 2) sweep_accum_ncl<CPT, 2>(ncl, xs4, beg4, end4, inv2, na2, acc2, clo, chi); break;
         case 3: if constexpr (CPT >= 4) sweep_accum_ncl<CPT, 3>(ncl, xs4, beg4, end4, inv2, na2, acc2, clo, chi); break;
         case 4: if constexpr (CPT >= 4) sweep_accum_ncl<CPT, 4>(ncl, xs4, beg4, end4, inv2, na2, acc2, clo, chi); break;
-        case 5: if constexpr (CPT >= 8) sweep_accum_ncl<CPT, 5>(ncl, xs4, beg4, end4, inv2, na2, acc2, clo, chi); break;
         case 6: if constexpr (CPT >= 8) sweep_accum_ncl<CPT, 6>(ncl, xs4, beg4, end4, inv2, na2, acc2, clo, chi); break;
-        case 7: if constexpr (CPT >= 8) sweep_accum_ncl<CPT, 7>(ncl, xs4, beg4, end4, inv2, na2, acc2, clo, chi); break;
         default: sweep_accum_ncl<CPT, CPT>(ncl, xs4, beg4, end4, inv2, na2, acc2, clo, chi); break;
     }
 }
@@ -331,7 +325,19 @@ __device__ __forceinline__ int magnitude_class(float x, float inv_thr, float inv
     const float r = ax * inv_thr;              // |x| / (0.4999*step)
     if (r <= 1.0f) return 0;
     const float f = (r - 1.0f) * inv_tg;       // slot sl needs x iff r > sl*tg + 1
-    return f >= (float)CPT ? CPT : (int)f + 1;
+    int nb = f >= (float)CPT ? CPT : (int)f + 1;
+    if (CPT == 8 && (nb == 5 || nb == 7)) ++nb;   // classes 5 and 7 are merged upwards: fewer sweep variants
+    return nb;
+}
+
+// Candidates with index below the returned value may saturate on an element of magnitude class nb
+// (nb < CPT bounds |x| from above: |x| < 0.4999*(nb*tg+1)*step, and candidate c saturates only if
+// |x| >= min(hi+1/2, 1/2-lo)*alpha_c); class CPT has no upper bound and keeps the row's own count.
+__device__ __forceinline__ int class_sat_count(int nb, int cpt, int tg, int c_sat_row, float flo, float fhi) {
+    if (nb >= cpt) return c_sat_row;
+    const float den = fminf(fhi + 0.5f, 0.5f - flo);
+    const int c = (int)(0.5f * (float)(nb * tg + 1) / den) + 2;
+    return min(c, c_sat_row);
 }
 
 // Per-candidate constants of one thread for the grid of Section 3.4 on a tensor with max|x| = m.

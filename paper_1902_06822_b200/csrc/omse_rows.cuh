@@ -236,7 +236,9 @@ __device__ PhiOut phi_block(const RowArgs& a, const RowSmem& s, int k, int k4, f
             const int first4 = s.seg[2 * b] >> 2, len4 = s.seg[2 * b + 1] >> 2;
             const int beg4 = first4 + (int)(((long long)len4 * grp) / a.groups);
             const int end4 = first4 + (int)(((long long)len4 * (grp + 1)) / a.groups);
-            sweep_dispatch<CPT>(b, ncl, xb4, beg4, end4, inv2, na2, dacc, kMagic + flo, kMagic + fhi);
+            int ncl_b = (class_sat_count(b, CPT, a.tg, g.c_sat, flo, fhi) - warp_t0 + a.tg - 1) / a.tg;
+            ncl_b = max(0, min(CPT, ncl_b));
+            sweep_dispatch<CPT>(b, ncl_b, xb4, beg4, end4, inv2, na2, dacc, kMagic + flo, kMagic + fhi);
         }
         if (grp == 0) {
 #pragma unroll

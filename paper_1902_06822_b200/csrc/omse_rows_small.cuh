@@ -441,9 +441,11 @@ __device__ void small_unit(const RowArgs& a, const RowTensor& T, long long unit_
             for (int b = CPT; b >= 1; --b) {
                 int i = seg[(r * (CPT + 1) + b) * 2] >> 2;
                 const int stop = i + (seg[(r * (CPT + 1) + b) * 2 + 1] >> 2);
+                int ncl_b = (class_sat_count(b, CPT, a.tg, rp.c_sat, flo, fhi) - (tid & ~31) + a.tg - 1) / a.tg;
+                ncl_b = max(0, min(CPT, ncl_b));
                 while (i < stop) {
                     const int n = min(stop - i, kFlushEvery4 - pending);
-                    sweep_accum_dispatch<CPT>(b, ncl, xb4, i, i + n, inv2, na2, acc2, kMagic + flo, kMagic + fhi);
+                    sweep_accum_dispatch<CPT>(b, ncl_b, xb4, i, i + n, inv2, na2, acc2, kMagic + flo, kMagic + fhi);
                     i += n;
                     pending += n;
                     if (pending == kFlushEvery4) {

@@ -237,7 +237,9 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
             const int first4 = base[b] >> 2;
             const int beg4 = first4 + (int)(((long long)len4[b] * grp) / a.groups);
             const int end4 = first4 + (int)(((long long)len4[b] * (grp + 1)) / a.groups);
-            sweep_dispatch<CPT>(b, ncl, tile4p, beg4, end4, inv2, na2, dacc, kMagic + flo, kMagic + fhi);
+            int ncl_b = (class_sat_count(b, CPT, a.tg, g.c_sat, flo, fhi) - warp_t0 + a.tg - 1) / a.tg;
+            ncl_b = max(0, min(CPT, ncl_b));
+            sweep_dispatch<CPT>(b, ncl_b, tile4p, beg4, end4, inv2, na2, dacc, kMagic + flo, kMagic + fhi);
         }
     }
     if (a.groups > 1) {

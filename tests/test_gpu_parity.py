@@ -232,3 +232,50 @@ def test_batched_launch_matches_per_tensor_results(gpu):
     gpu.ctx().omse_quantize_weights_batched(descs, 4, True, 1024, 1.0, 3)
     torch.cuda.synchronize()
     assert torch.equal(before, descs[2]["alpha"])
+
+
+# ---------------------------------------------------------------- magnitude-class regrouping (long and short rows)
+@pytest.mark.parametrize("n_cand", [1, 16, 50, 100, 256, 500, 1024, 2048, 4096])
+def test_long_rows_regrouped_for_every_candidate_layout(gpu, n_cand):
+    """Rows of 1024+ elements are regrouped by magnitude class; every candidates-per-thread layout."""
+    w = synth.student_t3(5 * 1500, seed=400, tensor_id=n_cand).reshape(5, 1500)
+    _run_and_check(gpu, w, 4, True, n_cand, 3, codes=True, packed=True)
+    w = synth.laplace(3 * 9000, 0.01, seed=401, tensor_id=n_cand).reshape(3, 9000)     # several element groups
+    _run_and_check(gpu, w, 3, True, n_cand, 2, codes=True, packed=False)
+
+
+@pytest.mark.parametrize("k", [192, 193, 256, 500, 640])
+def test_short_rows_regrouped_in_large_launches(gpu, k):
+    """Enough short rows for the batched short-row path, with regrouping (192 <= K <= 640)."""
+    s = 2500
+    w = synth.laplace(s * k, 0.03, seed=410, tensor_id=k).reshape(s, k)
+    _run_and_check(gpu, w, 4, True, 1024, 3, codes=True, packed=True, rows=np.arange(0, s, 7))
+    _run_and_check(gpu, np.abs(w), 4, False, 1024, 1, codes=False, packed=False, rows=np.arange(3, s, 11))
+
+
+def test_regrouping_corner_cases(gpu):
+    k = 2048
+    rng = np.random.default_rng(7)
+    rows = [
+        np.full(k, 0.37, np.float32),                                   # one magnitude: a single class
+        np.where(np.arange(k) % 2 == 0, 1.0, -1.0).astype(np.float32),  # +-max only
+        np.concatenate([[5.0], np.full(k - 1, 1e-6)]).astype(np.float32),   # one large element, rest below step/2
+        np.concatenate([[5.0], np.zeros(k - 1)]).astype(np.float32),    # one element, exact zeros
+        (rng.integers(-8, 8, k) * 0.125).astype(np.float32),            # already on a grid
+        np.linspace(-1.0, 1.0, k).astype(np.float32),                   # every class populated
+        (np.linspace(0.0, 1.0, k) ** 8).astype(np.float32),             # heavy concentration near zero
+    ]
+    w = np.stack(rows)
+    for bits, signed in [(4, True), (2, True), (8, True), (4, False), (3, False)]:
+        _run_and_check(gpu, w, bits, signed, 1024, 3, codes=True, packed=bits <= 4)
+    _run_and_check(gpu, w, 4, True, 1024, 3, hi_frac=1.0 / 7, codes=True, packed=True)     # grid far below max|x|
+    _run_and_check(gpu, w, 4, True, 1024, 3, hi_frac=2.0, codes=True, packed=True)         # grid beyond max|x|
+
+
+def test_residual_on_regrouped_long_rows(gpu):
+    t = synth.laplace_with_outliers(6 * 3000, 0.005, seed=420, outlier_prob=0.005).reshape(6, 3000)
+    _residual_step_by_step(gpu, t, (4, 4), 1024, 3, packed=True)
+    alpha, sse, q, _ = gpu.residual_quantize(t, (4, 3), True, 512, 1.0, 2, n_sweeps=2)
+    ref = orc.residual_rows(t, (4, 3), True, 512, 1.0, 2, n_sweeps=2)
+    np.testing.assert_allclose(alpha, ref.alpha, rtol=RTOL)
+    np.testing.assert_allclose(sse, ref.sse, rtol=RTOL)

@@ -306,6 +306,155 @@ void omse_oracle_residual_rows(const float *t, int64_t n_kernels, int64_t kernel
     *status |= st_all;
 }
 
+/*
+ * Dual line search (Section 3.5, the n = 2 case, third displayed equation of that section): for a
+ * pair of scales (alpha1, alpha2) every element picks the first code t in Z_p1 by enumeration, the
+ * second code being the rounding of what is left:
+ *     min over t in Z_p1 of ( T_j - alpha1*t - alpha2*[ (T_j - alpha1*t)/alpha2 ]_Zp2 )^2 ,
+ * and the pair of scales is found on a two-dimensional grid.  The paper gives no grid; here
+ * alpha1_c = (c+1)/C1 * hi_frac1 * max|T|  and  alpha2_{c,d} = (d+1)/C2 * hi_frac2 * alpha1_c,
+ * every operation in binary32 (same form as the one-dimensional grid).
+ * Decisions are taken in binary32: r = fmaf(-alpha1, t, x); q = [r/alpha2]_Zp2;
+ * e = fmaf(-alpha2, q, r); the t with the smallest e*e wins, lowest t on ties.  The reported error is
+ * the objective itself in binary64 for the chosen codes.
+ */
+static void dual_codes_of(float x, float a1, float a2, int lo1, int hi1, int lo2, int hi2, int *t_out,
+                          int *q_out)
+{
+    float best = INFINITY;
+    int bt = lo1, bq = 0;
+    for (int t = lo1; t <= hi1; ++t) {
+        float r = fmaf(-a1, (float)t, x);
+        int q = code_of(r, a2, lo2, hi2);
+        float e = fmaf(-a2, (float)q, r);
+        float ee = e * e;
+        if (ee < best) {
+            best = ee;
+            bt = t;
+            bq = q;
+        }
+    }
+    *t_out = bt;
+    *q_out = bq;
+}
+
+static double dual_sse_of(const float *x, int64_t k, float a1, float a2, int lo1, int hi1, int lo2,
+                          int hi2)
+{
+    double s = 0.0;
+    for (int64_t i = 0; i < k; ++i) {
+        int t, q;
+        dual_codes_of(x[i], a1, a2, lo1, hi1, lo2, hi2, &t, &q);
+        double d = (double)x[i] - (double)a1 * (double)t - (double)a2 * (double)q;
+        s += d * d;
+    }
+    return s;
+}
+
+double omse_oracle_dual_sse_at(const float *x, int64_t k, float a1, float a2, int bits1, int bits2,
+                               int is_signed)
+{
+    int lo1, hi1, lo2, hi2;
+    omse_oracle_grid_bounds(bits1, is_signed, &lo1, &hi1);
+    omse_oracle_grid_bounds(bits2, is_signed, &lo2, &hi2);
+    return dual_sse_of(x, k, a1, a2, lo1, hi1, lo2, hi2);
+}
+
+void omse_oracle_dual_scales(float max_abs, float hi_frac1, float hi_frac2, int n_cand1, int n_cand2,
+                             int c, int d, float *a1, float *a2)
+{
+    *a1 = omse_oracle_candidate(max_abs, hi_frac1, n_cand1, c);
+    *a2 = omse_oracle_candidate(*a1, hi_frac2, n_cand2, d);
+}
+
+/* One segment.  start_idx >= 0 skips the search and takes that flat pair index c*C2+d.
+ * Outputs: alpha[2], *sse, *best_idx (-1 degenerate), codes1[k], codes2[k] (nullable),
+ * sse_curve[C1*C2] (nullable, +inf for unusable pairs). */
+void omse_oracle_dual(const float *x, int64_t k, int bits1, int bits2, int is_signed, int n_cand1,
+                      int n_cand2, float hi_frac1, float hi_frac2, int start_idx, float *alpha,
+                      double *sse, int32_t *best_idx, int8_t *codes1, int8_t *codes2,
+                      double *sse_curve, uint32_t *status)
+{
+    int lo1, hi1, lo2, hi2;
+    uint32_t st = 0;
+    omse_oracle_grid_bounds(bits1, is_signed, &lo1, &hi1);
+    omse_oracle_grid_bounds(bits2, is_signed, &lo2, &hi2);
+    float m = max_abs_of(x, k, &st);
+    int best = -1;
+    double best_sse = INFINITY;
+    float a1, a2;
+    if (start_idx >= 0) {
+        omse_oracle_dual_scales(m, hi_frac1, hi_frac2, n_cand1, n_cand2, start_idx / n_cand2,
+                                start_idx % n_cand2, &a1, &a2);
+        if (a1 >= FLT_MIN && a2 >= FLT_MIN && a1 <= FLT_MAX) best = start_idx;
+    } else {
+        for (int c = 0; c < n_cand1; ++c)
+            for (int d = 0; d < n_cand2; ++d) {
+                omse_oracle_dual_scales(m, hi_frac1, hi_frac2, n_cand1, n_cand2, c, d, &a1, &a2);
+                double s = INFINITY;
+                if (a1 >= FLT_MIN && a2 >= FLT_MIN && a1 <= FLT_MAX)
+                    s = dual_sse_of(x, k, a1, a2, lo1, hi1, lo2, hi2);
+                if (sse_curve) sse_curve[c * n_cand2 + d] = s;
+                if (s < best_sse) {
+                    best_sse = s;
+                    best = c * n_cand2 + d;
+                }
+            }
+    }
+    if (best < 0) {
+        double s = 0.0;
+        for (int64_t i = 0; i < k; ++i) s += (double)x[i] * (double)x[i];
+        alpha[0] = alpha[1] = 0.0f;
+        *sse = s;
+        *best_idx = -1;
+        if (codes1) memset(codes1, 0, (size_t)k);
+        if (codes2) memset(codes2, 0, (size_t)k);
+        *status |= st | ORACLE_STATUS_DEGENERATE;
+        return;
+    }
+    omse_oracle_dual_scales(m, hi_frac1, hi_frac2, n_cand1, n_cand2, best / n_cand2, best % n_cand2,
+                            &a1, &a2);
+    alpha[0] = a1;
+    alpha[1] = a2;
+    *best_idx = best;
+    double s = 0.0;
+    for (int64_t i = 0; i < k; ++i) {
+        int t, q;
+        dual_codes_of(x[i], a1, a2, lo1, hi1, lo2, hi2, &t, &q);
+        if (codes1) codes1[i] = (int8_t)t;
+        if (codes2) codes2[i] = (int8_t)q;
+        double dd = (double)x[i] - (double)a1 * (double)t - (double)a2 * (double)q;
+        s += dd * dd;
+    }
+    *sse = s;
+    *status |= st;
+}
+
+/* Kernel-wise dual search; alpha [2][n_kernels], codes [2][n_kernels*kernel_len]. */
+void omse_oracle_dual_rows(const float *t, int64_t n_kernels, int64_t kernel_len, int bits1, int bits2,
+                           int is_signed, int n_cand1, int n_cand2, float hi_frac1, float hi_frac2,
+                           const int32_t *start_idx, float *alpha, double *sse, int32_t *best_idx,
+                           int8_t *codes, uint32_t *status)
+{
+    int64_t n = n_kernels * kernel_len;
+    uint32_t st_all = 0;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 1) reduction(| : st_all)
+#endif
+    for (int64_t s = 0; s < n_kernels; ++s) {
+        uint32_t st = 0;
+        float a[2];
+        omse_oracle_dual(t + s * kernel_len, kernel_len, bits1, bits2, is_signed, n_cand1, n_cand2,
+                         hi_frac1, hi_frac2, start_idx ? start_idx[s] : -1, a, &sse[s], &best_idx[s],
+                         codes ? codes + s * kernel_len : NULL,
+                         codes ? codes + n + s * kernel_len : NULL, NULL, &st);
+        alpha[s] = a[0];
+        alpha[n_kernels + s] = a[1];
+        st_all |= st;
+    }
+    *status |= st_all;
+}
+
 /* INT4 code emission.  The paper fixes no byte layout; this library's layout is: element e
  * (flat, row-major) goes to byte e/2, even e in bits 0-3, odd e in bits 4-7, the nibble being
  * the low four bits of the two's-complement code; a trailing odd element leaves bits 4-7 zero. */

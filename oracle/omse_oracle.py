@@ -55,6 +55,14 @@ def _load():
                                                  f32p, f64p, i32p, f64p, u32p]
     lib.omse_oracle_residual_rows.argtypes = [f32p, C.c_int64, C.c_int64, C.POINTER(C.c_int), C.c_int, C.c_int,
                                               C.c_float, C.c_int, C.c_int, C.c_int, f32p, f64p, i32p, i8p, u32p]
+    lib.omse_oracle_dual_sse_at.restype = C.c_double
+    lib.omse_oracle_dual_sse_at.argtypes = [f32p, C.c_int64, C.c_float, C.c_float, C.c_int, C.c_int, C.c_int]
+    lib.omse_oracle_dual_scales.argtypes = [C.c_float, C.c_float, C.c_float, C.c_int, C.c_int, C.c_int, C.c_int,
+                                            f32p, f32p]
+    lib.omse_oracle_dual.argtypes = [f32p, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_float,
+                                     C.c_float, C.c_int, f32p, f64p, i32p, i8p, i8p, f64p, u32p]
+    lib.omse_oracle_dual_rows.argtypes = [f32p, C.c_int64, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
+                                          C.c_float, C.c_float, i32p, f32p, f64p, i32p, i8p, u32p]
     lib.omse_oracle_pack_int4.argtypes = [i8p, C.c_int64, u8p]
     lib.omse_oracle_unpack_int4.argtypes = [u8p, C.c_int64, C.c_int, i8p]
     _lib = lib
@@ -187,6 +195,61 @@ def residual_rows(t, bits=(4, 4), is_signed=True, n_cand=1024, hi_frac=1.0, refi
                                       refine_iters, n, n_sweeps, _p(alpha, C.c_float), _p(sse, C.c_double),
                                       _p(idx, C.c_int32), _p(q, C.c_int8), C.byref(st))
     return ResidualResult(alpha, sse, idx, q, st.value)
+
+
+def dual_scales(max_abs, hi_frac1, hi_frac2, n_cand1, n_cand2, c, d):
+    a1, a2 = C.c_float(), C.c_float()
+    _load().omse_oracle_dual_scales(_c32(max_abs), _c32(hi_frac1), _c32(hi_frac2), n_cand1, n_cand2, c, d,
+                                    C.byref(a1), C.byref(a2))
+    return a1.value, a2.value
+
+
+def dual_sse_at(x, a1, a2, bits1=4, bits2=4, is_signed=True) -> float:
+    """Section 3.5 dual objective at a given pair of scales (per-element enumeration of the first code)."""
+    x = _f32(x).ravel()
+    return float(_load().omse_oracle_dual_sse_at(_p(x, C.c_float), x.size, _c32(a1), _c32(a2), bits1, bits2,
+                                                 int(is_signed)))
+
+
+@dataclass
+class DualResult:
+    alpha: np.ndarray      # [2] or [2, S]
+    sse: object            # float or [S] float64
+    best_idx: object       # flat pair index c*C2+d
+    codes: np.ndarray | None   # [2, K] or [2, S, K]
+    sse_curve: np.ndarray | None
+    status: int
+
+
+def dual(x, bits1=4, bits2=4, is_signed=True, n_cand1=32, n_cand2=32, hi_frac1=1.0, hi_frac2=0.25, start_idx=-1,
+         want_curve=False) -> DualResult:
+    """Dual line search of Section 3.5 on one segment."""
+    x = _f32(x).ravel()
+    a = np.zeros(2, np.float32)
+    s, i, st = C.c_double(), C.c_int32(), C.c_uint32(0)
+    q = np.zeros((2, x.size), np.int8)
+    curve = np.empty(n_cand1 * n_cand2, np.float64) if want_curve else None
+    _load().omse_oracle_dual(_p(x, C.c_float), x.size, bits1, bits2, int(is_signed), n_cand1, n_cand2,
+                             _c32(hi_frac1), _c32(hi_frac2), start_idx, _p(a, C.c_float), C.byref(s), C.byref(i),
+                             _p(q[0], C.c_int8), _p(q[1], C.c_int8), _p(curve, C.c_double), C.byref(st))
+    return DualResult(a, s.value, i.value, q, curve, st.value)
+
+
+def dual_rows(t, bits1=4, bits2=4, is_signed=True, n_cand1=32, n_cand2=32, hi_frac1=1.0, hi_frac2=0.25,
+              start_idx=None) -> DualResult:
+    """Kernel-wise dual line search over the rows of a 2-D array."""
+    t = _f32(t)
+    S, K = t.shape
+    alpha = np.zeros((2, S), np.float32)
+    sse = np.zeros(S, np.float64)
+    idx = np.zeros(S, np.int32)
+    q = np.zeros((2, S, K), np.int8)
+    st = C.c_uint32(0)
+    si = None if start_idx is None else np.ascontiguousarray(start_idx, dtype=np.int32)
+    _load().omse_oracle_dual_rows(_p(t, C.c_float), S, K, bits1, bits2, int(is_signed), n_cand1, n_cand2,
+                                  _c32(hi_frac1), _c32(hi_frac2), _p(si, C.c_int32), _p(alpha, C.c_float),
+                                  _p(sse, C.c_double), _p(idx, C.c_int32), _p(q, C.c_int8), C.byref(st))
+    return DualResult(alpha, sse, idx, q, None, st.value)
 
 
 def pack_int4(codes_) -> np.ndarray:

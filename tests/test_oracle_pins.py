@@ -299,3 +299,69 @@ def test_compression_ratio_of_resnet50_shape_set_matches_the_paper():
     cr = (packed_bytes + 4 * rows) / (4 * n)           # codes + one fp32 scale per kernel over the fp32 model
     assert float(gold["int4_non_dual_cr_approx"]) <= cr <= float(gold["resnet50_cr_with_dual_layers"]) + 5e-5
     assert cr == pytest.approx(0.12608, abs=1e-5)
+
+
+# ---------------------------------------------------------------- Section 3.5: dual line search (n = 2)
+def test_dual_per_element_enumeration_equals_joint_brute_force():
+    """The third equation of Section 3.5: minimising over the first code with the second one rounded
+    equals minimising over both codes jointly (brute force over all 16 x 16 pairs, float64)."""
+    rng = np.random.default_rng(3)
+    for trial in range(6):
+        x = rng.laplace(0.0, 0.02, 40).astype(np.float32)
+        a1 = np.float32(rng.uniform(0.004, 0.02))
+        a2 = np.float32(a1 * rng.uniform(0.03, 0.3))
+        t = np.arange(-8, 8)[:, None, None]
+        q = np.arange(-8, 8)[None, :, None]
+        err = (x.astype(np.float64)[None, None, :] - np.float64(a1) * t - np.float64(a2) * q) ** 2
+        joint = err.reshape(256, -1).min(axis=0).sum()
+        assert orc.dual_sse_at(x, a1, a2) == pytest.approx(joint, rel=1e-6)
+
+
+def test_dual_recovers_inputs_on_the_joint_grid_exactly():
+    a = 2.0 ** -4
+    rng = np.random.default_rng(9)
+    t = rng.integers(-8, 8, 50)
+    q = rng.integers(-8, 8, 50)
+    t[0], q[0] = -8, -8                              # max|x| = 8a + a/2 = 8.5a
+    x = (t * a + q * (a / 16)).astype(np.float32)
+    # one pair on the grid: alpha1 = hi_frac1*max = a, alpha2 = hi_frac2*alpha1 = a/16
+    r = orc.dual(x, 4, 4, True, 1, 1, hi_frac1=1.0 / 8.5, hi_frac2=1.0 / 16)
+    assert r.alpha[0] == pytest.approx(a, rel=1e-6) and r.alpha[1] == pytest.approx(a / 16, rel=1e-6)
+    if r.alpha[0] == a and r.alpha[1] == a / 16:
+        assert r.sse == 0.0 and np.array_equal(r.codes[0], t) and np.array_equal(r.codes[1], q)
+    assert r.sse <= 1e-12
+
+
+def test_dual_bookkeeping_argmin_and_invariants():
+    x = synth.laplace(147, 0.05, seed=31)
+    r = orc.dual(x, 4, 4, True, 12, 10, 1.0, 0.25, want_curve=True)
+    assert r.best_idx == int(np.argmin(r.sse_curve)) and r.sse == pytest.approx(r.sse_curve[r.best_idx], rel=1e-12)
+    c, d = divmod(r.best_idx, 10)
+    a1, a2 = orc.dual_scales(float(np.max(np.abs(x))), 1.0, 0.25, 12, 10, c, d)
+    assert (a1, a2) == (r.alpha[0], r.alpha[1])
+    m = np.float32(np.max(np.abs(x)))
+    assert a1 == np.float32(c + 1) * (m / np.float32(12)) and a2 == np.float32(d + 1) * (np.float32(0.25) * a1 / np.float32(10))
+    rec = np.float64(a1) * r.codes[0] + np.float64(a2) * r.codes[1]
+    assert r.sse == pytest.approx(np.sum((x.astype(np.float64) - rec) ** 2), rel=1e-12)
+    assert r.codes.min() >= -8 and r.codes.max() <= 7
+    again = orc.dual(x, 4, 4, True, 12, 10, 1.0, 0.25, start_idx=r.best_idx)
+    assert again.sse == r.sse and np.array_equal(again.codes, r.codes)
+    r8 = orc.dual(x * np.float32(4.0), 4, 4, True, 12, 10, 1.0, 0.25)
+    assert np.array_equal(r8.codes, r.codes) and r8.alpha[0] == 4 * r.alpha[0] and r8.sse == pytest.approx(16 * r.sse, rel=1e-12)
+    rows = orc.dual_rows(np.stack([x, -x, x[::-1]]), 4, 4, True, 12, 10, 1.0, 0.25)
+    assert rows.sse[0] == r.sse and np.array_equal(rows.codes[:, 0], r.codes) and rows.alpha[0, 0] == r.alpha[0]
+    z = orc.dual(np.zeros(5, np.float32), 4, 4, True, 4, 4)
+    assert z.best_idx == -1 and z.sse == 0.0 and z.status & orc.STATUS_DEGENERATE
+
+
+def test_dual_beats_the_residual_scheme_at_its_own_scales_and_on_average():
+    """At the residual scheme's (alpha1, alpha2) its codes are one of the choices the enumeration sees,
+    so the dual objective cannot be larger; over a grid it is smaller on average (Section 3.5)."""
+    w = synth.conv_layer(seed=1)[:12]
+    res = orc.residual_rows(w, (4, 4), True, 256, 1.0, 3, 1)
+    gain = []
+    for s in range(12):
+        at = orc.dual_sse_at(w[s], res.alpha[0, s], res.alpha[1, s])
+        assert at <= res.sse[1, s] * (1 + 1e-6)
+        gain.append(res.sse[1, s] / orc.dual(w[s], 4, 4, True, 24, 24, 1.0, 0.25).sse)
+    assert np.mean(gain) > 1.5

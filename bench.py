@@ -297,6 +297,48 @@ class Residual(Workload):
         return sub.size / dt, orc.max_threads(), f"every 64th kernel ({sub.size} elements, {dt:.1f} s)", sub.size
 
 
+class Dual(Workload):
+    """Dual line search (Section 3.5, n = 2) on one convolution-shaped tensor."""
+    kernel = "dual_kernel"
+    instr_per_eval = 7           # per (element, pair, first code): fma, fma, max, min, add, fma, mul+min
+    C1 = C2 = 32
+    HF2 = 0.25
+
+    def __init__(self, name, t):
+        self.name, self.t = name, t
+        self.n_cand = self.C1 * self.C2
+        self.evals_per_element = 1 << BITS          # first codes enumerated per pair
+
+    def setup(self, ctx, torch, dev):
+        s, k = self.t.shape
+        self.host_in = torch.from_numpy(self.t).pin_memory()
+        self.d_t = self.host_in.to(dev)
+        self.out = (torch.empty(2, s, device=dev), torch.empty(s, device=dev),
+                    torch.empty(2, (s * k + 1) // 2, dtype=torch.uint8, device=dev))
+        self.host_out = tuple(t.cpu().pin_memory() for t in self.out)
+        self.n_total = s * k
+        self.h2d, self.d2h = 4 * self.n_total, sum(t.numel() * t.element_size() for t in self.out)
+
+        def step():
+            ctx.omse_dual_quantize(self.d_t, s, k, BITS, BITS, True, self.C1, self.C2, HI_FRAC, self.HF2,
+                                   self.out[0], self.out[1], None, None, self.out[2])
+        self.step = step
+
+    def step_e2e(self):
+        self.d_t.copy_(self.host_in, non_blocking=True)
+        self.step()
+        for t, h in zip(self.out, self.host_out):
+            h.copy_(t, non_blocking=True)
+
+    def cpu(self):
+        from oracle import omse_oracle as orc
+        sub = np.ascontiguousarray(self.t[::32])
+        t0 = time.perf_counter()
+        orc.dual_rows(sub, BITS, BITS, True, self.C1, self.C2, HI_FRAC, self.HF2)
+        dt = time.perf_counter() - t0
+        return sub.size / dt, orc.max_threads(), f"every 32nd kernel ({sub.size} elements, {dt:.1f} s)", sub.size
+
+
 def make_workload(spec: str, rank: int):
     from paper_1902_06822_b200 import synth
     if spec == "c2":
@@ -318,6 +360,9 @@ def make_workload(spec: str, rank: int):
         stride = max(1, w.shape[0] // max(1, (6_000_000 // k)))
         return WeightSet(f"sweep_64M_student_t_K{k}_signed{bits}bit_1024cand_3refine", [w], bits, N_CAND, bits <= 4,
                          stride, f"every {stride}th kernel")
+    if spec == "dual":
+        w = synth.laplace(512 * 4608, 1.0 / np.sqrt(4608.0), 6 + 1000 * rank).reshape(512, 4608)
+        return Dual("dual_line_search_512x4608_conv_signed4bit_x2_32x32_grid_packed", w)
     raise SystemExit(f"unknown workload {spec}")
 
 
@@ -394,7 +439,8 @@ def run_ours(args, rank, world):
         value = whole_job_value(n_total, world, ms, args.steps)
         peak = N_SM * LANES_PER_SM * sm_max_mhz * 1e6                     # FP32 lane-instructions per second
         evals = wl.n_cand * wl.evals_per_element * n_total                 # (element, candidate) evaluations per step
-        achieved = INSTR_PER_EVAL * evals / per_step_s                     # algorithmic instructions per second
+        ipe = getattr(wl, "instr_per_eval", INSTR_PER_EVAL)
+        achieved = ipe * evals / per_step_s                                # algorithmic instructions per second
         out = {
             "metric": "elements quantized/sec (4-bit MMSE search)", "value": value, "unit": "elements/s",
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps,
@@ -410,7 +456,7 @@ def run_ours(args, rank, world):
                          "unit": "T FP32-instr/s", "frac": achieved / peak,
                          "traffic": NCU_TRAFFIC_BYTES if args.workload == "c2" else None,
                          "kernel": wl.kernel, "peak_source": f"148 SMs x 128 lanes x {sm_max_mhz:.0f} MHz ({peak_src} max clock)",
-                         "instr_per_eval": INSTR_PER_EVAL, "evaluations_per_s": evals / per_step_s},
+                         "instr_per_eval": ipe, "evaluations_per_s": evals / per_step_s},
         }
         if world == 1 and not args.no_cpu_baseline:
             v, cores, desc, _ = wl.cpu()
@@ -428,7 +474,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--workload", default="c2",
-                    help="c2 (default: the ResNet-50 weight set the metric is quoted on), c1, c3, c4, c5:K:bits")
+                    help="c2 (default: the ResNet-50 weight set the metric is quoted on), c1, c3, c4, c5:K:bits, dual")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))

@@ -151,6 +151,35 @@ int omse_residual_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, i
                            uint8_t* d_packed);
 
 /*
+ * Dual line search for two quantized tensors (Section 3.5, the special case n = 2, third displayed
+ * equation of the section): T ~ alpha1*Q1 + alpha2*Q2, kernel-wise.  The pair of scales is searched on
+ * a two-dimensional grid; for every pair each element picks its first code by enumerating all of
+ * Z_bits1, the second code being the rounding of the rest,
+ *     min over t in Z_bits1 of ( T_j - alpha1*t - alpha2*[ (T_j - alpha1*t)/alpha2 ]_Z_bits2 )^2,
+ * decided in binary32 (fused multiply-adds, IEEE division, lowest t on equal errors).  The paper gives
+ * no grid; this library's is alpha1_c = (c+1)/n_cand1 * hi_frac1 * max|T_k| and, for each alpha1,
+ * alpha2_d = (d+1)/n_cand2 * hi_frac2 * alpha1_c, in the binary32 form of omse_grid.  The pair with
+ * the smallest error wins, lowest c*n_cand2+d among equal errors; there is no polish step.
+ * The cost is n_cand1*n_cand2*2^bits1 evaluations per element: meant for small tensors (Section 3.5).
+ * Outputs: d_alpha [2][n_kernels], d_sse [n_kernels] (binary64 accumulation of the objective),
+ * d_best_idx [n_kernels] (nullable; -1 for a degenerate kernel), d_codes [2][n_kernels*kernel_len]
+ * (nullable), d_packed [2][ceil(n_kernels*kernel_len/2)] (nullable; needs bits1, bits2 <= 4).
+ * Limits: 1 <= n_cand1, n_cand2 <= OMSE_DUAL_MAX_CANDIDATES; bits1, bits2 in 2..8;
+ * 1 <= kernel_len <= OMSE_MAX_KERNEL_LEN.
+ */
+#define OMSE_DUAL_MAX_CANDIDATES 1024
+typedef struct {
+    int32_t n_cand1, n_cand2;
+    float hi_frac1; /* alpha1 grid reaches hi_frac1 * max|T_k|  */
+    float hi_frac2; /* alpha2 grid reaches hi_frac2 * alpha1     */
+} omse_dual_grid;
+
+int omse_dual_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, int64_t kernel_len,
+                       int bits1, int bits2, int is_signed, const omse_dual_grid* grid,
+                       float* d_alpha, float* d_sse, int32_t* d_best_idx, int8_t* d_codes,
+                       uint8_t* d_packed);
+
+/*
  * INT4 code emission.  The paper deploys INT4 tensors but fixes no byte layout; this library's is:
  * element e (flat index) goes to byte e/2, even e in bits 0-3 and odd e in bits 4-7, the nibble
  * being the low four bits of the two's-complement code; if n is odd, bits 4-7 of the last byte are 0.

@@ -21,7 +21,7 @@ STATIC_MAX_CANDIDATES = 2048
 
 EXPORTS = [
     "omse_create", "omse_destroy", "omse_set_stream", "omse_workspace_bytes", "omse_quantize_weights",
-    "omse_quantize_weights_batched",
+    "omse_quantize_weights_batched", "omse_dual_quantize",
     "omse_activation_scale", "omse_residual_quantize", "omse_pack_int4", "omse_last_device_status",
     "omse_status_string", "omse_activation_scale_static",
 ]
@@ -34,6 +34,10 @@ class OmseGrid(C.Structure):
 class OmseWeightTensor(C.Structure):
     _fields_ = [("d_w", C.c_void_p), ("n_kernels", C.c_int64), ("kernel_len", C.c_int64), ("d_alpha", C.c_void_p),
                 ("d_sse", C.c_void_p), ("d_best_idx", C.c_void_p), ("d_codes", C.c_void_p), ("d_packed", C.c_void_p)]
+
+
+class OmseDualGrid(C.Structure):
+    _fields_ = [("n_cand1", C.c_int32), ("n_cand2", C.c_int32), ("hi_frac1", C.c_float), ("hi_frac2", C.c_float)]
 
 
 class OmseError(RuntimeError):
@@ -65,6 +69,7 @@ def load_library() -> C.CDLL:
     lib.omse_residual_quantize.argtypes = [vp, vp, i64, i64, C.POINTER(C.c_int), i32, C.POINTER(OmseGrid), i32, i32,
                                            vp, vp, vp, vp]
     lib.omse_pack_int4.argtypes = [vp, vp, i64, i32, vp]
+    lib.omse_dual_quantize.argtypes = [vp, vp, i64, i64, i32, i32, i32, C.POINTER(OmseDualGrid), vp, vp, vp, vp, vp]
     lib.omse_activation_scale_static.argtypes = [i32, vp, vp, i64, i32, i32, C.POINTER(OmseGrid), vp, vp, vp, vp, vp]
     lib.omse_last_device_status.argtypes = [vp, C.POINTER(C.c_uint32)]
     lib.omse_status_string.argtypes = [i32]
@@ -190,6 +195,16 @@ class Context:
             _ptr(packed, torch.uint8))
         if rc != OK:
             raise OmseError(rc, "omse_residual_quantize")
+
+    def omse_dual_quantize(self, t, n_kernels, kernel_len, bits1, bits2, is_signed, n_cand1, n_cand2, hi_frac1,
+                           hi_frac2, alpha, sse, best_idx=None, codes=None, packed=None):
+        g = OmseDualGrid(n_cand1, n_cand2, hi_frac1, hi_frac2)
+        rc = load_library().omse_dual_quantize(
+            self._h, _ptr(t, torch.float32), n_kernels, kernel_len, bits1, bits2, int(is_signed), C.byref(g),
+            _ptr(alpha, torch.float32), _ptr(sse, torch.float32), _ptr(best_idx, torch.int32),
+            _ptr(codes, torch.int8), _ptr(packed, torch.uint8))
+        if rc != OK:
+            raise OmseError(rc, "omse_dual_quantize")
 
     def omse_pack_int4(self, codes, n, is_signed, packed):
         rc = load_library().omse_pack_int4(self._h, _ptr(codes, torch.int8), n, int(is_signed), _ptr(packed, torch.uint8))

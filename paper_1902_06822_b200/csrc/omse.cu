@@ -32,6 +32,7 @@
 
 #include "omse_rows.cuh"
 #include "omse_tensor.cuh"
+#include "omse_dual.cuh"
 
 namespace {
 
@@ -403,6 +404,59 @@ int omse_residual_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, i
     for (int j = 0; j < n_tensors; ++j) bounds(bits[j], is_signed, &a.lo[j], &a.hi[j]);
     a.keep_x0 = n_sweeps > 1 ? 1 : 0;
     return launch_rows(ctx, a, kernel_len);
+}
+
+int omse_dual_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, int64_t kernel_len, int bits1, int bits2,
+                       int is_signed, const omse_dual_grid* grid, float* d_alpha, float* d_sse, int32_t* d_best_idx,
+                       int8_t* d_codes, uint8_t* d_packed) {
+    if (!ctx || !grid || grid->n_cand1 < 1 || grid->n_cand2 < 1 || grid->n_cand1 > OMSE_DUAL_MAX_CANDIDATES ||
+        grid->n_cand2 > OMSE_DUAL_MAX_CANDIDATES || !(grid->hi_frac1 > 0.f) || !(grid->hi_frac2 > 0.f) ||
+        !(grid->hi_frac1 <= 3.0e38f) || !(grid->hi_frac2 <= 3.0e38f) || bits1 < 2 || bits1 > 8 || bits2 < 2 ||
+        bits2 > 8 || n_kernels < 0 || kernel_len < 1 || kernel_len > OMSE_MAX_KERNEL_LEN || n_kernels > (int64_t)1 << 40)
+        return OMSE_EINVAL;
+    if (d_packed && (bits1 > 4 || bits2 > 4)) return OMSE_EINVAL;
+    if (n_kernels == 0) return OMSE_OK;
+    if (!d_t || !d_alpha || !d_sse) return OMSE_EINVAL;
+    if (misaligned4(d_t) || misaligned4(d_alpha) || misaligned4(d_sse) || misaligned4(d_best_idx)) return OMSE_EINVAL;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return OMSE_ECUDA;
+    omse::DualArgs a;
+    memset(&a, 0, sizeof(a));
+    a.t = d_t;
+    a.S = n_kernels;
+    a.K = kernel_len;
+    a.n_cand1 = grid->n_cand1;
+    a.n_cand2 = grid->n_cand2;
+    a.hi_frac1 = grid->hi_frac1;
+    a.hi_frac2 = grid->hi_frac2;
+    bounds(bits1, is_signed, &a.lo1, &a.hi1);
+    bounds(bits2, is_signed, &a.lo2, &a.hi2);
+    a.alpha = d_alpha;
+    a.sse = d_sse;
+    a.best_idx = d_best_idx;
+    a.codes = reinterpret_cast<signed char*>(d_codes);
+    a.packed = d_packed;
+    a.status = &ctx->ws->status;
+    a.rows_per_unit = (d_packed && (kernel_len & 1)) ? 2 : 1;
+    const size_t smem = (size_t)((kernel_len + 3) & ~3ll) * 4 + 64 * 8 + omse::kDualListCap * 4 + 4 * 4;
+    static bool attr_set[64] = {};
+    if (!attr_set[ctx->device & 63]) {
+        if (cudaFuncSetAttribute(omse::dual_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess)
+            return OMSE_ECUDA;
+        attr_set[ctx->device & 63] = true;
+    }
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, omse::dual_kernel, omse::kDualThreads, smem) != cudaSuccess || occ < 1)
+        return OMSE_ECUDA;
+    const long long n_units = (n_kernels + a.rows_per_unit - 1) / a.rows_per_unit;
+    long long blocks = (long long)ctx->n_sm * occ;
+    if (blocks > n_units) blocks = n_units;
+    // every block keeps the fp32 grid of its current row in the context workspace
+    const long long cap = (long long)(kPartialBytes / ((size_t)grid->n_cand1 * grid->n_cand2 * 4));
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) return OMSE_EINVAL;
+    a.curve = reinterpret_cast<float*>(ctx->partials);
+    omse::dual_kernel<<<(unsigned)blocks, omse::kDualThreads, smem, ctx->stream>>>(a);
+    return cudaGetLastError() == cudaSuccess ? OMSE_OK : OMSE_ECUDA;
 }
 
 int omse_activation_scale(omse_ctx* ctx, const float* d_x, int64_t n, int bits, int is_signed, const omse_grid* grid,

@@ -54,3 +54,19 @@ def residual_quantize(t, bits=(4, 4), signed=True, n_cand=1024, hi_frac=1.0, ref
     torch.cuda.synchronize()
     return (alpha.cpu().numpy(), sse.cpu().numpy(), None if codes is None else codes.cpu().numpy(),
             None if packed is None else packed.cpu().numpy())
+
+
+def dual_quantize(t, bits1=4, bits2=4, signed=True, n_cand1=32, n_cand2=32, hi_frac1=1.0, hi_frac2=0.25,
+                  want_codes=True, want_packed=False):
+    S, K = t.shape
+    d_t = torch.from_numpy(np.ascontiguousarray(t)).cuda()
+    alpha = torch.full((2, S), -1.0, dtype=torch.float32, device="cuda")
+    sse = torch.full((S,), -1.0, dtype=torch.float32, device="cuda")
+    idx = torch.full((S,), -7, dtype=torch.int32, device="cuda")
+    codes = torch.full((2, S * K), 99, dtype=torch.int8, device="cuda") if want_codes else None
+    packed = torch.full((2, (S * K + 1) // 2), 0xAB, dtype=torch.uint8, device="cuda") if want_packed else None
+    ctx().omse_dual_quantize(d_t, S, K, bits1, bits2, signed, n_cand1, n_cand2, hi_frac1, hi_frac2, alpha, sse, idx,
+                             codes, packed)
+    torch.cuda.synchronize()
+    return (alpha.cpu().numpy(), sse.cpu().numpy(), idx.cpu().numpy(),
+            None if codes is None else codes.cpu().numpy(), None if packed is None else packed.cpu().numpy())

@@ -180,6 +180,31 @@ int omse_dual_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, int64
                        uint8_t* d_packed);
 
 /*
+ * Key layers (Section 3.5): "quantized layers with high MSE, or MSE bigger than some threshold tau" get a
+ * second quantized tensor.  For each layer l this call sums the per-kernel squared errors that
+ * omse_quantize_weights wrote (d_sse, [n_kernels] float) in binary64 in a fixed order, divides by the
+ * layer's element count and compares with tau: d_mse[l] = sum / (n_kernels*kernel_len),
+ * d_is_key[l] = (d_mse[l] > tau).  `layers` is a HOST array read before the call returns; d_mse
+ * [n_layers] double and d_is_key [n_layers] int32 (nullable) are device buffers.
+ * 0 <= n_layers <= OMSE_MAX_BATCH, tau >= 0.
+ */
+typedef struct {
+    const float* d_sse;
+    int64_t n_kernels, kernel_len;
+} omse_layer_error;
+
+int omse_select_key_layers(omse_ctx* ctx, const omse_layer_error* layers, int n_layers, float tau,
+                           double* d_mse, int32_t* d_is_key);
+
+/*
+ * Compression ratio (Section 3.5): size of the quantized model - bits[l] per code and one binary32
+ * scale per kernel, times n_tensors[l] quantized tensors - over the size of the binary32 model.
+ * Host arithmetic on HOST arrays of n_layers entries; returns -1 on invalid arguments.
+ */
+double omse_compression_ratio(const int64_t* n_kernels, const int64_t* kernel_len, const int* bits,
+                              const int* n_tensors, int n_layers);
+
+/*
  * INT4 code emission.  The paper deploys INT4 tensors but fixes no byte layout; this library's is:
  * element e (flat index) goes to byte e/2, even e in bits 0-3 and odd e in bits 4-7, the nibble
  * being the low four bits of the two's-complement code; if n is odd, bits 4-7 of the last byte are 0.

@@ -455,6 +455,30 @@ void omse_oracle_dual_rows(const float *t, int64_t n_kernels, int64_t kernel_len
     *status |= st_all;
 }
 
+/* Key layers (Section 3.5): a layer is a key layer when its MSE exceeds a threshold tau.  The MSE of a
+ * layer is the sum of its kernels' squared errors over its number of elements (Section 3.2 drops the
+ * mean factor inside the analysis; the threshold values the paper quotes, e.g. 8e-5, are per element). */
+double omse_oracle_layer_mse(const float *sse, int64_t n_kernels, int64_t kernel_len)
+{
+    double s = 0.0;
+    for (int64_t i = 0; i < n_kernels; ++i) s += (double)sse[i];
+    return s / ((double)n_kernels * (double)kernel_len);
+}
+
+/* Compression ratio (Section 3.5): size of the quantized model (codes and one binary32 scale per
+ * kernel and per quantized tensor) over the size of the binary32 model. */
+double omse_oracle_compression_ratio(const int64_t *n_kernels, const int64_t *kernel_len, const int *bits,
+                                     const int *n_tensors, int n_layers)
+{
+    double q = 0.0, f = 0.0;
+    for (int l = 0; l < n_layers; ++l) {
+        double n = (double)n_kernels[l] * (double)kernel_len[l];
+        q += (double)n_tensors[l] * (n * bits[l] + 32.0 * (double)n_kernels[l]);
+        f += 32.0 * n;
+    }
+    return q / f;
+}
+
 /* INT4 code emission.  The paper fixes no byte layout; this library's layout is: element e
  * (flat, row-major) goes to byte e/2, even e in bits 0-3, odd e in bits 4-7, the nibble being
  * the low four bits of the two's-complement code; a trailing odd element leaves bits 4-7 zero. */

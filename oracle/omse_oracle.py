@@ -63,6 +63,11 @@ def _load():
                                      C.c_float, C.c_int, f32p, f64p, i32p, i8p, i8p, f64p, u32p]
     lib.omse_oracle_dual_rows.argtypes = [f32p, C.c_int64, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
                                           C.c_float, C.c_float, i32p, f32p, f64p, i32p, i8p, u32p]
+    lib.omse_oracle_layer_mse.restype = C.c_double
+    lib.omse_oracle_layer_mse.argtypes = [f32p, C.c_int64, C.c_int64]
+    lib.omse_oracle_compression_ratio.restype = C.c_double
+    lib.omse_oracle_compression_ratio.argtypes = [C.POINTER(C.c_int64), C.POINTER(C.c_int64), C.POINTER(C.c_int),
+                                                  C.POINTER(C.c_int), C.c_int]
     lib.omse_oracle_pack_int4.argtypes = [i8p, C.c_int64, u8p]
     lib.omse_oracle_unpack_int4.argtypes = [u8p, C.c_int64, C.c_int, i8p]
     _lib = lib
@@ -250,6 +255,21 @@ def dual_rows(t, bits1=4, bits2=4, is_signed=True, n_cand1=32, n_cand2=32, hi_fr
                                   _c32(hi_frac1), _c32(hi_frac2), _p(si, C.c_int32), _p(alpha, C.c_float),
                                   _p(sse, C.c_double), _p(idx, C.c_int32), _p(q, C.c_int8), C.byref(st))
     return DualResult(alpha, sse, idx, q, None, st.value)
+
+
+def layer_mse(sse, kernel_len: int) -> float:
+    """Section 3.5: MSE of a layer from its kernels' squared errors (fp32 values as the library outputs them)."""
+    e = _f32(sse).ravel()
+    return float(_load().omse_oracle_layer_mse(_p(e, C.c_float), e.size, kernel_len))
+
+
+def compression_ratio(n_kernels, kernel_len, bits, n_tensors) -> float:
+    n = len(n_kernels)
+    a = (C.c_int64 * n)(*n_kernels)
+    b = (C.c_int64 * n)(*kernel_len)
+    c = (C.c_int * n)(*bits)
+    d = (C.c_int * n)(*n_tensors)
+    return float(_load().omse_oracle_compression_ratio(a, b, c, d, n))
 
 
 def pack_int4(codes_) -> np.ndarray:

@@ -21,7 +21,7 @@ STATIC_MAX_CANDIDATES = 2048
 
 EXPORTS = [
     "omse_create", "omse_destroy", "omse_set_stream", "omse_workspace_bytes", "omse_quantize_weights",
-    "omse_quantize_weights_batched", "omse_dual_quantize",
+    "omse_quantize_weights_batched", "omse_dual_quantize", "omse_select_key_layers", "omse_compression_ratio",
     "omse_activation_scale", "omse_residual_quantize", "omse_pack_int4", "omse_last_device_status",
     "omse_status_string", "omse_activation_scale_static",
 ]
@@ -38,6 +38,10 @@ class OmseWeightTensor(C.Structure):
 
 class OmseDualGrid(C.Structure):
     _fields_ = [("n_cand1", C.c_int32), ("n_cand2", C.c_int32), ("hi_frac1", C.c_float), ("hi_frac2", C.c_float)]
+
+
+class OmseLayerError(C.Structure):
+    _fields_ = [("d_sse", C.c_void_p), ("n_kernels", C.c_int64), ("kernel_len", C.c_int64)]
 
 
 class OmseError(RuntimeError):
@@ -69,6 +73,9 @@ def load_library() -> C.CDLL:
     lib.omse_residual_quantize.argtypes = [vp, vp, i64, i64, C.POINTER(C.c_int), i32, C.POINTER(OmseGrid), i32, i32,
                                            vp, vp, vp, vp]
     lib.omse_pack_int4.argtypes = [vp, vp, i64, i32, vp]
+    lib.omse_select_key_layers.argtypes = [vp, C.POINTER(OmseLayerError), i32, C.c_float, vp, vp]
+    lib.omse_compression_ratio.argtypes = [C.POINTER(i64), C.POINTER(i64), C.POINTER(i32), C.POINTER(i32), i32]
+    lib.omse_compression_ratio.restype = C.c_double
     lib.omse_dual_quantize.argtypes = [vp, vp, i64, i64, i32, i32, i32, C.POINTER(OmseDualGrid), vp, vp, vp, vp, vp]
     lib.omse_activation_scale_static.argtypes = [i32, vp, vp, i64, i32, i32, C.POINTER(OmseGrid), vp, vp, vp, vp, vp]
     lib.omse_last_device_status.argtypes = [vp, C.POINTER(C.c_uint32)]
@@ -111,6 +118,13 @@ def omse_activation_scale_static(x, n, bits, is_signed, n_cand, hi_frac, refine_
         _ptr(sse_curve, torch.float64), _ptr(status, torch.int32))
     if rc != OK:
         raise OmseError(rc, "omse_activation_scale_static")
+
+
+def omse_compression_ratio(n_kernels, kernel_len, bits, n_tensors) -> float:
+    """Section 3.5 compression ratio of a set of layers (host arithmetic)."""
+    n = len(n_kernels)
+    return float(load_library().omse_compression_ratio((C.c_int64 * n)(*n_kernels), (C.c_int64 * n)(*kernel_len),
+                                                       (C.c_int * n)(*bits), (C.c_int * n)(*n_tensors), n))
 
 
 class Context:
@@ -205,6 +219,16 @@ class Context:
             _ptr(codes, torch.int8), _ptr(packed, torch.uint8))
         if rc != OK:
             raise OmseError(rc, "omse_dual_quantize")
+
+    def omse_select_key_layers(self, layers, tau, mse, is_key=None):
+        """layers: sequence of (sse tensor, n_kernels, kernel_len); mse: float64 [n]; is_key: int32 [n]."""
+        arr = (OmseLayerError * len(layers))()
+        for d, (sse, s, k) in zip(arr, layers):
+            d.d_sse, d.n_kernels, d.kernel_len = _ptr(sse, torch.float32), s, k
+        rc = load_library().omse_select_key_layers(self._h, arr, len(layers), tau, _ptr(mse, torch.float64),
+                                                   _ptr(is_key, torch.int32))
+        if rc != OK:
+            raise OmseError(rc, "omse_select_key_layers")
 
     def omse_pack_int4(self, codes, n, is_signed, packed):
         rc = load_library().omse_pack_int4(self._h, _ptr(codes, torch.int8), n, int(is_signed), _ptr(packed, torch.uint8))

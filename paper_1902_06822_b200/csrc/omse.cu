@@ -459,6 +459,43 @@ int omse_dual_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, int64
     return cudaGetLastError() == cudaSuccess ? OMSE_OK : OMSE_ECUDA;
 }
 
+int omse_select_key_layers(omse_ctx* ctx, const omse_layer_error* layers, int n_layers, float tau, double* d_mse,
+                           int32_t* d_is_key) {
+    if (!ctx || n_layers < 0 || n_layers > OMSE_MAX_BATCH || (n_layers > 0 && (!layers || !d_mse)) || !(tau >= 0.f))
+        return OMSE_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(d_mse) & 7) || misaligned4(d_is_key)) return OMSE_EINVAL;
+    static_assert(sizeof(omse::LayerError) <= sizeof(omse::RowTensor), "descriptor buffer too small");
+    std::vector<omse::LayerError> list((size_t)n_layers);
+    for (int i = 0; i < n_layers; ++i) {
+        if (!layers[i].d_sse || layers[i].n_kernels < 1 || layers[i].kernel_len < 1 || misaligned4(layers[i].d_sse))
+            return OMSE_EINVAL;
+        list[i].sse = layers[i].d_sse;
+        list[i].n_kernels = layers[i].n_kernels;
+        list[i].kernel_len = layers[i].kernel_len;
+    }
+    if (n_layers == 0) return OMSE_OK;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return OMSE_ECUDA;
+    omse::LayerError* d_layers = reinterpret_cast<omse::LayerError*>(ctx->d_tensors);
+    if (cudaMemcpyAsync(d_layers, list.data(), sizeof(omse::LayerError) * list.size(), cudaMemcpyHostToDevice,
+                        ctx->stream) != cudaSuccess)
+        return OMSE_ECUDA;
+    omse::layer_mse_kernel<<<(unsigned)n_layers, 256, 0, ctx->stream>>>(d_layers, tau, d_mse, d_is_key);
+    return cudaGetLastError() == cudaSuccess ? OMSE_OK : OMSE_ECUDA;
+}
+
+double omse_compression_ratio(const int64_t* n_kernels, const int64_t* kernel_len, const int* bits, const int* n_tensors,
+                              int n_layers) {
+    if (!n_kernels || !kernel_len || !bits || !n_tensors || n_layers < 1) return -1.0;
+    double q = 0.0, f = 0.0;
+    for (int l = 0; l < n_layers; ++l) {
+        if (n_kernels[l] < 0 || kernel_len[l] < 1 || bits[l] < 1 || n_tensors[l] < 1) return -1.0;
+        const double n = (double)n_kernels[l] * (double)kernel_len[l];
+        q += (double)n_tensors[l] * (n * (double)bits[l] + 32.0 * (double)n_kernels[l]);
+        f += 32.0 * n;
+    }
+    return f > 0.0 ? q / f : -1.0;
+}
+
 int omse_activation_scale(omse_ctx* ctx, const float* d_x, int64_t n, int bits, int is_signed, const omse_grid* grid,
                           float* d_alpha, float* d_sse, int32_t* d_best_idx, double* d_sse_curve) {
     if (!ctx || !grid_ok(grid) || bits < 2 || bits > 8 || n < 0 || !d_alpha || !d_sse) return OMSE_EINVAL;

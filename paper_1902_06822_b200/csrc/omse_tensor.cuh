@@ -449,6 +449,28 @@ __global__ void __launch_bounds__(256) tensor_pass_kernel(const TensorArgs a) {
     }
 }
 
+// Key layers (Section 3.5): MSE of each layer = sum of its kernels' squared errors / elements, compared
+// with the threshold tau.  One block per layer, fixed-order sum in fp64.
+struct LayerError {
+    const float* sse;        // [n_kernels] squared error per kernel, as the quantize calls output it
+    long long n_kernels, kernel_len;
+};
+
+__global__ void __launch_bounds__(256) layer_mse_kernel(const LayerError* __restrict__ layers, float tau,
+                                                         double* __restrict__ mse, int* __restrict__ is_key) {
+    __shared__ double scratch[64];
+    const LayerError L = layers[blockIdx.x];
+    double s = 0.0;
+    for (long long i = threadIdx.x; i < L.n_kernels; i += blockDim.x) s += (double)L.sse[i];
+    long long zero = 0;
+    block_sum2(s, zero, scratch);
+    if (threadIdx.x == 0) {
+        const double m = s / ((double)L.n_kernels * (double)L.kernel_len);
+        mse[blockIdx.x] = m;
+        if (is_key) is_key[blockIdx.x] = m > (double)tau ? 1 : 0;
+    }
+}
+
 // INT4 emission: byte e/2 holds element e (even) in bits 0-3 and element e+1 in bits 4-7.
 __global__ void __launch_bounds__(256) pack_int4_kernel(const signed char* __restrict__ codes, long long n,
                                                          unsigned char* __restrict__ packed) {

@@ -365,3 +365,26 @@ def test_dual_beats_the_residual_scheme_at_its_own_scales_and_on_average():
         assert at <= res.sse[1, s] * (1 + 1e-6)
         gain.append(res.sse[1, s] / orc.dual(w[s], 4, 4, True, 24, 24, 1.0, 0.25).sse)
     assert np.mean(gain) > 1.5
+
+
+# ---------------------------------------------------------------- Section 3.5: key layers, compression ratio
+def test_layer_mse_and_compression_ratio_by_hand():
+    # two kernels of three weights with squared errors 0.03 and 0.09: MSE = 0.12 / 6 = 0.02
+    assert orc.layer_mse(np.array([0.03, 0.09], np.float32), 3) == pytest.approx(0.02, rel=1e-6)
+    # one layer of 10 kernels x 100 weights at 4 bits: (1000*4 + 10*32) / (1000*32) = 0.135
+    assert orc.compression_ratio([10], [100], [4], [1]) == pytest.approx(0.135)
+    # the same layer with two quantized tensors costs twice as much; mixed with a plain layer of equal size
+    assert orc.compression_ratio([10, 10], [100, 100], [4, 4], [2, 1]) == pytest.approx(3 * 4320 / 64000)
+    shapes = synth.resnet50_shapes()
+    ks, ls = [s for _, s, k in shapes], [k for _, s, k in shapes]
+    plain = orc.compression_ratio(ks, ls, [4] * 54, [1] * 54)
+    assert plain == pytest.approx(0.12608, abs=1e-5)
+    # Section 3.5, Table 3: ResNet-50 with its dual layers reads 0.1261; Table 6 reports 3.7 % dual layers = 2 of 54.
+    # Doubling the two smallest layers moves the ratio by < 1e-4, doubling the two largest by ~0.02.
+    order = np.argsort([s * k for _, s, k in shapes])
+    nt = np.ones(54, int)
+    nt[order[:2]] = 2
+    assert orc.compression_ratio(ks, ls, [4] * 54, nt.tolist()) - plain < 1e-4
+    nt = np.ones(54, int)
+    nt[order[-2:]] = 2
+    assert 0.01 < orc.compression_ratio(ks, ls, [4] * 54, nt.tolist()) - plain < 0.03

@@ -279,3 +279,36 @@ def test_residual_on_regrouped_long_rows(gpu):
     ref = orc.residual_rows(t, (4, 3), True, 512, 1.0, 2, n_sweeps=2)
     np.testing.assert_allclose(alpha, ref.alpha, rtol=RTOL)
     np.testing.assert_allclose(sse, ref.sse, rtol=RTOL)
+
+
+# ---------------------------------------------------------------- seeded random configurations
+@pytest.mark.parametrize("seed", range(24))
+def test_random_configurations(gpu, seed):
+    """Random shapes, grids, bit widths and value distributions (seeded): every launch path gets hit."""
+    rng = np.random.default_rng(1000 + seed)
+    k = int(rng.choice([3, 17, 27, 64, 100, 147, 200, 333, 576, 640, 641, 1023, 1024, 2000, 4608, 9000]))
+    max_rows = max(2, min(4000, 600_000 // k))
+    s = int(rng.integers(1, max_rows))
+    n_cand = int(rng.choice([7, 32, 50, 64, 128, 256, 500, 1024, 1024, 1024, 2048, 4096]))
+    bits = int(rng.choice([2, 3, 4, 4, 8]))
+    signed = bool(rng.integers(0, 2))
+    refine = int(rng.integers(0, 4))
+    hi_frac = float(rng.choice([1.0, 1.0, 0.5, 1.0 / 7, 1.5]))
+    kind = int(rng.integers(0, 4))
+    if kind == 0:
+        w = synth.laplace(s * k, 0.02, seed=2000 + seed).reshape(s, k)
+    elif kind == 1:
+        w = synth.student_t3(s * k, seed=2000 + seed).reshape(s, k)
+    elif kind == 2:
+        w = synth.relu_activations(s * k, seed=2000 + seed, zero_prob=0.6).reshape(s, k)
+    else:
+        w = synth.laplace_with_outliers(s * k, 0.005, seed=2000 + seed, outlier_prob=0.01).reshape(s, k)
+    if not signed and kind != 2 and seed % 2:
+        w = np.abs(w)
+    packed = bits <= 4
+    rows = None if s * k * n_cand < 3e8 else np.unique(rng.integers(0, s, 300))
+    alpha, sse, idx, q, pk = gpu.quantize_weights(w, bits, signed, n_cand, hi_frac, refine, True, packed)
+    st = check_rows(w, alpha, sse, idx, q, pk if rows is None else None, bits, signed, n_cand, hi_frac, refine, rows=rows)
+    assert st["idx_diff"] <= max(1, st["rows"] // 50) and st["alpha_bitwise"] >= 0.98, st
+    if pk is not None:
+        assert np.array_equal(pk, orc.pack_int4(q))

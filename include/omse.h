@@ -151,6 +151,19 @@ int omse_residual_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, i
                            uint8_t* d_packed);
 
 /*
+ * omse_residual_quantize with one signedness flag per quantized tensor and the convergence history of
+ * Algorithm 1 (Section 3.5: "until convergence").  is_signed: HOST array [n_tensors] (a non-negative
+ * tensor may take an unsigned first tensor and a signed tensor for its residual, whose rounding errors
+ * have both signs).  d_sse_history (nullable): [n_sweeps][n_tensors][n_kernels] float, the squared
+ * error after every update, in the order the updates are made; its last [n_tensors][n_kernels] block
+ * equals d_sse.  Everything else as in omse_residual_quantize.
+ */
+int omse_alg1_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, int64_t kernel_len,
+                       const int* bits, const int* is_signed, const omse_grid* grid, int n_tensors,
+                       int n_sweeps, float* d_alpha, float* d_sse, float* d_sse_history,
+                       int8_t* d_codes, uint8_t* d_packed);
+
+/*
  * Dual line search for two quantized tensors (Section 3.5, the special case n = 2, third displayed
  * equation of the section): T ~ alpha1*Q1 + alpha2*Q2, kernel-wise.  The pair of scales is searched on
  * a two-dimensional grid; for every pair each element picks its first code by enumerating all of

@@ -256,11 +256,13 @@ void omse_oracle_activation_scale(const float *x, int64_t n, int bits, int is_si
  * Outputs (last sweep): alpha[n], sse[n] (error after tensors 1..j were updated),
  * best_idx[n], codes[n][k]; r_scratch[k] is caller-provided scratch.
  */
-static void alg1_segment(const float *x, int64_t k, const int *bits, int is_signed, int n_cand,
+static void alg1_segment(const float *x, int64_t k, const int *bits, const int *is_signed, int n_cand,
                          float hi_frac, int refine_iters, int n_tensors, int n_sweeps,
                          int64_t out_stride, float *alpha, double *sse, int32_t *best_idx,
-                         int8_t *codes, int64_t code_stride, float *r, uint32_t *status)
-{
+                         int8_t *codes, int64_t code_stride, float *r, double *sse_sweeps,
+                         uint32_t *status)
+{   /* is_signed: one flag per quantized tensor; sse_sweeps (nullable): [n_sweeps][n_tensors] with stride
+     * out_stride, the error after every update, i.e. the convergence history of the while-loop */
     for (int j = 0; j < n_tensors; ++j) {
         alpha[j * out_stride] = 0.0f;
         memset(codes + j * code_stride, 0, (size_t)k);
@@ -275,18 +277,21 @@ static void alg1_segment(const float *x, int64_t k, const int *bits, int is_sign
                 r[e] = v;
             }
             double s_j;
-            omse_oracle_phi(r, k, bits[j], is_signed, n_cand, hi_frac, refine_iters, -1,
+            omse_oracle_phi(r, k, bits[j], is_signed[j], n_cand, hi_frac, refine_iters, -1,
                             &alpha[j * out_stride], &s_j, &best_idx[j * out_stride],
                             codes + j * code_stride, NULL, status);
             sse[j * out_stride] = s_j;
+            if (sse_sweeps) sse_sweeps[((int64_t)sweep * n_tensors + j) * out_stride] = s_j;
         }
     }
 }
 
-void omse_oracle_residual_rows(const float *t, int64_t n_kernels, int64_t kernel_len,
-                               const int *bits, int is_signed, int n_cand, float hi_frac,
-                               int refine_iters, int n_tensors, int n_sweeps, float *alpha,
-                               double *sse, int32_t *best_idx, int8_t *codes, uint32_t *status)
+/* Algorithm 1 kernel-wise with one signedness flag per quantized tensor and the error after every
+ * update: sse_sweeps (nullable) is [n_sweeps][n_tensors][n_kernels]. */
+void omse_oracle_alg1_rows(const float *t, int64_t n_kernels, int64_t kernel_len, const int *bits,
+                           const int *is_signed, int n_cand, float hi_frac, int refine_iters,
+                           int n_tensors, int n_sweeps, float *alpha, double *sse, int32_t *best_idx,
+                           int8_t *codes, double *sse_sweeps, uint32_t *status)
 {
     /* layouts: alpha/sse/best_idx [n_tensors][n_kernels]; codes [n_tensors][n_kernels*kernel_len] */
     int64_t n = n_kernels * kernel_len;
@@ -299,11 +304,22 @@ void omse_oracle_residual_rows(const float *t, int64_t n_kernels, int64_t kernel
         float *r = (float *)malloc(sizeof(float) * (size_t)kernel_len);
         alg1_segment(t + s * kernel_len, kernel_len, bits, is_signed, n_cand, hi_frac, refine_iters,
                      n_tensors, n_sweeps, n_kernels, alpha + s, sse + s, best_idx + s,
-                     codes + s * kernel_len, n, r, &st);
+                     codes + s * kernel_len, n, r, sse_sweeps ? sse_sweeps + s : NULL, &st);
         free(r);
         st_all |= st;
     }
     *status |= st_all;
+}
+
+void omse_oracle_residual_rows(const float *t, int64_t n_kernels, int64_t kernel_len,
+                               const int *bits, int is_signed, int n_cand, float hi_frac,
+                               int refine_iters, int n_tensors, int n_sweeps, float *alpha,
+                               double *sse, int32_t *best_idx, int8_t *codes, uint32_t *status)
+{
+    int flags[16];
+    for (int j = 0; j < n_tensors && j < 16; ++j) flags[j] = is_signed;
+    omse_oracle_alg1_rows(t, n_kernels, kernel_len, bits, flags, n_cand, hi_frac, refine_iters, n_tensors,
+                          n_sweeps, alpha, sse, best_idx, codes, NULL, status);
 }
 
 /*

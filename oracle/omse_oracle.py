@@ -68,6 +68,8 @@ def _load():
     lib.omse_oracle_compression_ratio.restype = C.c_double
     lib.omse_oracle_compression_ratio.argtypes = [C.POINTER(C.c_int64), C.POINTER(C.c_int64), C.POINTER(C.c_int),
                                                   C.POINTER(C.c_int), C.c_int]
+    lib.omse_oracle_alg1_rows.argtypes = [f32p, C.c_int64, C.c_int64, C.POINTER(C.c_int), C.POINTER(C.c_int), C.c_int,
+                                          C.c_float, C.c_int, C.c_int, C.c_int, f32p, f64p, i32p, i8p, f64p, u32p]
     lib.omse_oracle_pack_int4.argtypes = [i8p, C.c_int64, u8p]
     lib.omse_oracle_unpack_int4.argtypes = [u8p, C.c_int64, C.c_int, i8p]
     _lib = lib
@@ -270,6 +272,26 @@ def compression_ratio(n_kernels, kernel_len, bits, n_tensors) -> float:
     c = (C.c_int * n)(*bits)
     d = (C.c_int * n)(*n_tensors)
     return float(_load().omse_oracle_compression_ratio(a, b, c, d, n))
+
+
+def alg1_rows(t, bits=(4, 4), is_signed=(True, True), n_cand=1024, hi_frac=1.0, refine_iters=3, n_sweeps=2):
+    """Algorithm 1 with one signedness flag per quantized tensor; also returns the error after every update
+    as sse_sweeps [n_sweeps, n_tensors, S]."""
+    t = _f32(t)
+    S, K = t.shape
+    n = len(bits)
+    b = (C.c_int * n)(*bits)
+    f = (C.c_int * n)(*[int(x) for x in is_signed])
+    alpha = np.zeros((n, S), np.float32)
+    sse = np.zeros((n, S), np.float64)
+    idx = np.zeros((n, S), np.int32)
+    q = np.zeros((n, S, K), np.int8)
+    hist = np.zeros((n_sweeps, n, S), np.float64)
+    st = C.c_uint32(0)
+    _load().omse_oracle_alg1_rows(_p(t, C.c_float), S, K, b, f, n_cand, _c32(hi_frac), refine_iters, n, n_sweeps,
+                                  _p(alpha, C.c_float), _p(sse, C.c_double), _p(idx, C.c_int32), _p(q, C.c_int8),
+                                  _p(hist, C.c_double), C.byref(st))
+    return ResidualResult(alpha, sse, idx, q, st.value), hist
 
 
 def pack_int4(codes_) -> np.ndarray:

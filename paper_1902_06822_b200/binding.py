@@ -22,6 +22,7 @@ STATIC_MAX_CANDIDATES = 2048
 EXPORTS = [
     "omse_create", "omse_destroy", "omse_set_stream", "omse_workspace_bytes", "omse_quantize_weights",
     "omse_quantize_weights_batched", "omse_dual_quantize", "omse_select_key_layers", "omse_compression_ratio",
+    "omse_alg1_quantize",
     "omse_activation_scale", "omse_residual_quantize", "omse_pack_int4", "omse_last_device_status",
     "omse_status_string", "omse_activation_scale_static",
 ]
@@ -73,6 +74,8 @@ def load_library() -> C.CDLL:
     lib.omse_residual_quantize.argtypes = [vp, vp, i64, i64, C.POINTER(C.c_int), i32, C.POINTER(OmseGrid), i32, i32,
                                            vp, vp, vp, vp]
     lib.omse_pack_int4.argtypes = [vp, vp, i64, i32, vp]
+    lib.omse_alg1_quantize.argtypes = [vp, vp, i64, i64, C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(OmseGrid),
+                                       i32, i32, vp, vp, vp, vp, vp]
     lib.omse_select_key_layers.argtypes = [vp, C.POINTER(OmseLayerError), i32, C.c_float, vp, vp]
     lib.omse_compression_ratio.argtypes = [C.POINTER(i64), C.POINTER(i64), C.POINTER(i32), C.POINTER(i32), i32]
     lib.omse_compression_ratio.restype = C.c_double
@@ -229,6 +232,18 @@ class Context:
                                                    _ptr(is_key, torch.int32))
         if rc != OK:
             raise OmseError(rc, "omse_select_key_layers")
+
+    def omse_alg1_quantize(self, t, n_kernels, kernel_len, bits, is_signed, n_cand, hi_frac, refine_iters, n_sweeps,
+                           alpha, sse, sse_history=None, codes=None, packed=None):
+        g = OmseGrid(n_cand, hi_frac, refine_iters)
+        b = (C.c_int * len(bits))(*bits)
+        f = (C.c_int * len(bits))(*[int(x) for x in is_signed])
+        rc = load_library().omse_alg1_quantize(
+            self._h, _ptr(t, torch.float32), n_kernels, kernel_len, b, f, C.byref(g), len(bits), n_sweeps,
+            _ptr(alpha, torch.float32), _ptr(sse, torch.float32), _ptr(sse_history, torch.float32),
+            _ptr(codes, torch.int8), _ptr(packed, torch.uint8))
+        if rc != OK:
+            raise OmseError(rc, "omse_alg1_quantize")
 
     def omse_pack_int4(self, codes, n, is_signed, packed):
         rc = load_library().omse_pack_int4(self._h, _ptr(codes, torch.int8), n, int(is_signed), _ptr(packed, torch.uint8))

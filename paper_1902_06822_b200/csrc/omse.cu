@@ -377,7 +377,16 @@ int omse_quantize_weights_batched(omse_ctx* ctx, const omse_weight_tensor* tenso
 int omse_residual_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, int64_t kernel_len, const int* bits,
                            int is_signed, const omse_grid* grid, int n_tensors, int n_sweeps, float* d_alpha,
                            float* d_sse, int8_t* d_codes, uint8_t* d_packed) {
-    if (!ctx || !grid_ok(grid) || !bits || n_tensors < 1 || n_tensors > OMSE_MAX_TENSORS || n_sweeps < 1 ||
+    int flags[OMSE_MAX_TENSORS];
+    for (int j = 0; j < OMSE_MAX_TENSORS; ++j) flags[j] = is_signed;
+    return omse_alg1_quantize(ctx, d_t, n_kernels, kernel_len, bits, flags, grid, n_tensors, n_sweeps, d_alpha, d_sse,
+                              nullptr, d_codes, d_packed);
+}
+
+int omse_alg1_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, int64_t kernel_len, const int* bits,
+                       const int* is_signed, const omse_grid* grid, int n_tensors, int n_sweeps, float* d_alpha,
+                       float* d_sse, float* d_sse_history, int8_t* d_codes, uint8_t* d_packed) {
+    if (!ctx || !grid_ok(grid) || !bits || !is_signed || n_tensors < 1 || n_tensors > OMSE_MAX_TENSORS || n_sweeps < 1 ||
         n_sweeps > 64 || n_kernels < 0 || kernel_len < 1 || kernel_len > OMSE_MAX_KERNEL_LEN ||
         n_kernels > (int64_t)1 << 40)
         return OMSE_EINVAL;
@@ -388,7 +397,7 @@ int omse_residual_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, i
     if (n_sweeps > 1 && (!d_codes || kernel_len > OMSE_MAX_KERNEL_LEN_MULTISWEEP)) return OMSE_EINVAL;
     if (n_kernels == 0) return OMSE_OK;
     if (!d_t || !d_alpha || !d_sse) return OMSE_EINVAL;
-    if (misaligned4(d_t) || misaligned4(d_alpha) || misaligned4(d_sse)) return OMSE_EINVAL;
+    if (misaligned4(d_t) || misaligned4(d_alpha) || misaligned4(d_sse) || misaligned4(d_sse_history)) return OMSE_EINVAL;
     if (cudaSetDevice(ctx->device) != cudaSuccess) return OMSE_ECUDA;
     omse::RowArgs a;
     memset(&a, 0, sizeof(a));
@@ -401,8 +410,9 @@ int omse_residual_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, i
     a.refine_iters = grid->refine_iters;
     a.n_tensors = n_tensors;
     a.n_sweeps = n_sweeps;
-    for (int j = 0; j < n_tensors; ++j) bounds(bits[j], is_signed, &a.lo[j], &a.hi[j]);
+    for (int j = 0; j < n_tensors; ++j) bounds(bits[j], is_signed[j], &a.lo[j], &a.hi[j]);
     a.keep_x0 = n_sweeps > 1 ? 1 : 0;
+    a.sse_history = d_sse_history;
     return launch_rows(ctx, a, kernel_len);
 }
 

@@ -37,6 +37,7 @@ struct RowArgs {
     int refine_iters;
     int n_tensors, n_sweeps;    // Algorithm 1: quantized tensors per row, sweeps
     int lo[4], hi[4];           // grid bounds per quantized tensor (Section 3.1)
+    float* sse_history;         // [n_sweeps][n_tensors][S] error after every update of Algorithm 1, nullable (single tensor launches)
     unsigned int* status;
     int groups;                 // element groups per block
     int tg;                     // threads per group (multiple of 32); candidate c = slot*tg + t
@@ -517,6 +518,7 @@ __global__ void __launch_bounds__(OMSE_ROWS_MAX_THREADS) rows_kernel(const RowAr
                     if (tid == 0) {
                         T.alpha[(long long)j * T.S + row] = r.alpha;
                         T.sse[(long long)j * T.S + row] = (float)sse;
+                        if (a.sse_history) a.sse_history[((long long)sweep * a.n_tensors + j) * T.S + row] = (float)sse;
                         if (T.best_idx && j == 0) T.best_idx[row] = r.idx;
                     }
                     if (!a.keep_x0 && j + 1 < a.n_tensors) {

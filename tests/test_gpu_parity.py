@@ -312,3 +312,26 @@ def test_random_configurations(gpu, seed):
     assert st["idx_diff"] <= max(1, st["rows"] // 50) and st["alpha_bitwise"] >= 0.98, st
     if pk is not None:
         assert np.array_equal(pk, orc.pack_int4(q))
+
+
+def test_algorithm_1_history_and_mixed_signedness_match_oracle(gpu):
+    import torch
+    t = np.abs(synth.student_t3(10 * 1200, seed=88)).reshape(10, 1200)
+    S, K = t.shape
+    d_t = torch.from_numpy(t).cuda()
+    alpha = torch.empty(2, S, device="cuda")
+    sse = torch.empty(2, S, device="cuda")
+    hist = torch.full((3, 2, S), -1.0, device="cuda")
+    codes = torch.empty(2, S * K, dtype=torch.int8, device="cuda")
+    gpu.ctx().omse_alg1_quantize(d_t, S, K, [4, 3], [False, True], 256, 1.0, 2, 3, alpha, sse, hist, codes)
+    torch.cuda.synchronize()
+    ref, ref_hist = orc.alg1_rows(t, (4, 3), (False, True), 256, 1.0, 2, n_sweeps=3)
+    np.testing.assert_allclose(alpha.cpu().numpy(), ref.alpha, rtol=RTOL)
+    np.testing.assert_allclose(sse.cpu().numpy(), ref.sse, rtol=RTOL)
+    np.testing.assert_allclose(hist.cpu().numpy(), ref_hist, rtol=RTOL)
+    same = np.all(alpha.cpu().numpy() == ref.alpha, axis=0)
+    assert same.mean() >= 0.8
+    q = codes.cpu().numpy().reshape(2, S, K)
+    assert np.array_equal(q[:, same], ref.codes[:, same])
+    assert q[0].min() >= 0 and q[1].min() < 0
+    assert torch.equal(hist[-1], sse)

@@ -388,3 +388,23 @@ def test_layer_mse_and_compression_ratio_by_hand():
     nt = np.ones(54, int)
     nt[order[-2:]] = 2
     assert 0.01 < orc.compression_ratio(ks, ls, [4] * 54, nt.tolist()) - plain < 0.03
+
+
+def test_algorithm_1_history_and_mixed_signedness():
+    """The error after every update is non-increasing up to the grid resolution, ends at the reported error,
+    and a non-negative tensor may take an unsigned first tensor with a signed residual tensor."""
+    t = synth.student_t3(6 * 120, seed=77).reshape(6, 120)
+    res, hist = orc.alg1_rows(t, (3, 3), (True, True), 64, 1.0, 2, n_sweeps=3)
+    same = orc.residual_rows(t, (3, 3), True, 64, 1.0, 2, n_sweeps=3)
+    assert np.array_equal(res.alpha, same.alpha) and np.array_equal(res.codes, same.codes)
+    assert np.array_equal(hist[-1], res.sse)
+    flat = hist.reshape(-1, 6)
+    assert np.all(flat[1:] <= flat[:-1] * 1.05)                # each update re-solves one tensor with the rest fixed
+    assert np.all(flat[-1] <= flat[1] * (1 + 1e-9))
+    x = np.abs(t)
+    mixed, _ = orc.alg1_rows(x, (4, 4), (False, True), 64, 1.0, 2, n_sweeps=1)
+    assert mixed.codes[0].min() >= 0 and mixed.codes[0].max() <= 15 and mixed.codes[1].min() < 0
+    uns, _ = orc.alg1_rows(x, (4, 4), (False, False), 64, 1.0, 2, n_sweeps=1)
+    assert mixed.sse[1].sum() < uns.sse[1].sum()               # an unsigned residual tensor cannot fix negative rests
+    first = orc.quantize_rows(x, 4, False, 64, 1.0, 2)
+    assert np.array_equal(mixed.alpha[0], first.alpha) and np.array_equal(mixed.codes[0], first.codes)

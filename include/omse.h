@@ -151,6 +151,22 @@ int omse_residual_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, i
                            uint8_t* d_packed);
 
 /*
+ * Quantization with offset (Section 3.1, first displayed scheme: T^ = alpha*[(T - delta)/alpha]_Zp + delta,
+ * delta = min_i T_i, unsigned range Z_p = {0..2^p-1}) with the scale found by the MMSE search of
+ * Section 3.4 instead of the (max - delta)/(2^p - 1) rule.  Each kernel (omse_quantize_weights_offset) or
+ * the whole tensor (omse_activation_scale_offset) is shifted by its minimum in binary32, fl(T_i - delta),
+ * and searched on the unsigned grid; d_delta receives the offsets ([n_kernels] or [1]).  The reported
+ * error is that of the shifted values.  Codes are unsigned: for bits = 8 the int8 buffer holds the byte.
+ * Everything else as in omse_quantize_weights / omse_activation_scale.
+ */
+int omse_quantize_weights_offset(omse_ctx* ctx, const float* d_w, int64_t n_kernels, int64_t kernel_len,
+                                 int bits, const omse_grid* grid, float* d_alpha, float* d_delta,
+                                 float* d_sse, int32_t* d_best_idx, int8_t* d_codes, uint8_t* d_packed);
+int omse_activation_scale_offset(omse_ctx* ctx, const float* d_x, int64_t n, int bits,
+                                 const omse_grid* grid, float* d_alpha, float* d_delta, float* d_sse,
+                                 int32_t* d_best_idx, double* d_sse_curve);
+
+/*
  * omse_residual_quantize with one signedness flag per quantized tensor and the convergence history of
  * Algorithm 1 (Section 3.5: "until convergence").  is_signed: HOST array [n_tensors] (a non-negative
  * tensor may take an unsigned first tensor and a signed tensor for its residual, whose rounding errors

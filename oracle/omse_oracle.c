@@ -471,6 +471,46 @@ void omse_oracle_dual_rows(const float *t, int64_t n_kernels, int64_t kernel_len
     *status |= st_all;
 }
 
+/*
+ * Quantization with offset (Section 3.1, first displayed scheme: T^ = alpha*[(T - delta)/alpha]_Zp + delta with
+ * delta = min_i T_i and the unsigned range), with the scale found by the MMSE search instead of the
+ * (max - delta)/(2^p - 1) rule: the shifted tensor fl(T_i - delta) (binary32 subtraction) goes through the
+ * same phi on the unsigned grid.  The error is that of the shifted tensor.
+ */
+void omse_oracle_offset_phi(const float *x, int64_t k, int bits, int n_cand, float hi_frac, int refine_iters,
+                            int start_idx, float *alpha, float *delta, double *sse, int32_t *best_idx,
+                            int8_t *codes, uint32_t *status)
+{
+    float d = INFINITY;
+    for (int64_t i = 0; i < k; ++i)
+        if (fabsf(x[i]) <= FLT_MAX && x[i] < d) d = x[i];
+    if (!(d < INFINITY)) d = 0.0f;
+    float *r = (float *)malloc(sizeof(float) * (size_t)(k > 0 ? k : 1));
+    for (int64_t i = 0; i < k; ++i) r[i] = x[i] - d;
+    omse_oracle_phi(r, k, bits, 0, n_cand, hi_frac, refine_iters, start_idx, alpha, sse, best_idx, codes, NULL,
+                    status);
+    *delta = d;
+    free(r);
+}
+
+void omse_oracle_offset_rows(const float *w, int64_t n_kernels, int64_t kernel_len, int bits, int n_cand,
+                             float hi_frac, int refine_iters, const int32_t *start_idx, float *alpha,
+                             float *delta, double *sse, int32_t *best_idx, int8_t *codes, uint32_t *status)
+{
+    uint32_t st_all = 0;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 1) reduction(| : st_all)
+#endif
+    for (int64_t s = 0; s < n_kernels; ++s) {
+        uint32_t st = 0;
+        omse_oracle_offset_phi(w + s * kernel_len, kernel_len, bits, n_cand, hi_frac, refine_iters,
+                               start_idx ? start_idx[s] : -1, &alpha[s], &delta[s], &sse[s], &best_idx[s],
+                               codes ? codes + s * kernel_len : NULL, &st);
+        st_all |= st;
+    }
+    *status |= st_all;
+}
+
 /* Key layers (Section 3.5): a layer is a key layer when its MSE exceeds a threshold tau.  The MSE of a
  * layer is the sum of its kernels' squared errors over its number of elements (Section 3.2 drops the
  * mean factor inside the analysis; the threshold values the paper quotes, e.g. 8e-5, are per element). */

@@ -70,6 +70,8 @@ def _load():
                                                   C.POINTER(C.c_int), C.c_int]
     lib.omse_oracle_alg1_rows.argtypes = [f32p, C.c_int64, C.c_int64, C.POINTER(C.c_int), C.POINTER(C.c_int), C.c_int,
                                           C.c_float, C.c_int, C.c_int, C.c_int, f32p, f64p, i32p, i8p, f64p, u32p]
+    lib.omse_oracle_offset_rows.argtypes = [f32p, C.c_int64, C.c_int64, C.c_int, C.c_int, C.c_float, C.c_int, i32p,
+                                            f32p, f32p, f64p, i32p, i8p, u32p]
     lib.omse_oracle_pack_int4.argtypes = [i8p, C.c_int64, u8p]
     lib.omse_oracle_unpack_int4.argtypes = [u8p, C.c_int64, C.c_int, i8p]
     _lib = lib
@@ -292,6 +294,32 @@ def alg1_rows(t, bits=(4, 4), is_signed=(True, True), n_cand=1024, hi_frac=1.0, 
                                   _p(alpha, C.c_float), _p(sse, C.c_double), _p(idx, C.c_int32), _p(q, C.c_int8),
                                   _p(hist, C.c_double), C.byref(st))
     return ResidualResult(alpha, sse, idx, q, st.value), hist
+
+
+@dataclass
+class OffsetResult:
+    alpha: np.ndarray
+    delta: np.ndarray
+    sse: np.ndarray
+    best_idx: np.ndarray
+    codes: np.ndarray
+    status: int
+
+
+def offset_rows(w, bits=4, n_cand=256, hi_frac=1.0, refine_iters=3, start_idx=None) -> OffsetResult:
+    """Section 3.1 quantization with offset delta = min, scale by the MMSE search, row by row
+    (a 1-row array is the per-tensor case)."""
+    w = _f32(w)
+    S, K = w.shape
+    alpha, delta = np.empty(S, np.float32), np.empty(S, np.float32)
+    sse, idx = np.empty(S, np.float64), np.empty(S, np.int32)
+    q = np.empty((S, K), np.int8)
+    st = C.c_uint32(0)
+    si = None if start_idx is None else np.ascontiguousarray(start_idx, dtype=np.int32)
+    _load().omse_oracle_offset_rows(_p(w, C.c_float), S, K, bits, n_cand, _c32(hi_frac), refine_iters,
+                                    _p(si, C.c_int32), _p(alpha, C.c_float), _p(delta, C.c_float),
+                                    _p(sse, C.c_double), _p(idx, C.c_int32), _p(q, C.c_int8), C.byref(st))
+    return OffsetResult(alpha, delta, sse, idx, q, st.value)
 
 
 def pack_int4(codes_) -> np.ndarray:

@@ -22,7 +22,7 @@ STATIC_MAX_CANDIDATES = 2048
 EXPORTS = [
     "omse_create", "omse_destroy", "omse_set_stream", "omse_workspace_bytes", "omse_quantize_weights",
     "omse_quantize_weights_batched", "omse_dual_quantize", "omse_select_key_layers", "omse_compression_ratio",
-    "omse_alg1_quantize",
+    "omse_alg1_quantize", "omse_quantize_weights_offset", "omse_activation_scale_offset",
     "omse_activation_scale", "omse_residual_quantize", "omse_pack_int4", "omse_last_device_status",
     "omse_status_string", "omse_activation_scale_static",
 ]
@@ -74,6 +74,8 @@ def load_library() -> C.CDLL:
     lib.omse_residual_quantize.argtypes = [vp, vp, i64, i64, C.POINTER(C.c_int), i32, C.POINTER(OmseGrid), i32, i32,
                                            vp, vp, vp, vp]
     lib.omse_pack_int4.argtypes = [vp, vp, i64, i32, vp]
+    lib.omse_quantize_weights_offset.argtypes = [vp, vp, i64, i64, i32, C.POINTER(OmseGrid), vp, vp, vp, vp, vp, vp]
+    lib.omse_activation_scale_offset.argtypes = [vp, vp, i64, i32, C.POINTER(OmseGrid), vp, vp, vp, vp, vp]
     lib.omse_alg1_quantize.argtypes = [vp, vp, i64, i64, C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(OmseGrid),
                                        i32, i32, vp, vp, vp, vp, vp]
     lib.omse_select_key_layers.argtypes = [vp, C.POINTER(OmseLayerError), i32, C.c_float, vp, vp]
@@ -244,6 +246,26 @@ class Context:
             _ptr(codes, torch.int8), _ptr(packed, torch.uint8))
         if rc != OK:
             raise OmseError(rc, "omse_alg1_quantize")
+
+    def omse_quantize_weights_offset(self, w, n_kernels, kernel_len, bits, n_cand, hi_frac, refine_iters, alpha, delta,
+                                     sse, best_idx=None, codes=None, packed=None):
+        g = OmseGrid(n_cand, hi_frac, refine_iters)
+        rc = load_library().omse_quantize_weights_offset(
+            self._h, _ptr(w, torch.float32), n_kernels, kernel_len, bits, C.byref(g), _ptr(alpha, torch.float32),
+            _ptr(delta, torch.float32), _ptr(sse, torch.float32), _ptr(best_idx, torch.int32),
+            _ptr(codes, torch.int8), _ptr(packed, torch.uint8))
+        if rc != OK:
+            raise OmseError(rc, "omse_quantize_weights_offset")
+
+    def omse_activation_scale_offset(self, x, n, bits, n_cand, hi_frac, refine_iters, alpha, delta, sse,
+                                     best_idx=None, sse_curve=None):
+        g = OmseGrid(n_cand, hi_frac, refine_iters)
+        rc = load_library().omse_activation_scale_offset(
+            self._h, _ptr(x, torch.float32), n, bits, C.byref(g), _ptr(alpha, torch.float32),
+            _ptr(delta, torch.float32), _ptr(sse, torch.float32), _ptr(best_idx, torch.int32),
+            _ptr(sse_curve, torch.float64))
+        if rc != OK:
+            raise OmseError(rc, "omse_activation_scale_offset")
 
     def omse_pack_int4(self, codes, n, is_signed, packed):
         rc = load_library().omse_pack_int4(self._h, _ptr(codes, torch.int8), n, int(is_signed), _ptr(packed, torch.uint8))

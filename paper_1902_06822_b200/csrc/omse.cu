@@ -156,6 +156,7 @@ void fill_tensor(omse::RowTensor& t, const float* w, int64_t S, int64_t K, float
     t.best_idx = idx;
     t.codes = reinterpret_cast<signed char*>(codes);
     t.packed = packed;
+    t.delta = nullptr;
     t.unit_begin = 0;
     t.rows_per_unit = (packed && (K & 1)) ? 2 : 1;
     t.small = 0;
@@ -199,6 +200,74 @@ int launch_tensor_sweep_t(omse_ctx* ctx, omse::TensorArgs& a, size_t smem, int* 
 }
 
 }  // namespace
+
+namespace {
+
+// Launch for a list of weight tensors (bounds already set by the caller).
+int quantize_list(omse_ctx* ctx, std::vector<omse::RowTensor>& list, long long max_k, int bits, int is_signed,
+                  const omse_grid* grid) {
+    if (list.empty()) return OMSE_OK;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return OMSE_ECUDA;
+    // Short rows are batched per work unit when the block is a single element group and the launch
+    // still has a few work units per SM afterwards (otherwise one row per block fills the GPU better).
+    size_t smem_small = 0;
+    if (single_group(grid->n_cand, max_k)) {
+        const int cpt = cpt_for(grid->n_cand);
+        const int ncs = cpt * group_threads(grid->n_cand);
+        long long units_if_small = 0;
+        for (const auto& t : list) {
+            const int b = t.K > OMSE_SMALL_K ? t.rows_per_unit : (t.K <= 128 ? 8 : 4);
+            units_if_small += (t.S + b - 1) / b;
+        }
+        if (units_if_small >= 4ll * ctx->n_sm) {
+            for (auto& t : list) {
+                if (t.K > OMSE_SMALL_K) continue;
+                const bool prune = OMSE_PRUNE && t.K >= OMSE_SMALL_PRUNE_K;
+                t.small = prune ? 3 : 1;
+                t.rows_per_unit = t.K <= 128 ? 8 : 4;
+                const size_t kpad = (size_t)((t.K + 3) & ~3ll);
+                // per row: the row, its error curve, its grid; when regrouping also skipped sums, class table, regrouped row
+                const size_t need = (size_t)t.rows_per_unit *
+                    (kpad * 4 + (size_t)ncs * 4 + 16 +
+                     (prune ? (size_t)cpt * 8 + 2 * (cpt + 1) * 4 + (kpad + 4 * cpt) * 4 : 0));
+                if (need > smem_small) smem_small = need;
+            }
+        }
+    }
+    // longest rows first: the dispenser then hands out work in decreasing size and the tail is short
+    std::stable_sort(list.begin(), list.end(), [](const omse::RowTensor& x, const omse::RowTensor& y) { return x.K > y.K; });
+    long long units = 0;
+    for (auto& t : list) {
+        t.unit_begin = units;
+        units += (t.S + t.rows_per_unit - 1) / t.rows_per_unit;
+    }
+    omse::RowArgs a;
+    memset(&a, 0, sizeof(a));
+    a.n_launch_tensors = (int)list.size();
+    a.n_units = units;
+    if (list.size() == 1) {
+        a.tensors = nullptr;
+        a.one = list[0];
+    } else {
+        if (cudaMemcpyAsync(ctx->d_tensors, list.data(), sizeof(omse::RowTensor) * list.size(), cudaMemcpyHostToDevice,
+                            ctx->stream) != cudaSuccess)
+            return OMSE_ECUDA;
+        a.tensors = ctx->d_tensors;
+    }
+    a.n_cand = grid->n_cand;
+    a.hi_frac = grid->hi_frac;
+    a.refine_iters = grid->refine_iters;
+    a.n_tensors = 1;
+    a.n_sweeps = 1;
+    bounds(bits, is_signed, &a.lo[0], &a.hi[0]);
+    a.keep_x0 = 0;
+    return launch_rows(ctx, a, max_k, smem_small);
+}
+
+}  // namespace
+
+static int activation_impl(omse_ctx* ctx, const float* d_x, int64_t n, int bits, int is_signed, const omse_grid* grid,
+                           float* d_alpha, float* d_delta, float* d_sse, int32_t* d_best_idx, double* d_sse_curve);
 
 extern "C" {
 
@@ -316,62 +385,23 @@ int omse_quantize_weights_batched(omse_ctx* ctx, const omse_weight_tensor* tenso
         list.push_back(t);
         if (u.kernel_len > max_k) max_k = u.kernel_len;
     }
-    if (list.empty()) return OMSE_OK;
-    if (cudaSetDevice(ctx->device) != cudaSuccess) return OMSE_ECUDA;
-    // Short rows are batched per work unit when the block is a single element group and the launch
-    // still has a few work units per SM afterwards (otherwise one row per block fills the GPU better).
-    size_t smem_small = 0;
-    if (single_group(grid->n_cand, max_k)) {
-        const int cpt = cpt_for(grid->n_cand);
-        const int ncs = cpt * group_threads(grid->n_cand);
-        long long units_if_small = 0;
-        for (const auto& t : list) {
-            const int b = t.K > OMSE_SMALL_K ? t.rows_per_unit : (t.K <= 128 ? 8 : 4);
-            units_if_small += (t.S + b - 1) / b;
-        }
-        if (units_if_small >= 4ll * ctx->n_sm) {
-            for (auto& t : list) {
-                if (t.K > OMSE_SMALL_K) continue;
-                const bool prune = OMSE_PRUNE && t.K >= OMSE_SMALL_PRUNE_K;
-                t.small = prune ? 3 : 1;
-                t.rows_per_unit = t.K <= 128 ? 8 : 4;
-                const size_t kpad = (size_t)((t.K + 3) & ~3ll);
-                // per row: the row, its error curve, its grid; when regrouping also skipped sums, class table, regrouped row
-                const size_t need = (size_t)t.rows_per_unit *
-                    (kpad * 4 + (size_t)ncs * 4 + 16 +
-                     (prune ? (size_t)cpt * 8 + 2 * (cpt + 1) * 4 + (kpad + 4 * cpt) * 4 : 0));
-                if (need > smem_small) smem_small = need;
-            }
-        }
-    }
-    // longest rows first: the dispenser then hands out work in decreasing size and the tail is short
-    std::stable_sort(list.begin(), list.end(), [](const omse::RowTensor& x, const omse::RowTensor& y) { return x.K > y.K; });
-    long long units = 0;
-    for (auto& t : list) {
-        t.unit_begin = units;
-        units += (t.S + t.rows_per_unit - 1) / t.rows_per_unit;
-    }
-    omse::RowArgs a;
-    memset(&a, 0, sizeof(a));
-    a.n_launch_tensors = (int)list.size();
-    a.n_units = units;
-    if (list.size() == 1) {
-        a.tensors = nullptr;
-        a.one = list[0];
-    } else {
-        if (cudaMemcpyAsync(ctx->d_tensors, list.data(), sizeof(omse::RowTensor) * list.size(), cudaMemcpyHostToDevice,
-                            ctx->stream) != cudaSuccess)
-            return OMSE_ECUDA;
-        a.tensors = ctx->d_tensors;
-    }
-    a.n_cand = grid->n_cand;
-    a.hi_frac = grid->hi_frac;
-    a.refine_iters = grid->refine_iters;
-    a.n_tensors = 1;
-    a.n_sweeps = 1;
-    bounds(bits, is_signed, &a.lo[0], &a.hi[0]);
-    a.keep_x0 = 0;
-    return launch_rows(ctx, a, max_k, smem_small);
+    return quantize_list(ctx, list, max_k, bits, is_signed, grid);
+}
+
+int omse_quantize_weights_offset(omse_ctx* ctx, const float* d_w, int64_t n_kernels, int64_t kernel_len, int bits,
+                                 const omse_grid* grid, float* d_alpha, float* d_delta, float* d_sse,
+                                 int32_t* d_best_idx, int8_t* d_codes, uint8_t* d_packed) {
+    if (!ctx || !grid_ok(grid) || bits < 2 || bits > 8 || n_kernels < 0 || kernel_len < 1 ||
+        kernel_len > OMSE_MAX_KERNEL_LEN || n_kernels > (int64_t)1 << 40 || (d_packed && bits > 4))
+        return OMSE_EINVAL;
+    if (n_kernels == 0) return OMSE_OK;
+    if (!d_w || !d_alpha || !d_sse || !d_delta) return OMSE_EINVAL;
+    if (misaligned4(d_w) || misaligned4(d_alpha) || misaligned4(d_sse) || misaligned4(d_best_idx) || misaligned4(d_delta))
+        return OMSE_EINVAL;
+    std::vector<omse::RowTensor> list(1);
+    fill_tensor(list[0], d_w, n_kernels, kernel_len, d_alpha, d_sse, d_best_idx, d_codes, d_packed);
+    list[0].delta = d_delta;
+    return quantize_list(ctx, list, kernel_len, bits, /*is_signed=*/0, grid);
 }
 
 int omse_residual_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, int64_t kernel_len, const int* bits,
@@ -508,6 +538,20 @@ double omse_compression_ratio(const int64_t* n_kernels, const int64_t* kernel_le
 
 int omse_activation_scale(omse_ctx* ctx, const float* d_x, int64_t n, int bits, int is_signed, const omse_grid* grid,
                           float* d_alpha, float* d_sse, int32_t* d_best_idx, double* d_sse_curve) {
+    return activation_impl(ctx, d_x, n, bits, is_signed, grid, d_alpha, nullptr, d_sse, d_best_idx, d_sse_curve);
+}
+
+int omse_activation_scale_offset(omse_ctx* ctx, const float* d_x, int64_t n, int bits, const omse_grid* grid,
+                                 float* d_alpha, float* d_delta, float* d_sse, int32_t* d_best_idx,
+                                 double* d_sse_curve) {
+    if (!d_delta || misaligned4(d_delta)) return OMSE_EINVAL;
+    return activation_impl(ctx, d_x, n, bits, /*is_signed=*/0, grid, d_alpha, d_delta, d_sse, d_best_idx, d_sse_curve);
+}
+
+}  // extern "C"
+
+static int activation_impl(omse_ctx* ctx, const float* d_x, int64_t n, int bits, int is_signed, const omse_grid* grid,
+                           float* d_alpha, float* d_delta, float* d_sse, int32_t* d_best_idx, double* d_sse_curve) {
     if (!ctx || !grid_ok(grid) || bits < 2 || bits > 8 || n < 0 || !d_alpha || !d_sse) return OMSE_EINVAL;
     if (n > 0 && !d_x) return OMSE_EINVAL;
     if ((reinterpret_cast<uintptr_t>(d_x) & 15) || (reinterpret_cast<uintptr_t>(d_alpha) & 3) ||
@@ -533,6 +577,7 @@ int omse_activation_scale(omse_ctx* ctx, const float* d_x, int64_t n, int bits, 
     a.alpha_out = d_alpha;
     a.sse_out = d_sse;
     a.idx_out = d_best_idx;
+    a.delta_out = d_delta;
     a.status = &ctx->ws->status;
     cudaStream_t s = ctx->stream;
 
@@ -543,6 +588,7 @@ int omse_activation_scale(omse_ctx* ctx, const float* d_x, int64_t n, int bits, 
     int n_blocks = 1;
     if (n > 0) {
         omse::tensor_absmax_kernel<<<(unsigned)pass_grid, 256, 0, s>>>(d_x, n, a.st, a.status);
+        if (d_delta) omse::tensor_offset_kernel<<<1, 32, 0, s>>>(a.st);
         const size_t smem = (size_t)a.tile4 * 16 + (size_t)cpt * 16 + (size_t)(a.groups - 1) * cpt * a.tg * 8;
         int rc;
         switch (cpt) {
@@ -559,6 +605,8 @@ int omse_activation_scale(omse_ctx* ctx, const float* d_x, int64_t n, int bits, 
     omse::tensor_pass_kernel<2><<<(unsigned)pass_grid, 256, 0, s>>>(a);
     return cudaGetLastError() == cudaSuccess ? OMSE_OK : OMSE_ECUDA;
 }
+
+extern "C" {
 
 int omse_pack_int4(omse_ctx* ctx, const int8_t* d_codes, int64_t n, int is_signed, uint8_t* d_packed) {
     (void)is_signed;
@@ -616,6 +664,9 @@ __global__ void static_begin_kernel(StaticScratch* s) {
         s->tstate.step = 0.f;
         s->tstate.n_list = 0;
         s->tstate.list_overflow = 0;
+        s->tstate.key_min = 0x7fffffff;
+        s->tstate.key_max = (int)0x80000000;
+        s->tstate.delta = 0.f;
     }
 }
 

@@ -19,6 +19,7 @@ struct RowTensor {
     int* best_idx;           // [S] (single quantized tensor only), nullable
     signed char* codes;      // [n_tensors][N], nullable
     unsigned char* packed;   // [n_tensors][ceil(N/2)], nullable
+    float* delta;            // [S] offset subtracted from each row (Section 3.1 scheme with offset), nullable = no offset
     long long unit_begin;    // index of this tensor's first work unit in the launch-wide numbering
     int rows_per_unit;       // long rows: 2 when nibble packing needs an even element count per unit (odd K), else 1;
                              // short rows: the batch size B (even)
@@ -485,6 +486,25 @@ __global__ void __launch_bounds__(OMSE_ROWS_MAX_THREADS) rows_kernel(const RowAr
                 }
             }
             if (bad) st |= 1u;
+            if (T.delta) {
+                // quantization with offset: delta = min of the row, the shifted row fl(x - delta) is what gets searched
+                __syncthreads();
+                float lo = INFINITY;
+                for (int i = tid; i < k; i += nthr) {
+                    const float v = s.xs[i];
+                    if (fabsf(v) <= FLT_MAX) lo = fminf(lo, v);
+                }
+                __shared__ float s_min[32];
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+                if ((tid & 31) == 0) s_min[tid >> 5] = lo;
+                __syncthreads();
+                float d = INFINITY;
+                for (int w = 0; w < ((nthr + 31) >> 5); ++w) d = fminf(d, s_min[w]);
+                if (!(d < INFINITY)) d = 0.f;
+                for (int i = tid; i < k; i += nthr) s.xs[i] = s.xs[i] - d;
+                if (tid == 0) T.delta[row] = d;
+            }
             if (a.keep_x0) {
                 __syncthreads();
                 for (int i = tid; i < 4 * k4; i += nthr) s.x0[i] = s.xs[i];

@@ -297,6 +297,19 @@ __device__ void small_unit(const RowArgs& a, const RowTensor& T, long long unit_
 
     // ---- max of the positive and negative part of every row, and the row's grid: a warp per row
     for (int r = warp; r < nrows; r += nwarp) {
+        if (T.delta) {   // quantization with offset: subtract the row minimum first
+            float lo = INFINITY;
+            for (int i = lane; i < k; i += 32) {
+                const float v = xs[r * kpad + i];
+                if (fabsf(v) <= FLT_MAX) lo = fminf(lo, v);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+            if (!(lo < INFINITY)) lo = 0.f;
+            for (int i = lane; i < k; i += 32) xs[r * kpad + i] = xs[r * kpad + i] - lo;
+            if (lane == 0) T.delta[row0 + r] = lo;
+            __syncwarp();
+        }
         float mp = 0.f, mn = 0.f;
         for (int i = lane; i < k; i += 32) {
             const float v = xs[r * kpad + i];

@@ -19,7 +19,8 @@ struct TensorState {          // lives in the context workspace
     int n_list;
     int list_overflow;
     int list[kListCap];
-    int pad_;
+    int key_min, key_max;                // offset mode: order-preserving integer keys of min and max of the tensor
+    float delta;                         // offset subtracted from every element (0 without offset)
 };
 
 struct TensorArgs {
@@ -37,6 +38,7 @@ struct TensorArgs {
     float* alpha_out;
     float* sse_out;
     int* idx_out;
+    float* delta_out;       // offset mode: receives delta; nullptr = no offset
     unsigned int* status;
 };
 
@@ -50,13 +52,33 @@ __global__ void tensor_init_kernel(TensorState* st) {
         st->step = 0.f;
         st->n_list = 0;
         st->list_overflow = 0;
+        st->key_min = 0x7fffffff;
+        st->key_max = (int)0x80000000;
+        st->delta = 0.f;
+    }
+}
+
+// order-preserving map float -> int (finite values)
+__device__ __forceinline__ int float_key(float f) {
+    const int i = __float_as_int(f);
+    return i >= 0 ? i : i ^ 0x7fffffff;
+}
+__device__ __forceinline__ float key_float(int k) { return __int_as_float(k >= 0 ? k : k ^ 0x7fffffff); }
+
+// Offset mode (Section 3.1 scheme with offset): delta = min, and the search range is that of the shifted tensor.
+__global__ void tensor_offset_kernel(TensorState* st) {
+    if (threadIdx.x == 0 && st->key_min <= st->key_max) {
+        const float lo = key_float(st->key_min), hi = key_float(st->key_max);
+        st->delta = lo;
+        st->mpos_bits = __float_as_uint(hi - lo);    // max of fl(x - delta): subtraction is monotone
+        st->mneg_bits = 0u;
     }
 }
 
 __global__ void __launch_bounds__(256) tensor_absmax_kernel(const float* __restrict__ x, long long n,
                                                              TensorState* st, unsigned int* status) {
     __shared__ double scratch[64];
-    float mpos = 0.f, mneg = 0.f;
+    float mpos = 0.f, mneg = 0.f, lo = INFINITY, hi = -INFINITY;
     bool bad = false;
     const long long n4 = n >> 2;
     const float4* x4 = reinterpret_cast<const float4*>(x);
@@ -69,6 +91,8 @@ __global__ void __launch_bounds__(256) tensor_absmax_kernel(const float* __restr
             if (fabsf(e[j]) <= FLT_MAX) {
                 mpos = fmaxf(mpos, e[j]);
                 mneg = fmaxf(mneg, -e[j]);
+                lo = fminf(lo, e[j]);
+                hi = fmaxf(hi, e[j]);
             } else {
                 bad = true;
             }
@@ -79,9 +103,20 @@ __global__ void __launch_bounds__(256) tensor_absmax_kernel(const float* __restr
         if (fabsf(v) <= FLT_MAX) {
             mpos = fmaxf(mpos, v);
             mneg = fmaxf(mneg, -v);
+            lo = fminf(lo, v);
+            hi = fmaxf(hi, v);
         } else {
             bad = true;
         }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+        hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+    }
+    if ((threadIdx.x & 31) == 0 && lo <= hi) {   // the warp saw a finite value: integer atomics on order-preserving keys
+        atomicMin(&st->key_min, float_key(lo));
+        atomicMax(&st->key_max, float_key(hi));
     }
     block_max2(mpos, mneg, scratch);
     if (threadIdx.x == 0) {
@@ -113,6 +148,7 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
     if (!(m > 0.f) || !(a_last >= FLT_MIN)) return;   // degenerate tensor: finish kernel reports it
     const float inv_thr = g.rstep * (1.0f / 0.4999f);
     const float inv_tg = 1.0f / (float)a.tg;
+    const float delta = a.st->delta;                  // 0 unless the offset scheme is used
 
     u64 inv2[CPT], na2[CPT];
     double dacc[CPT];
@@ -151,10 +187,14 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
                 const long long e = (base4 + i) << 2;
                 if (e + 3 < a.n) {
                     v = __ldg(x4 + base4 + i);
+                    v.x -= delta;
+                    v.y -= delta;
+                    v.z -= delta;
+                    v.w -= delta;
                 } else {   // ragged end of the tensor: missing elements count as zeros
-                    v.x = e < a.n ? a.x[e] : 0.f;
-                    v.y = e + 1 < a.n ? a.x[e + 1] : 0.f;
-                    v.z = e + 2 < a.n ? a.x[e + 2] : 0.f;
+                    v.x = e < a.n ? a.x[e] - delta : 0.f;
+                    v.y = e + 1 < a.n ? a.x[e + 1] - delta : 0.f;
+                    v.z = e + 2 < a.n ? a.x[e + 2] - delta : 0.f;
                 }
             }
             const float e4[4] = {v.x, v.y, v.z, v.w};
@@ -343,6 +383,7 @@ __global__ void __launch_bounds__(256) tensor_pass_kernel(const TensorArgs a) {
     const int n_list = MODE == 0 ? st->n_list : 1;
     if (MODE == 0 && n_list == 0) return;
     const float alpha_now = st->alpha;
+    const float delta = st->delta;
     if (MODE == 1 && !(alpha_now > 0.f)) return;
     double* part_d = a.partials;                                         // [grid][kListCap]
     long long* part_q = reinterpret_cast<long long*>(a.partials + (size_t)gridDim.x * kListCap);  // [grid]
@@ -383,12 +424,12 @@ __global__ void __launch_bounds__(256) tensor_pass_kernel(const TensorArgs a) {
         };
         for (long long i = tid0; i < n4; i += stride) {
             const float4 v = __ldg(x4 + i);
-            element(v.x);
-            element(v.y);
-            element(v.z);
-            element(v.w);
+            element(v.x - delta);
+            element(v.y - delta);
+            element(v.z - delta);
+            element(v.w - delta);
         }
-        for (long long i = (n4 << 2) + tid0; i < a.n; i += stride) element(a.x[i]);
+        for (long long i = (n4 << 2) + tid0; i < a.n; i += stride) element(a.x[i] - delta);
         const int nj = MODE == 0 ? 4 : 1;
         for (int j = 0; j < nj; ++j) {
             long long q = sqq;
@@ -443,6 +484,7 @@ __global__ void __launch_bounds__(256) tensor_pass_kernel(const TensorArgs a) {
             }
         } else {
             *a.alpha_out = st->alpha;
+            if (a.delta_out) *a.delta_out = st->delta;
             *a.sse_out = (float)tot_d[0];
             if (a.idx_out) *a.idx_out = st->best_idx;
         }

@@ -408,3 +408,35 @@ def test_algorithm_1_history_and_mixed_signedness():
     assert mixed.sse[1].sum() < uns.sse[1].sum()               # an unsigned residual tensor cannot fix negative rests
     first = orc.quantize_rows(x, 4, False, 64, 1.0, 2)
     assert np.array_equal(mixed.alpha[0], first.alpha) and np.array_equal(mixed.codes[0], first.codes)
+
+
+# ---------------------------------------------------------------- Section 3.1: quantization with offset
+def test_offset_quantizer_pins():
+    x = synth.student_t3(4 * 150, seed=91).reshape(4, 150)
+    # (a) one candidate at (max - min)/(2^p - 1) is the uniform scheme with offset of Section 3.1
+    r = orc.offset_rows(x, 4, 1, 1.0 / 15, 0)
+    for s in range(4):
+        lo, hi = float(x[s].min()), float(x[s].max())
+        assert r.delta[s] == np.float32(lo)
+        assert r.alpha[s] == pytest.approx((hi - lo) / 15, rel=1e-6)
+        rec = r.alpha[s].astype(np.float64) * (r.codes[s].astype(np.int64) & 0xFF) + np.float64(r.delta[s])
+        assert np.max(np.abs(rec - x[s])) <= r.alpha[s] * 0.5 * (1 + 1e-5)
+        assert r.codes[s].min() == 0 and r.codes[s].max() == 15
+    # (b) non-negative data whose minimum is 0: the offset changes nothing
+    a = np.abs(x)
+    a[:, 0] = 0.0
+    plain = orc.quantize_rows(a, 4, False, 128, 1.0, 3)
+    off = orc.offset_rows(a, 4, 128, 1.0, 3)
+    assert np.array_equal(off.alpha, plain.alpha) and np.array_equal(off.codes, plain.codes) and not off.delta.any()
+    # (c) an exactly representable shift moves delta and nothing else
+    g = (np.random.default_rng(4).integers(-40, 40, (3, 64)) * 2.0 ** -6).astype(np.float32)
+    o1, o2 = orc.offset_rows(g, 4, 64, 1.0, 2), orc.offset_rows(g + np.float32(8.0), 4, 64, 1.0, 2)
+    assert np.array_equal(o1.alpha, o2.alpha) and np.array_equal(o1.codes, o2.codes)
+    assert np.array_equal(o2.delta, o1.delta + np.float32(8.0)) and np.array_equal(o1.sse, o2.sse)
+    # (d) the reported error is the reconstruction error of alpha*q + delta
+    o = orc.offset_rows(x, 4, 128, 1.0, 3)
+    rec = o.alpha[:, None].astype(np.float64) * o.codes + o.delta[:, None].astype(np.float64)
+    np.testing.assert_allclose(o.sse, np.sum((x.astype(np.float64) - rec) ** 2, axis=1), rtol=1e-5)
+    # (e) for skewed data the offset beats the signed grid of the same width (the extra level of Section 3.1)
+    skew = (np.abs(x) - np.float32(0.3)).astype(np.float32)
+    assert orc.offset_rows(skew, 3, 128, 1.0, 3).sse.sum() < orc.quantize_rows(skew, 3, True, 128, 1.0, 3).sse.sum()

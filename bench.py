@@ -228,7 +228,7 @@ class WeightSet(Workload):
 
 class Activation(Workload):
     kernel = "tensor_sweep_kernel<8>"
-    launches_per_step = 9        # init, absmax, sweep, finish, re-score, 3 polish, final
+    launches_per_step = 10       # init, absmax, sweep, curve, finish, re-score, 3 polish, final
 
     def __init__(self, name, x, n_cand):
         self.name, self.x, self.n_cand = name, x, n_cand

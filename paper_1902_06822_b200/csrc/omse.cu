@@ -599,7 +599,8 @@ static int activation_impl(omse_ctx* ctx, const float* d_x, int64_t n, int bits,
         }
         if (rc != OMSE_OK) return rc;
     }
-    omse::tensor_finish_kernel<<<1, 1024, 0, s>>>(a, n_blocks);
+    omse::tensor_curve_kernel<<<(unsigned)((a.n_cand + 63) / 64), 64, 0, s>>>(a, n_blocks);
+    omse::tensor_finish_kernel<<<1, 1024, 0, s>>>(a);
     omse::tensor_pass_kernel<0><<<(unsigned)pass_grid, 256, 0, s>>>(a);
     for (int it = 0; it < grid->refine_iters; ++it) omse::tensor_pass_kernel<1><<<(unsigned)pass_grid, 256, 0, s>>>(a);
     omse::tensor_pass_kernel<2><<<(unsigned)pass_grid, 256, 0, s>>>(a);
@@ -759,7 +760,8 @@ extern "C" int omse_activation_scale_static(int device, void* cuda_stream, const
         }
         if (rc != OMSE_OK) return rc;
     }
-    omse::tensor_finish_kernel<<<1, 1024, 0, s>>>(a, n_blocks);
+    omse::tensor_curve_kernel<<<(unsigned)((a.n_cand + 63) / 64), 64, 0, s>>>(a, n_blocks);
+    omse::tensor_finish_kernel<<<1, 1024, 0, s>>>(a);
     omse::tensor_pass_kernel<0><<<(unsigned)pass_grid, 256, 0, s>>>(a);
     for (int it = 0; it < grid->refine_iters; ++it) omse::tensor_pass_kernel<1><<<(unsigned)pass_grid, 256, 0, s>>>(a);
     omse::tensor_pass_kernel<2><<<(unsigned)pass_grid, 256, 0, s>>>(a);

@@ -314,9 +314,28 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
     }
 }
 
-// One block: sums the per-block partials in block order, takes the argmin and lists the candidates
-// inside the fp32 noise band of the minimum.
-__global__ void __launch_bounds__(1024) tensor_finish_kernel(const TensorArgs a, int n_blocks) {
+// Sums the per-block partial curves in block order: one thread per candidate, several blocks.
+__global__ void __launch_bounds__(64) tensor_curve_kernel(const TensorArgs a, int n_blocks) {
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= a.n_cand) return;
+    TensorState* st = a.st;
+    const float mpos = __uint_as_float(st->mpos_bits), mneg = __uint_as_float(st->mneg_bits);
+    const GridSetup g = grid_setup(mpos, mneg, a.hi_frac, a.n_cand, (float)a.lo, (float)a.hi);
+    const float a_last = __fmul_rn((float)a.n_cand, g.step);
+    double s = INFINITY;
+    if ((fmaxf(mpos, mneg) > 0.f) && (a_last >= FLT_MIN)) {
+        s = 0.0;
+#pragma unroll 8
+        for (int b = 0; b < n_blocks; ++b) s += __ldcg(&a.partials[(long long)b * a.n_cand + c]);
+        const float ac = __fmul_rn((float)(c + 1), g.step);
+        if (!(ac >= FLT_MIN)) s = INFINITY;
+    }
+    a.curve[c] = s;
+    if (a.curve_out) a.curve_out[c] = s;
+}
+
+// One block: argmin of the summed curve and the list of candidates inside the fp32 noise band of the minimum.
+__global__ void __launch_bounds__(1024) tensor_finish_kernel(const TensorArgs a) {
     __shared__ double scratch[64];
     __shared__ int cnt;
     TensorState* st = a.st;
@@ -329,12 +348,7 @@ __global__ void __launch_bounds__(1024) tensor_finish_kernel(const TensorArgs a,
     int bi = 0x7fffffff;
     if (!degenerate) {
         for (int c = threadIdx.x; c < a.n_cand; c += blockDim.x) {
-            double s = 0.0;
-            for (int b = 0; b < n_blocks; ++b) s += a.partials[(long long)b * a.n_cand + c];
-            const float ac = __fmul_rn((float)(c + 1), g.step);
-            if (!(ac >= FLT_MIN)) s = INFINITY;
-            a.curve[c] = s;
-            if (a.curve_out) a.curve_out[c] = s;
+            const double s = a.curve[c];
             if (s < bv) {
                 bv = s;
                 bi = c;
@@ -350,8 +364,6 @@ __global__ void __launch_bounds__(1024) tensor_finish_kernel(const TensorArgs a,
             st->n_list = 0;
             atomicOr(a.status, 2u);
         }
-        if (degenerate && a.curve_out)
-            for (int c = threadIdx.x; c < a.n_cand; c += blockDim.x) a.curve_out[c] = INFINITY;
         return;
     }
     const double band = bv * (1.0 + kRescoreBand);
@@ -422,7 +434,8 @@ __global__ void __launch_bounds__(256) tensor_pass_kernel(const TensorArgs a) {
                 acc[0] += d * d;
             }
         };
-        for (long long i = tid0; i < n4; i += stride) {
+#pragma unroll 4
+        for (long long i = tid0; i < n4; i += stride) {   // several 128-bit loads in flight per thread
             const float4 v = __ldg(x4 + i);
             element(v.x - delta);
             element(v.y - delta);

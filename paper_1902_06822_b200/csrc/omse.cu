@@ -26,6 +26,9 @@
 #ifndef OMSE_SMALL_PRUNE_K
 #define OMSE_SMALL_PRUNE_K 192      /* short rows at least this long are regrouped by magnitude class */
 #endif
+#ifndef OMSE_TINY_K
+#define OMSE_TINY_K 32              /* rows up to this length, in large numbers, get one thread each */
+#endif
 #ifndef OMSE_SMALL_K
 #define OMSE_SMALL_K 640            /* rows up to this length are batched per work unit */
 #endif
@@ -219,9 +222,19 @@ int quantize_list(omse_ctx* ctx, std::vector<omse::RowTensor>& list, long long m
             const int b = t.K > OMSE_SMALL_K ? t.rows_per_unit : (t.K <= 128 ? 8 : 4);
             units_if_small += (t.S + b - 1) / b;
         }
+        // very short rows in large numbers: a thread per row, a block-sized batch of rows per unit
+        const int threads = group_threads(grid->n_cand);
+        for (auto& t : list) {
+            if (t.K > OMSE_TINY_K || t.S < 64ll * ctx->n_sm) continue;
+            t.small = 4;
+            t.rows_per_unit = threads;
+            const size_t need = (size_t)((threads * t.K + 3) & ~3ll) * 4 + (size_t)((grid->n_cand + 3) & ~3) * 4 +
+                                (size_t)threads * t.K + 16;
+            if (need > smem_small) smem_small = need;
+        }
         if (units_if_small >= 4ll * ctx->n_sm) {
             for (auto& t : list) {
-                if (t.K > OMSE_SMALL_K) continue;
+                if (t.K > OMSE_SMALL_K || t.small) continue;
                 const bool prune = OMSE_PRUNE && t.K >= OMSE_SMALL_PRUNE_K;
                 t.small = prune ? 3 : 1;
                 t.rows_per_unit = t.K <= 128 ? 8 : 4;

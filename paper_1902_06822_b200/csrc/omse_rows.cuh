@@ -24,7 +24,8 @@ struct RowTensor {
     int rows_per_unit;       // long rows: 2 when nibble packing needs an even element count per unit (odd K), else 1;
                              // short rows: the batch size B (even)
     int small;               // bit 0: short-row path (batch of rows per unit, a warp finishes each row);
-                             // bit 1: that path regroups rows by magnitude class
+                             // bit 1: that path regroups rows by magnitude class;
+                             // bit 2: thread-per-row path for very short rows (rows_per_unit = block size)
 };
 
 struct RowArgs {
@@ -50,6 +51,7 @@ struct RowArgs {
 }  // namespace omse
 
 #include "omse_rows_small.cuh"
+#include "omse_rows_tiny.cuh"
 
 namespace omse {
 
@@ -447,6 +449,10 @@ __global__ void __launch_bounds__(OMSE_ROWS_MAX_THREADS) rows_kernel(const RowAr
             tp = a.tensors + ti;
         }
         const RowTensor& T = *tp;
+        if (T.small & 4) {
+            tiny_dispatch<CPT>(a, T, unit - T.unit_begin, smem_raw, st);
+            continue;
+        }
         if (T.small) {
             small_unit<CPT>(a, T, unit - T.unit_begin, smem_raw, rcp, st);
             continue;

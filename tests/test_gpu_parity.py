@@ -335,3 +335,24 @@ def test_algorithm_1_history_and_mixed_signedness_match_oracle(gpu):
     assert np.array_equal(q[:, same], ref.codes[:, same])
     assert q[0].min() >= 0 and q[1].min() < 0
     assert torch.equal(hist[-1], sse)
+
+
+# ---------------------------------------------------------------- very short rows in large numbers: a thread per row
+@pytest.mark.parametrize("k,bits,signed", [(1, 4, True), (2, 4, True), (3, 2, True), (9, 4, False), (17, 3, True),
+                                           (27, 4, True), (27, 2, True), (28, 8, True), (32, 4, True), (31, 4, False)])
+def test_very_short_rows_thread_per_row_path(gpu, k, bits, signed):
+    s = 9600 + 37                                  # at least 64 rows per SM; the last unit is ragged
+    w = synth.student_t3(s * k, seed=900 + k, tensor_id=bits).reshape(s, k)
+    if not signed and k != 31:
+        w = np.abs(w)
+    w[5] = 0.0                                     # a degenerate row inside a unit
+    rows = np.unique(np.concatenate([np.arange(0, s, 13), [5, s - 1, s - 2, 127, 128, 129]]))
+    alpha, sse, idx, q, pk = gpu.quantize_weights(w, bits, signed, 1024, 1.0, 3, True, bits <= 4)
+    good = rows[rows != 5]
+    st = check_rows(w, alpha, sse, idx, q, None, bits, signed, 1024, 1.0, 3, rows=good)
+    assert st["idx_diff"] <= max(1, st["rows"] // 50) and st["alpha_bitwise"] >= 0.98, st
+    assert alpha[5] == 0.0 and idx[5] == -1 and not q.reshape(s, k)[5].any()
+    if pk is not None:
+        assert np.array_equal(pk, orc.pack_int4(q))
+    lo, hi = (-(1 << (bits - 1)), (1 << (bits - 1)) - 1) if signed else (0, (1 << bits) - 1)
+    assert q.astype(np.int16).min() >= (lo if signed or bits < 8 else -128)

@@ -356,3 +356,25 @@ def test_very_short_rows_thread_per_row_path(gpu, k, bits, signed):
         assert np.array_equal(pk, orc.pack_int4(q))
     lo, hi = (-(1 << (bits - 1)), (1 << (bits - 1)) - 1) if signed else (0, (1 << bits) - 1)
     assert q.astype(np.int16).min() >= (lo if signed or bits < 8 else -128)
+
+
+def test_non_finite_and_zero_rows_on_every_launch_path(gpu):
+    """NaN / Inf / all-zero / denormal rows never fault and never disturb their neighbours, whichever path
+    (long regrouped rows, batched short rows, thread-per-row) the launch takes."""
+    for s, k in [(12, 3000), (2600, 256), (9700, 27)]:
+        w = synth.laplace(s * k, 0.02, seed=950 + k).reshape(s, k).copy()
+        w[1] = 0.0
+        w[3, k // 2] = np.nan
+        w[5, 0] = np.inf
+        w[7] = 1e-42
+        gpu.ctx().omse_last_device_status()
+        alpha, sse, idx, q, pk = gpu.quantize_weights(w, 4, True, 1024, 1.0, 3, True, True)
+        st = gpu.ctx().omse_last_device_status()
+        assert st & 1 and st & 2
+        for r in (1, 3, 5, 7):
+            assert alpha[r] == 0.0 and idx[r] == -1 and not q.reshape(s, k)[r].any(), (k, r)
+        assert sse[1] == 0.0
+        assert q.min() >= -8 and q.max() <= 7
+        good = np.array([0, 2, 4, 6, 8, 9, 10, 11, s - 1])
+        check_rows(w, alpha, sse, idx, q, None, 4, True, 1024, 1.0, 3, rows=good)
+        assert np.array_equal(pk, orc.pack_int4(q))

@@ -438,7 +438,9 @@ def run_ours(args, rank, world):
     for _ in range(max(args.warmup, 3)):
         wl.step()
     torch.cuda.synchronize()
+    ctx.omse_read_evaluations()                     # clear the instrumentation counter
     ms = timed(wl.step, args.steps)
+    executed = ctx.omse_read_evaluations() / args.steps   # evaluations the kernels really executed per step
     clocks = sampler.stop() if sampler else None
     wl.step_e2e()
     ms_e2e = timed(wl.step_e2e, args.steps)
@@ -467,7 +469,11 @@ def run_ours(args, rank, world):
                          "unit": "T FP32-instr/s", "frac": achieved / peak,
                          "traffic": NCU_TRAFFIC_BYTES if args.workload == "c2" else None,
                          "kernel": wl.kernel, "peak_source": f"148 SMs x 128 lanes x {sm_max_mhz:.0f} MHz ({peak_src} max clock)",
-                         "instr_per_eval": ipe, "evaluations_per_s": evals / per_step_s},
+                         "instr_per_eval": ipe, "evaluations_per_s": evals / per_step_s,
+                         # the kernels skip, exactly, evaluations whose code is provably zero: what was executed,
+                         # and the FMA-pipe lane operations (4 per executed evaluation) against the same peak
+                         "executed_evaluations_per_step": executed, "executed_share": executed / evals,
+                         "executed_fma_frac": 4.0 * executed / per_step_s / peak},
         }
         if world == 1 and not args.no_cpu_baseline:
             v, cores, desc, _ = wl.cpu()

@@ -278,6 +278,13 @@ int omse_activation_scale_static(int device, void* cuda_stream, const float* d_x
  * since the last read) to *host_out and clears it. */
 int omse_last_device_status(omse_ctx* ctx, uint32_t* host_out);
 
+/* Instrumentation (no counterpart in the paper): synchronises the stream and returns in *host_out how many
+ * (element, candidate) evaluations the search kernels of this context actually executed since the last read,
+ * then clears the counter.  The algorithmic count of a call is n_cand * elements (* quantized tensors); the
+ * kernels execute fewer because a candidate skips, exactly, the elements it is known to code as zero.  For
+ * omse_dual_quantize the unit is (element, pair, first code).  omse_activation_scale_static does not count. */
+int omse_read_evaluations(omse_ctx* ctx, uint64_t* host_out);
+
 /* Static description of a return value. */
 const char* omse_status_string(int status);
 

@@ -22,7 +22,7 @@ STATIC_MAX_CANDIDATES = 2048
 EXPORTS = [
     "omse_create", "omse_destroy", "omse_set_stream", "omse_workspace_bytes", "omse_quantize_weights",
     "omse_quantize_weights_batched", "omse_dual_quantize", "omse_select_key_layers", "omse_compression_ratio",
-    "omse_alg1_quantize", "omse_quantize_weights_offset", "omse_activation_scale_offset",
+    "omse_alg1_quantize", "omse_read_evaluations", "omse_quantize_weights_offset", "omse_activation_scale_offset",
     "omse_activation_scale", "omse_residual_quantize", "omse_pack_int4", "omse_last_device_status",
     "omse_status_string", "omse_activation_scale_static",
 ]
@@ -84,6 +84,7 @@ def load_library() -> C.CDLL:
     lib.omse_dual_quantize.argtypes = [vp, vp, i64, i64, i32, i32, i32, C.POINTER(OmseDualGrid), vp, vp, vp, vp, vp]
     lib.omse_activation_scale_static.argtypes = [i32, vp, vp, i64, i32, i32, C.POINTER(OmseGrid), vp, vp, vp, vp, vp]
     lib.omse_last_device_status.argtypes = [vp, C.POINTER(C.c_uint32)]
+    lib.omse_read_evaluations.argtypes = [vp, C.POINTER(C.c_uint64)]
     lib.omse_status_string.argtypes = [i32]
     lib.omse_status_string.restype = C.c_char_p
     _lib = lib
@@ -271,6 +272,13 @@ class Context:
         rc = load_library().omse_pack_int4(self._h, _ptr(codes, torch.int8), n, int(is_signed), _ptr(packed, torch.uint8))
         if rc != OK:
             raise OmseError(rc, "omse_pack_int4")
+
+    def omse_read_evaluations(self) -> int:
+        out = C.c_uint64(0)
+        rc = load_library().omse_read_evaluations(self._h, C.byref(out))
+        if rc != OK:
+            raise OmseError(rc, "omse_read_evaluations")
+        return out.value
 
     def omse_last_device_status(self) -> int:
         out = C.c_uint32(0)

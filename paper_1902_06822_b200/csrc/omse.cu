@@ -46,6 +46,7 @@ struct Workspace {
     unsigned int status;
     unsigned int pad_[3];
     unsigned long long ticket[2];   // work-unit dispenser of the row kernels (self-resetting)
+    unsigned long long evals;       // executed evaluations since the last omse_read_evaluations
     omse::TensorState tstate;
     double curve[OMSE_MAX_CANDIDATES];
 };
@@ -141,6 +142,7 @@ int launch_rows(omse_ctx* ctx, omse::RowArgs& a, long long max_k, size_t smem_sm
     if (smem_small > smem) smem = smem_small;
     a.ticket = ctx->ws->ticket;
     a.status = &ctx->ws->status;
+    a.evals = &ctx->ws->evals;
     switch (cpt) {
         case 1: return launch_rows_t<1>(ctx, a, smem);
         case 2: return launch_rows_t<2>(ctx, a, smem);
@@ -361,6 +363,17 @@ int omse_last_device_status(omse_ctx* ctx, uint32_t* host_out) {
     return cudaStreamSynchronize(ctx->stream) == cudaSuccess ? OMSE_OK : OMSE_ECUDA;
 }
 
+int omse_read_evaluations(omse_ctx* ctx, uint64_t* host_out) {
+    if (!ctx || !host_out) return OMSE_EINVAL;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return OMSE_ECUDA;
+    unsigned long long v = 0;
+    if (cudaMemcpyAsync(&v, &ctx->ws->evals, sizeof(v), cudaMemcpyDeviceToHost, ctx->stream) != cudaSuccess) return OMSE_ECUDA;
+    if (cudaMemsetAsync(&ctx->ws->evals, 0, sizeof(v), ctx->stream) != cudaSuccess) return OMSE_ECUDA;
+    if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return OMSE_ECUDA;
+    *host_out = v;
+    return OMSE_OK;
+}
+
 int omse_quantize_weights(omse_ctx* ctx, const float* d_w, int64_t n_kernels, int64_t kernel_len, int bits,
                           int is_signed, const omse_grid* grid, float* d_alpha, float* d_sse,
                           int32_t* d_best_idx, int8_t* d_codes, uint8_t* d_packed) {
@@ -508,6 +521,7 @@ int omse_dual_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, int64
     if (blocks > cap) blocks = cap;
     if (blocks < 1) return OMSE_EINVAL;
     a.curve = reinterpret_cast<float*>(ctx->partials);
+    a.evals = &ctx->ws->evals;
     omse::dual_kernel<<<(unsigned)blocks, omse::kDualThreads, smem, ctx->stream>>>(a);
     return cudaGetLastError() == cudaSuccess ? OMSE_OK : OMSE_ECUDA;
 }
@@ -591,6 +605,7 @@ static int activation_impl(omse_ctx* ctx, const float* d_x, int64_t n, int bits,
     a.sse_out = d_sse;
     a.idx_out = d_best_idx;
     a.delta_out = d_delta;
+    a.evals = &ctx->ws->evals;
     a.status = &ctx->ws->status;
     cudaStream_t s = ctx->stream;
 

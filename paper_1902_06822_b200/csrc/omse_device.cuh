@@ -340,6 +340,14 @@ __device__ __forceinline__ int class_sat_count(int nb, int cpt, int tg, int c_sa
     return min(c, c_sat_row);
 }
 
+// Adds this thread's count of executed (element, candidate) evaluations to a global counter: one atomic per warp.
+__device__ __forceinline__ void report_evaluations(unsigned long long* counter, unsigned long long mine) {
+    if (!counter) return;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);
+    if ((threadIdx.x & 31) == 0 && mine) atomicAdd(counter, mine);
+}
+
 // Per-candidate constants of one thread for the grid of Section 3.4 on a tensor with max|x| = m.
 // Candidate c has alpha_c = fl(fl(c+1)*step), step = fl(fl(hi_frac*m)/fl(C)), all binary32.
 // In the sweep x/alpha_c is replaced by x*inv_c with inv_c within 2 ulp of 1/alpha_c: a code can

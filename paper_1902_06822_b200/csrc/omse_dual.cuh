@@ -30,6 +30,7 @@ struct DualArgs {
     int* best_idx;           // [S] flat pair index c*n_cand2+d, nullable
     signed char* codes;      // [2][N], nullable
     unsigned char* packed;   // [2][ceil(N/2)], nullable
+    unsigned long long* evals;   // executed (element, pair, first code) evaluations (instrumentation), nullable
     float* curve;            // workspace: [gridDim.x][n_cand1*n_cand2] fp32 grid values of the block's current row
     unsigned int* status;
     int rows_per_unit;       // 2 when nibble packing needs an even element count per unit (odd K)
@@ -79,6 +80,7 @@ __global__ void __launch_bounds__(kDualThreads) dual_kernel(const DualArgs a) {
     const float half_range2 = fmaxf(fhi2, -flo2) + 0.5f;
     const int n_levels = a.hi1 - a.lo1 + 1;
     unsigned int st = 0;
+    unsigned long long ev = 0ull;
 
     for (long long unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
         for (int ru = 0; ru < a.rows_per_unit; ++ru) {
@@ -127,6 +129,7 @@ __global__ void __launch_bounds__(kDualThreads) dual_kernel(const DualArgs a) {
                     const int w = (int)(half_range2 * fminf(ratio, 16.f) * 1.0001f) + 2;
                     const bool full = !(ratio <= 16.f) || 2 * w + 1 >= n_levels;
                     const int n_t = full ? n_levels : 2 * w + 1;
+                    ev += (unsigned long long)k * (unsigned long long)(2 * ((n_t + 1) / 2)) * kDualDpt;
                     for (int i = 0; i < k; ++i) {
                         const float x = xs[i];
                         const float t0 = full ? (float)a.lo1 : rintf(x * inv1) - (float)w;
@@ -280,6 +283,7 @@ __global__ void __launch_bounds__(kDualThreads) dual_kernel(const DualArgs a) {
         }
     }
     if (st) atomicOr(a.status, st);
+    report_evaluations(a.evals, ev);
 }
 
 }  // namespace omse

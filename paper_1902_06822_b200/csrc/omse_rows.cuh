@@ -41,6 +41,7 @@ struct RowArgs {
     int lo[4], hi[4];           // grid bounds per quantized tensor (Section 3.1)
     float* sse_history;         // [n_sweeps][n_tensors][S] error after every update of Algorithm 1, nullable (single tensor launches)
     unsigned int* status;
+    unsigned long long* evals;  // executed (element, candidate) evaluations, summed over the launch (instrumentation), nullable
     int groups;                 // element groups per block
     int tg;                     // threads per group (multiple of 32); candidate c = slot*tg + t
     int keep_x0;                // n_sweeps > 1: keep the original row next to the residual
@@ -190,7 +191,7 @@ __device__ void partition_row(const RowSmem& s, int k, const GridSetup& g, int t
 // The quantization mapping phi of Section 3.4 on the row held in s.xs (k elements, k4 float4s).
 template <int CPT>
 __device__ PhiOut phi_block(const RowArgs& a, const RowSmem& s, int k, int k4, float flo, float fhi,
-                             const float (&rcp)[CPT]) {
+                             const float (&rcp)[CPT], unsigned long long& ev) {
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int grp = tid / a.tg, t = tid - grp * a.tg;
     const float4* xs4 = reinterpret_cast<const float4*>(s.xs);
@@ -243,6 +244,7 @@ __device__ PhiOut phi_block(const RowArgs& a, const RowSmem& s, int k, int k4, f
             int ncl_b = (class_sat_count(b, CPT, a.tg, g.c_sat, flo, fhi) - warp_t0 + a.tg - 1) / a.tg;
             ncl_b = max(0, min(CPT, ncl_b));
             sweep_dispatch<CPT>(b, ncl_b, xb4, beg4, end4, inv2, na2, dacc, kMagic + flo, kMagic + fhi);
+            ev += (unsigned long long)(end4 - beg4) * 4ull * (unsigned long long)b;
         }
         if (grp == 0) {
 #pragma unroll
@@ -251,7 +253,7 @@ __device__ PhiOut phi_block(const RowArgs& a, const RowSmem& s, int k, int k4, f
     } else {
         const int beg4 = (int)(((long long)k4 * grp) / a.groups);
         const int end4 = (int)(((long long)k4 * (grp + 1)) / a.groups);
-        sweep_dispatch<CPT>(ncl, xs4, beg4, end4, inv2, na2, dacc, kMagic + flo, kMagic + fhi);
+        sweep_dispatch<CPT>(ncl, xs4, beg4, end4, inv2, na2, dacc, kMagic + flo, kMagic + fhi);        ev += (unsigned long long)(end4 - beg4) * 4ull * CPT;
     }
 
     if (a.groups > 1) {
@@ -429,6 +431,7 @@ __global__ void __launch_bounds__(OMSE_ROWS_MAX_THREADS) rows_kernel(const RowAr
     s.seg = s.list + kListCap;
     s.misc = s.seg + 2 * (CPT + 1);
     unsigned int st = 0;
+    unsigned long long ev = 0ull;      // (element, candidate) evaluations this thread executed
 
     // 1/(c+1) for this thread's candidates: 1/alpha_c = (1/(c+1)) * (1/step) to within 2 ulp
     float rcp[CPT];
@@ -450,11 +453,11 @@ __global__ void __launch_bounds__(OMSE_ROWS_MAX_THREADS) rows_kernel(const RowAr
         }
         const RowTensor& T = *tp;
         if (T.small & 4) {
-            tiny_dispatch<CPT>(a, T, unit - T.unit_begin, smem_raw, st);
+            tiny_dispatch<CPT>(a, T, unit - T.unit_begin, smem_raw, st, ev);
             continue;
         }
         if (T.small) {
-            small_unit<CPT>(a, T, unit - T.unit_begin, smem_raw, rcp, st);
+            small_unit<CPT>(a, T, unit - T.unit_begin, smem_raw, rcp, st, ev);
             continue;
         }
         const int k = (int)T.K;
@@ -535,7 +538,7 @@ __global__ void __launch_bounds__(OMSE_ROWS_MAX_THREADS) rows_kernel(const RowAr
                         }
                         __syncthreads();
                     }
-                    PhiOut r = phi_block<CPT>(a, s, k, k4, flo, fhi, rcp);
+                    PhiOut r = phi_block<CPT>(a, s, k, k4, flo, fhi, rcp, ev);
                     if (r.degenerate) st |= 2u;
                     const double sse = emit_block(s, k, r.alpha, flo, fhi,
                                                   T.codes ? T.codes + (long long)j * n_total : nullptr,
@@ -561,6 +564,7 @@ __global__ void __launch_bounds__(OMSE_ROWS_MAX_THREADS) rows_kernel(const RowAr
         }
     }
     if (st) atomicOr(a.status, st);   // any thread that saw a flag reports it
+    report_evaluations(a.evals, ev);
     // ---- the last block to leave re-arms the ticket pair for the next launch (no block waits)
     if (tid == 0) {
         __threadfence();

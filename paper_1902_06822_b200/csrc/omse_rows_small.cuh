@@ -251,7 +251,7 @@ __device__ __forceinline__ float small_row_epilogue(const RowArgs& a, const RowT
 // element group (blockDim.x == a.tg) and a single quantized tensor per row.
 template <int CPT>
 __device__ void small_unit(const RowArgs& a, const RowTensor& T, long long unit_local, unsigned char* smem_raw,
-                           const float (&rcp)[CPT], unsigned int& st) {
+                           const float (&rcp)[CPT], unsigned int& st, unsigned long long& ev) {
     const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
     const int k = (int)T.K, kpad = (k + 3) & ~3, k4 = kpad >> 2;
     const int B = T.rows_per_unit;
@@ -459,6 +459,7 @@ __device__ void small_unit(const RowArgs& a, const RowTensor& T, long long unit_
                 while (i < stop) {
                     const int n = min(stop - i, kFlushEvery4 - pending);
                     sweep_accum_dispatch<CPT>(b, ncl_b, xb4, i, i + n, inv2, na2, acc2, kMagic + flo, kMagic + fhi);
+                    ev += (unsigned long long)n * 4ull * (unsigned long long)b;
                     i += n;
                     pending += n;
                     if (pending == kFlushEvery4) {
@@ -481,6 +482,7 @@ __device__ void small_unit(const RowArgs& a, const RowTensor& T, long long unit_
                 cvr[sl * a.tg + tid] = ok[sl] ? (float)v : INFINITY;
             }
         } else if (short_rows) {
+            ev += (unsigned long long)k4 * 4ull * CPT;
             float out[CPT];
             sweep_short_dispatch<CPT>(ncl, xr4, k4, inv2, na2, out, kMagic + flo, kMagic + fhi);
 #pragma unroll
@@ -490,6 +492,7 @@ __device__ void small_unit(const RowArgs& a, const RowTensor& T, long long unit_
 #pragma unroll
             for (int sl = 0; sl < CPT; ++sl) dacc[sl] = 0.0;
             sweep_dispatch<CPT>(ncl, xr4, 0, k4, inv2, na2, dacc, kMagic + flo, kMagic + fhi);
+            ev += (unsigned long long)k4 * 4ull * CPT;
 #pragma unroll
             for (int sl = 0; sl < CPT; ++sl) cvr[sl * a.tg + tid] = ok[sl] ? (float)dacc[sl] : INFINITY;
         }

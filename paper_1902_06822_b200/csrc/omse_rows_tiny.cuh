@@ -11,7 +11,7 @@ namespace omse {
 
 template <int KP>
 __device__ void tiny_unit(const RowArgs& a, const RowTensor& T, long long unit_local, unsigned char* smem_raw,
-                          unsigned int& st) {
+                          unsigned int& st, unsigned long long& ev) {
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int k = (int)T.K;
     const int B = T.rows_per_unit;                       // == blockDim.x
@@ -117,6 +117,7 @@ __device__ void tiny_unit(const RowArgs& a, const RowTensor& T, long long unit_l
                     b2i = c;
                 }
             }
+            ev += (unsigned long long)a.n_cand * (2ull * KP);
             if (b1i == 0x7fffffff) degenerate = true;    // every error Inf/NaN
         }
         if (degenerate) {
@@ -188,13 +189,13 @@ __device__ void tiny_unit(const RowArgs& a, const RowTensor& T, long long unit_l
 
 template <int CPT_UNUSED>
 __device__ __forceinline__ void tiny_dispatch(const RowArgs& a, const RowTensor& T, long long unit_local,
-                                              unsigned char* smem_raw, unsigned int& st) {
+                                              unsigned char* smem_raw, unsigned int& st, unsigned long long& ev) {
     const int k = (int)T.K;
-    if (k <= 8) tiny_unit<4>(a, T, unit_local, smem_raw, st);
-    else if (k <= 16) tiny_unit<8>(a, T, unit_local, smem_raw, st);
-    else if (k <= 24) tiny_unit<12>(a, T, unit_local, smem_raw, st);
-    else if (k <= 28) tiny_unit<14>(a, T, unit_local, smem_raw, st);
-    else tiny_unit<16>(a, T, unit_local, smem_raw, st);
+    if (k <= 8) tiny_unit<4>(a, T, unit_local, smem_raw, st, ev);
+    else if (k <= 16) tiny_unit<8>(a, T, unit_local, smem_raw, st, ev);
+    else if (k <= 24) tiny_unit<12>(a, T, unit_local, smem_raw, st, ev);
+    else if (k <= 28) tiny_unit<14>(a, T, unit_local, smem_raw, st, ev);
+    else tiny_unit<16>(a, T, unit_local, smem_raw, st, ev);
 }
 
 }  // namespace omse

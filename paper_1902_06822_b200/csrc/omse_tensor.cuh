@@ -39,6 +39,7 @@ struct TensorArgs {
     float* sse_out;
     int* idx_out;
     float* delta_out;       // offset mode: receives delta; nullptr = no offset
+    unsigned long long* evals;   // executed (element, candidate) evaluations (instrumentation), nullable
     unsigned int* status;
 };
 
@@ -170,6 +171,7 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
     const long long n_tiles = (n4_total + a.tile4 - 1) / a.tile4;
     const float4* x4 = reinterpret_cast<const float4*>(a.x);
     const int per_thread4 = a.tile4 / nthr;          // consecutive float4s staged by one thread (<= 4)
+    unsigned long long ev = 0ull;                    // evaluations this thread executed
     double skipped[CPT + 1];                         // squared sums per class over this block's tiles
 #pragma unroll
     for (int b = 0; b <= CPT; ++b) skipped[b] = 0.0;
@@ -280,6 +282,7 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
             int ncl_b = (class_sat_count(b, CPT, a.tg, g.c_sat, flo, fhi) - warp_t0 + a.tg - 1) / a.tg;
             ncl_b = max(0, min(CPT, ncl_b));
             sweep_dispatch<CPT>(b, ncl_b, tile4p, beg4, end4, inv2, na2, dacc, kMagic + flo, kMagic + fhi);
+            ev += (unsigned long long)(end4 - beg4) * 4ull * (unsigned long long)b;
         }
     }
     if (a.groups > 1) {
@@ -295,6 +298,7 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
                 for (int sl = 0; sl < CPT; ++sl) dacc[sl] += xg[((gg - 1) * CPT + sl) * a.tg + t];
         }
     }
+    report_evaluations(a.evals, ev);
     // ---- what each slot skipped in this block: classes 0..sl (block sums in fixed order)
     long long zero = 0;
     double run = 0.0;

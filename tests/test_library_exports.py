@@ -30,3 +30,21 @@ def test_header_limits_match_binding_constants():
                       ("OMSE_MAX_KERNEL_LEN_MULTISWEEP", binding.MAX_KERNEL_LEN_MULTISWEEP),
                       ("OMSE_MAX_TENSORS", binding.MAX_TENSORS)]:
         assert int(re.search(rf"#define {name}\s+(\d+)", hdr).group(1)) == val
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    """No fallback of any kind: without libomse.so the binding raises instead of computing elsewhere."""
+    import pytest
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(build, "LIB_PATH", str(tmp_path / "libomse.so"))
+    with pytest.raises(FileNotFoundError):
+        binding.load_library()
+
+
+def test_product_path_never_imports_the_oracle():
+    pkg = os.path.join(ROOT, "paper_1902_06822_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert "oracle" not in text.lower(), f

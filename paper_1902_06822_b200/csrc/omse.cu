@@ -693,6 +693,7 @@ __global__ void static_begin_kernel(StaticScratch* s) {
         s->tstate.step = 0.f;
         s->tstate.n_list = 0;
         s->tstate.list_overflow = 0;
+        s->tstate.polish_done = 0;
         s->tstate.key_min = 0x7fffffff;
         s->tstate.key_max = (int)0x80000000;
         s->tstate.delta = 0.f;

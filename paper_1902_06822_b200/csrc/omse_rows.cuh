@@ -336,6 +336,7 @@ __device__ PhiOut phi_block(const RowArgs& a, const RowSmem& s, int k, int k4, f
         if (sqq == 0) break;
         const float a_new = (float)(sxq / (double)sqq);
         if (!(a_new >= FLT_MIN) || !(a_new <= FLT_MAX)) break;
+        if (a_new == alpha) break;   // fixed point: further steps would repeat it exactly
         alpha = a_new;
     }
     out.alpha = alpha;

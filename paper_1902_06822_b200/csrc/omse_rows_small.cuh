@@ -174,6 +174,7 @@ __device__ __forceinline__ float small_row_epilogue(const RowArgs& a, const RowT
                 if (sqq == 0) break;
                 const float a_new = (float)(sxq / (double)sqq);
                 if (!(a_new >= FLT_MIN) || !(a_new <= FLT_MAX)) break;
+                if (a_new == alpha) break;   // fixed point: further steps would repeat it exactly
                 alpha = a_new;
             }
         }

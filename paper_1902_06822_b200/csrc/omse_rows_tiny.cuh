@@ -155,6 +155,7 @@ __device__ void tiny_unit(const RowArgs& a, const RowTensor& T, long long unit_l
                 if (sqq == 0) break;
                 const float a_new = (float)(sxq / (double)sqq);
                 if (!(a_new >= FLT_MIN) || !(a_new <= FLT_MAX)) break;
+                if (a_new == alpha) break;   // fixed point: further steps would repeat it exactly
                 alpha = a_new;
             }
         }

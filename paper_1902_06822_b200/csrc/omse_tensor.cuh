@@ -17,7 +17,8 @@ struct TensorState {          // lives in the context workspace
     float alpha;
     float step;
     int n_list;
-    int list_overflow;
+    int list_overflow;               // (unused)
+    int polish_done;                 // set when a polish step stops or reaches a fixed point: later steps return at once
     int list[kListCap];
     int key_min, key_max;                // offset mode: order-preserving integer keys of min and max of the tensor
     float delta;                         // offset subtracted from every element (0 without offset)
@@ -53,6 +54,7 @@ __global__ void tensor_init_kernel(TensorState* st) {
         st->step = 0.f;
         st->n_list = 0;
         st->list_overflow = 0;
+        st->polish_done = 0;
         st->key_min = 0x7fffffff;
         st->key_max = (int)0x80000000;
         st->delta = 0.f;
@@ -400,7 +402,7 @@ __global__ void __launch_bounds__(256) tensor_pass_kernel(const TensorArgs a) {
     if (MODE == 0 && n_list == 0) return;
     const float alpha_now = st->alpha;
     const float delta = st->delta;
-    if (MODE == 1 && !(alpha_now > 0.f)) return;
+    if (MODE == 1 && (!(alpha_now > 0.f) || st->polish_done)) return;
     double* part_d = a.partials;                                         // [grid][kListCap]
     long long* part_q = reinterpret_cast<long long*>(a.partials + (size_t)gridDim.x * kListCap);  // [grid]
     const long long stride = (long long)gridDim.x * blockDim.x;
@@ -495,10 +497,15 @@ __global__ void __launch_bounds__(256) tensor_pass_kernel(const TensorArgs a) {
             st->best_idx = best;
             st->alpha = __fmul_rn((float)(best + 1), st->step);
         } else if (MODE == 1) {
+            bool moved = false;
             if (tot_q != 0) {
                 const float a_new = (float)(tot_d[0] / (double)tot_q);
-                if (a_new >= FLT_MIN && a_new <= FLT_MAX) st->alpha = a_new;
+                if (a_new >= FLT_MIN && a_new <= FLT_MAX && a_new != st->alpha) {
+                    st->alpha = a_new;
+                    moved = true;
+                }
             }
+            if (!moved) st->polish_done = 1;   // stopped or fixed point: the remaining polish launches have nothing to do
         } else {
             *a.alpha_out = st->alpha;
             if (a.delta_out) *a.delta_out = st->delta;

@@ -33,7 +33,7 @@ N_CAND, BITS, REFINE, HI_FRAC = 1024, 4, 3, 1.0
 INSTR_PER_EVAL = 6            # reference FP32 sequence per (element, candidate): 3 fma + 2 min/max + 1 add
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the timed kernel, from the ncu capture summarised
 # in profiles/rows_kernel_resnet50_weight_set.md; set to None whenever the kernel changes after the capture
-NCU_TRAFFIC_BYTES = 109_463_808
+NCU_TRAFFIC_BYTES = 108_999_936
 E2E_CHUNKS = 12               # batched launches per end-to-end step (copies of later chunks overlap earlier searches)
 N_SM, LANES_PER_SM = 148, 128
 WORKLOAD = "resnet50_weight_set_54_tensors_25.5M_params_signed4bit_kernelwise_1024cand_3refine_packed"

@@ -49,6 +49,7 @@ struct Workspace {
     unsigned long long evals;       // executed evaluations since the last omse_read_evaluations
     omse::TensorState tstate;
     double curve[OMSE_MAX_CANDIDATES];
+    int list[OMSE_MAX_CANDIDATES];  // candidates of the per-tensor search that are re-scored in fp64
 };
 
 }  // namespace
@@ -126,8 +127,8 @@ int launch_rows(omse_ctx* ctx, omse::RowArgs& a, long long max_k, size_t smem_sm
     if (groups > k4 / 8) groups = k4 / 8;
     if (groups < 1) groups = 1;
     a.groups = groups;
-    // fixed part: reduction scratch, skipped sums, near-minimal list, class table, misc
-    const size_t fixed = (size_t)omse::kScratchDoubles * 8 + (size_t)cpt * 8 + omse::kListCap * 4 + 2 * (cpt + 1) * 4 + 8 * 4;
+    // fixed part: reduction scratch, skipped sums, class table, misc
+    const size_t fixed = (size_t)omse::kScratchDoubles * 8 + (size_t)cpt * 8 + 2 * (cpt + 1) * 4 + 8 * 4;
     auto smem_for = [&](int gr) {
         return (size_t)(a.keep_x0 ? 2 : 1) * k4 * 16 + (a.prune ? (size_t)k4 * 16 + (size_t)cpt * 16 : 0) +
                (size_t)(gr - 1) * cpt * a.tg * 8 + fixed;
@@ -596,9 +597,11 @@ static int activation_impl(omse_ctx* ctx, const float* d_x, int64_t n, int bits,
     const int cpt = cpt_for(a.n_cand);
     a.tg = (((a.n_cand + cpt - 1) / cpt) + 31) & ~31;
     a.groups = 256 / a.tg < 1 ? 1 : 256 / a.tg;
-    a.tile4 = 1024;
+    a.tile4 = 4 * a.groups * a.tg;   // every thread stages exactly four float4s of a tile
     a.st = &ctx->ws->tstate;
     a.partials = ctx->partials;
+    a.partial_doubles = (long long)(kPartialBytes / 8);
+    a.list = ctx->ws->list;
     a.curve = ctx->ws->curve;
     a.curve_out = d_sse_curve;
     a.alpha_out = d_alpha;
@@ -666,6 +669,7 @@ struct StaticScratch {
     unsigned int pad_[3];
     omse::TensorState tstate;
     double curve[OMSE_STATIC_MAX_CANDIDATES];
+    int list[OMSE_STATIC_MAX_CANDIDATES];
     double partials[kStaticPartialDoubles];
 };
 static_assert(sizeof(StaticScratch) <= OMSE_STATIC_SCRATCH_BYTES, "static scratch larger than documented");
@@ -760,9 +764,11 @@ extern "C" int omse_activation_scale_static(int device, void* cuda_stream, const
     const int cpt = cpt_for(a.n_cand);
     a.tg = (((a.n_cand + cpt - 1) / cpt) + 31) & ~31;
     a.groups = 256 / a.tg < 1 ? 1 : 256 / a.tg;
-    a.tile4 = 1024;
+    a.tile4 = 4 * a.groups * a.tg;   // every thread stages exactly four float4s of a tile
     a.st = &sc->tstate;
     a.partials = sc->partials;
+    a.partial_doubles = (long long)kStaticPartialDoubles;
+    a.list = sc->list;
     a.curve = sc->curve;
     a.curve_out = d_sse_curve;
     a.alpha_out = d_alpha;
@@ -773,8 +779,6 @@ extern "C" int omse_activation_scale_static(int device, void* cuda_stream, const
     static_begin_kernel<<<1, 32, 0, s>>>(sc);
     long long pass_grid = (n + 1023) / 1024;
     if (pass_grid > (long long)sd.n_sm * 8) pass_grid = (long long)sd.n_sm * 8;
-    const long long pass_cap = (long long)(kStaticPartialDoubles / (omse::kListCap + 1));
-    if (pass_grid > pass_cap) pass_grid = pass_cap;
     if (pass_grid < 1) pass_grid = 1;
     int n_blocks = 1;
     if (n > 0) {

@@ -27,7 +27,6 @@ constexpr float kMagic = 12582912.0f;   // 1.5 * 2^23
 #endif
 constexpr int kUnroll = OMSE_UNROLL;      // float4 loads per unrolled step of the sweep loop
 constexpr int kFlushEvery4 = OMSE_FLUSH4;   // float4 loads between folds of the fp32 partial sums into fp64
-constexpr int kListCap = 32;            // most near-minimal candidates re-scored in fp64
 constexpr double kRescoreBand = 4e-6;   // candidates within this relative band of the fp32 minimum are re-scored
 
 __device__ __forceinline__ u64 pack2(float a, float b) {

@@ -17,7 +17,7 @@ namespace omse {
 
 constexpr int kDualDpt = 4;        // alpha2 candidates per thread
 constexpr int kDualThreads = 256;
-constexpr int kDualListCap = 256;  // most near-minimal pairs re-scored with the full enumeration
+constexpr int kDualListCap = 256;  // near-minimal pairs listed at a time for re-scoring with the full enumeration
 
 struct DualArgs {
     const float* t;          // [S][K]
@@ -203,11 +203,10 @@ __global__ void __launch_bounds__(kDualThreads) dual_kernel(const DualArgs a) {
                 __syncthreads();
                 const int n_list = misc[0];
                 best_pair = bi;
-                if (n_list > 1 && n_list <= kDualListCap) {
+                if (n_list > 1) {
                     double best_sse = INFINITY;
                     best_pair = 0x7fffffff;
-                    for (int l = 0; l < n_list; ++l) {
-                        const int p = list[l];
+                    auto rescore = [&](int p) {      // full enumeration in the reference arithmetic, fp64 sum
                         float a1, a2;
                         dual_scales(m, a, p / a.n_cand2, p % a.n_cand2, a1, a2);
                         double ss = 0.0;
@@ -222,6 +221,23 @@ __global__ void __launch_bounds__(kDualThreads) dual_kernel(const DualArgs a) {
                         if (ss < best_sse || (ss == best_sse && p < best_pair)) {
                             best_sse = ss;
                             best_pair = p;
+                        }
+                    };
+                    if (n_list <= kDualListCap) {
+                        for (int l = 0; l < n_list; ++l) rescore(list[l]);
+                    } else {
+                        // more pairs in the band than the list holds: the same re-scoring, one window of
+                        // kDualListCap consecutive pairs at a time
+                        for (int base = 0; base < n_pairs_grid; base += kDualListCap) {
+                            __syncthreads();
+                            if (tid == 0) misc[0] = 0;
+                            __syncthreads();
+                            const int stop = min(base + kDualListCap, n_pairs_grid);
+                            for (int p = base + tid; p < stop; p += nthr)
+                                if ((double)curve[p] <= band) list[atomicAdd(&misc[0], 1)] = p;
+                            __syncthreads();
+                            const int n_win = misc[0];
+                            for (int l = 0; l < n_win; ++l) rescore(list[l]);
                         }
                     }
                 }

@@ -74,8 +74,7 @@ struct RowSmem {
     double* scratch;  // [kScratchDoubles] reductions
     double* skip;     // [CPT] squared sum of the elements a candidate slot does not evaluate
     int* seg;         // [2*(CPT+1)] first element and padded length of each magnitude class in xb
-    int* list;        // [kListCap] near-minimal candidates
-    int* misc;        // [8]: 0 list count; 1..4 nibble carried to the next row, per tensor
+    int* misc;        // [8]: 1..4 nibble carried to the next row, per tensor
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -283,28 +282,34 @@ __device__ PhiOut phi_block(const RowArgs& a, const RowSmem& s, int k, int k4, f
             bi = c;
         }
     }
-    if (tid == 0) s.misc[0] = 0;
-    block_argmin(bv, bi, s.scratch);   // contains __syncthreads: the zeroed counter is visible after it
+    block_argmin(bv, bi, s.scratch);
     if (bi == 0x7fffffff) return out;  // every error is Inf/NaN (non-finite input): same as no usable scale
     out.degenerate = false;
 
-    // ---- candidates within the fp32 noise band of the minimum are re-scored in fp64 with true division
+    // ---- every candidate within the fp32 noise band of the minimum is re-scored in fp64 with true division,
+    //      in increasing index order, however many there are (the block agrees on the next one by a reduction)
     const double band = bv * (1.0 + kRescoreBand);
+    int mine = 0;
 #pragma unroll
-    for (int sl = 0; sl < CPT; ++sl) {
-        if (dacc[sl] <= band) {
-            const int pos = atomicAdd(&s.misc[0], 1);
-            if (pos < kListCap) s.list[pos] = sl * a.tg + t;
-        }
-    }
-    __syncthreads();
-    const int n_list = s.misc[0];
+    for (int sl = 0; sl < CPT; ++sl) mine += (dacc[sl] <= band) ? 1 : 0;
+    const int holders = __syncthreads_count(mine > 0);
+    const int multi = __syncthreads_or(mine > 1);
     int best = bi;
-    if (n_list > 1 && n_list <= kListCap) {
+    if (holders > 1 || multi) {
         double best_sse = INFINITY;
         best = 0x7fffffff;
-        for (int l = 0; l < n_list; ++l) {
-            const int c = s.list[l];
+        int prev = -1;
+        for (;;) {
+            int c = 0x7fffffff;
+#pragma unroll
+            for (int sl = CPT - 1; sl >= 0; --sl) {
+                const int cc = sl * a.tg + t;
+                if (dacc[sl] <= band && cc > prev) c = cc;   // descending slots: the smallest index above prev stays
+            }
+            double cv = (double)c;
+            block_argmin(cv, c, s.scratch);
+            if (c == 0x7fffffff) break;
+            prev = c;
             const float ac = __fmul_rn((float)(c + 1), g.step);
             double ss = 0.0;
             long long zero = 0;
@@ -314,7 +319,7 @@ __device__ PhiOut phi_block(const RowArgs& a, const RowSmem& s, int k, int k4, f
                 ss += d * d;
             }
             block_sum2(ss, zero, s.scratch);
-            if (ss < best_sse || (ss == best_sse && c < best)) {
+            if (ss < best_sse) {   // increasing index: strict < keeps the lowest among equal errors
                 best_sse = ss;
                 best = c;
             }
@@ -428,8 +433,7 @@ __global__ void __launch_bounds__(OMSE_ROWS_MAX_THREADS) rows_kernel(const RowAr
     s.xg = reinterpret_cast<double*>(s.xb + (a.prune ? 4 * a.max_k4 + 4 * CPT : 0));
     s.scratch = s.xg + (size_t)(a.groups - 1) * CPT * a.tg;
     s.skip = s.scratch + kScratchDoubles;
-    s.list = reinterpret_cast<int*>(s.skip + CPT);
-    s.seg = s.list + kListCap;
+    s.seg = reinterpret_cast<int*>(s.skip + CPT);
     s.misc = s.seg + 2 * (CPT + 1);
     unsigned int st = 0;
     unsigned long long ev = 0ull;      // (element, candidate) evaluations this thread executed

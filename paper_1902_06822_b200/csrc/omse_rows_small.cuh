@@ -135,7 +135,7 @@ __device__ __forceinline__ float small_row_epilogue(const RowArgs& a, const RowT
                 cnt += (v.x <= band) + (v.y <= band) + (v.z <= band) + (v.w <= band);
             }
             cnt = warp_allsum(cnt);
-            if (cnt > 1 && cnt <= kListCap) {
+            if (cnt > 1) {   // every candidate in the band is re-scored, however many there are
                 double best_sse = INFINITY;
                 best = 0x7fffffff;
                 for (int c0 = 0; c0 < a.n_cand; c0 += 32) {

@@ -70,51 +70,69 @@ __device__ void tiny_unit(const RowArgs& a, const RowTensor& T, long long unit_l
 #pragma unroll
         for (int p = 0; p < KP; ++p) x2[p] = pack2(x[2 * p], x[2 * p + 1]);
 
-        // ---- the whole grid, serially: best and second-best fp32 error
-        float b1v = INFINITY, b2v = INFINITY;
+        // ---- the whole grid, serially: the three smallest fp32 errors (two with their indices)
+        const u64 M2 = pack2(kMagic, kMagic), NM2 = pack2(-kMagic, -kMagic);
+        const float clo = kMagic + flo, chi = kMagic + fhi;
+        auto sweep_error = [&](int c, float cf) -> float {   // fp32 error of candidate c on this row; cf = c + 1
+            const float ac = __fmul_rn(cf, g.step);
+            const float inv = g.tiny ? __fdiv_rn(1.0f, ac) : rcpt[c] * g.rstep;
+            const u64 inv2 = pack2(inv, inv), na2 = pack2(-ac, -ac);
+            u64 acc = 0ull, acc_b = 0ull;             // two accumulators: shorter dependency chain
+            if (c < g.c_sat) {      // candidates that may saturate on this row (divergence only near c_sat)
+#pragma unroll
+                for (int p = 0; p < KP; ++p) {
+                    float t0, t1;
+                    unpack2(fma2(x2[p], inv2, M2), t0, t1);
+                    t0 = fminf(fmaxf(t0, clo), chi);
+                    t1 = fminf(fmaxf(t1, clo), chi);
+                    const u64 e = fma2(na2, add2(pack2(t0, t1), NM2), x2[p]);
+                    if (p & 1) acc_b = fma2(e, e, acc_b);
+                    else acc = fma2(e, e, acc);
+                }
+            } else {
+#pragma unroll
+                for (int p = 0; p < KP; ++p) {
+                    const u64 e = fma2(na2, add2(fma2(x2[p], inv2, M2), NM2), x2[p]);
+                    if (p & 1) acc_b = fma2(e, e, acc_b);
+                    else acc = fma2(e, e, acc);
+                }
+            }
+            acc = add2(acc, acc_b);
+            float p0, p1;
+            unpack2(acc, p0, p1);
+            return (ac >= FLT_MIN) ? p0 + p1 : INFINITY;
+        };
+        auto exact_error = [&](int c) -> double {            // fp64 error with true division
+            const float ac = __fmul_rn((float)(c + 1), g.step);
+            double ss = 0.0;
+#pragma unroll
+            for (int i = 0; i < 2 * KP; ++i) {
+                if (i < k) {
+                    const double d = (double)x[i] - (double)ac * (double)code_of(x[i], ac, flo, fhi);
+                    ss += d * d;
+                }
+            }
+            return ss;
+        };
+        float b1v = INFINITY, b2v = INFINITY, b3v = INFINITY;
         int b1i = 0x7fffffff, b2i = 0x7fffffff;
         if (!degenerate) {
-            const u64 M2 = pack2(kMagic, kMagic), NM2 = pack2(-kMagic, -kMagic);
-            const float clo = kMagic + flo, chi = kMagic + fhi;
             float cf = 0.f;                               // c + 1 as a float (exact: n_cand <= 4096)
             for (int c = 0; c < a.n_cand; ++c) {
                 cf += 1.0f;
-                const float ac = __fmul_rn(cf, g.step);
-                const float inv = g.tiny ? __fdiv_rn(1.0f, ac) : rcpt[c] * g.rstep;
-                const u64 inv2 = pack2(inv, inv), na2 = pack2(-ac, -ac);
-                u64 acc = 0ull, acc_b = 0ull;             // two accumulators: shorter dependency chain
-                if (c < g.c_sat) {      // candidates that may saturate on this row (divergence only near c_sat)
-#pragma unroll
-                    for (int p = 0; p < KP; ++p) {
-                        float t0, t1;
-                        unpack2(fma2(x2[p], inv2, M2), t0, t1);
-                        t0 = fminf(fmaxf(t0, clo), chi);
-                        t1 = fminf(fmaxf(t1, clo), chi);
-                        const u64 e = fma2(na2, add2(pack2(t0, t1), NM2), x2[p]);
-                        if (p & 1) acc_b = fma2(e, e, acc_b);
-                        else acc = fma2(e, e, acc);
-                    }
-                    acc = add2(acc, acc_b);
-                } else {
-#pragma unroll
-                    for (int p = 0; p < KP; ++p) {
-                        const u64 e = fma2(na2, add2(fma2(x2[p], inv2, M2), NM2), x2[p]);
-                        if (p & 1) acc_b = fma2(e, e, acc_b);
-                        else acc = fma2(e, e, acc);
-                    }
-                    acc = add2(acc, acc_b);
-                }
-                float p0, p1;
-                unpack2(acc, p0, p1);
-                const float v = (ac >= FLT_MIN) ? p0 + p1 : INFINITY;
+                const float v = sweep_error(c, cf);
                 if (v < b1v) {          // ascending c: strict < keeps the lowest index
+                    b3v = b2v;
                     b2v = b1v;
                     b2i = b1i;
                     b1v = v;
                     b1i = c;
                 } else if (v < b2v) {
+                    b3v = b2v;
                     b2v = v;
                     b2i = c;
+                } else if (v < b3v) {
+                    b3v = v;
                 }
             }
             ev += (unsigned long long)a.n_cand * (2ull * KP);
@@ -124,19 +142,26 @@ __device__ void tiny_unit(const RowArgs& a, const RowTensor& T, long long unit_l
             st |= 2u;
         } else {
             best = b1i;
-            // ---- runner-up within the fp32 noise band: decide in fp64 with true division
-            if ((double)b2v <= (double)b1v * (1.0 + kRescoreBand)) {
-                double s1 = 0.0, s2 = 0.0;
-                const float a1 = __fmul_rn((float)(b1i + 1), g.step), a2 = __fmul_rn((float)(b2i + 1), g.step);
-#pragma unroll
-                for (int i = 0; i < 2 * KP; ++i) {
-                    if (i < k) {
-                        const double d1 = (double)x[i] - (double)a1 * (double)code_of(x[i], a1, flo, fhi);
-                        const double d2 = (double)x[i] - (double)a2 * (double)code_of(x[i], a2, flo, fhi);
-                        s1 += d1 * d1;
-                        s2 += d2 * d2;
+            // ---- candidates within the fp32 noise band of the minimum: decide in fp64 with true division
+            const double band = (double)b1v * (1.0 + kRescoreBand);
+            if ((double)b3v <= band) {
+                // three or more: walk the grid once more and re-score every candidate in the band
+                double best_sse = INFINITY;
+                best = 0x7fffffff;
+                float cf = 0.f;
+                for (int c = 0; c < a.n_cand; ++c) {
+                    cf += 1.0f;
+                    if ((double)sweep_error(c, cf) <= band) {
+                        const double ss = exact_error(c);
+                        if (ss < best_sse) {   // ascending c: strict < keeps the lowest index
+                            best_sse = ss;
+                            best = c;
+                        }
                     }
                 }
+                ev += (unsigned long long)a.n_cand * (2ull * KP);
+            } else if ((double)b2v <= band) {
+                const double s1 = exact_error(b1i), s2 = exact_error(b2i);
                 if (s2 < s1 || (s2 == s1 && b2i < b1i)) best = b2i;
             }
             // ---- polish

@@ -16,10 +16,9 @@ struct TensorState {          // lives in the context workspace
     int best_idx;
     float alpha;
     float step;
-    int n_list;
+    int n_list;                      // candidates to re-score in fp64 (0: the fp32 winner is the only one in the band)
     int list_overflow;               // (unused)
     int polish_done;                 // set when a polish step stops or reaches a fixed point: later steps return at once
-    int list[kListCap];
     int key_min, key_max;                // offset mode: order-preserving integer keys of min and max of the tensor
     float delta;                         // offset subtracted from every element (0 without offset)
 };
@@ -33,7 +32,9 @@ struct TensorArgs {
     int tg, groups;         // sweep block = groups*tg threads; candidate c = slot*tg + t
     int tile4;              // float4s per tile
     TensorState* st;
-    double* partials;       // sweep: [grid][n_cand]; passes: [grid][kListCap] doubles + [grid] int64
+    double* partials;       // sweep: [grid][n_cand]; passes: [blocks][listed candidates] doubles + [blocks] int64
+    long long partial_doubles;   // capacity of `partials`
+    int* list;              // [n_cand] candidates inside the fp32 noise band of the minimum (workspace)
     double* curve;          // [n_cand] summed error per candidate (workspace)
     double* curve_out;      // user copy, nullable
     float* alpha_out;
@@ -375,8 +376,7 @@ __global__ void __launch_bounds__(1024) tensor_finish_kernel(const TensorArgs a)
     const double band = bv * (1.0 + kRescoreBand);
     for (int c = threadIdx.x; c < a.n_cand; c += blockDim.x) {
         if (a.curve[c] <= band) {
-            const int pos = atomicAdd(&cnt, 1);
-            if (pos < kListCap) st->list[pos] = c;
+            a.list[atomicAdd(&cnt, 1)] = c;   // at most n_cand entries: the list holds them all
         }
     }
     __syncthreads();
@@ -384,60 +384,91 @@ __global__ void __launch_bounds__(1024) tensor_finish_kernel(const TensorArgs a)
         st->step = g.step;
         st->best_idx = bi;
         st->alpha = __fmul_rn((float)(bi + 1), g.step);
-        st->n_list = (cnt > 1 && cnt <= kListCap) ? cnt : 0;   // 0: the fp32 winner stands
+        st->n_list = cnt > 1 ? cnt : 0;   // a single candidate in the band needs no re-scoring
     }
 }
 
-// Grid-wide pass over the tensor in fp64 with true division.
+// [x/alpha]_Zp without a division on the common path.  t = fl(x*inv + M) rounds the exact product to the
+// nearest integer (ties to even); with inv = fl(1/alpha) the product is within 2^-24 relative of x/alpha, and
+// so is the IEEE quotient, so both round to the same integer unless the product lies within
+// (|integer| + 1) * 2^-21 of a half-integer: `ambiguous` reports that, and the caller then takes the division.
+// Returns M + code (the code sits in the low mantissa bits).
+__device__ __forceinline__ float magic_code(float x, float inv, float clo, float chi, bool& ambiguous) {
+    const float t = fmaf(x, inv, kMagic);
+    const float rq = t - kMagic;
+    const float delta = fmaf(x, inv, -rq);
+    ambiguous = fabsf(delta) > 0.5f - (fabsf(rq) + 1.0f) * 4.76837158203125e-7f;
+    return fminf(fmaxf(t, clo), chi);
+}
+
+// integer held by M + q as an int, and as a double without a conversion instruction
+__device__ __forceinline__ int magic_int(float tc) { return __float_as_int(tc) - 0x4B400000; }
+__device__ __forceinline__ double int_double(int q) {
+    return __hiloint2double(0x43380000 + (q >> 31), q) - 6755399441055744.0;   // (1.5*2^52 + q) - 1.5*2^52, exact
+}
+
+// Grid-wide pass over the tensor; sums in fp64, codes equal to those of the IEEE division (see magic_code).
 //   MODE 0 (rescore): squared error at each listed candidate; the last block picks the best.
 //   MODE 1 (refine):  <x,q> and <q,q> at st->alpha; the last block sets alpha <- <x,q>/<q,q>.
 //   MODE 2 (final):   squared error at st->alpha; the last block writes the outputs.
+// Every block keeps its partial sums in its own slot of `partials`; blocks without a slot (a long list of
+// candidates on a small scratch) leave at once and the others stride over the whole tensor.
 template <int MODE>
 __global__ void __launch_bounds__(256) tensor_pass_kernel(const TensorArgs a) {
     __shared__ double scratch[64];
     __shared__ bool is_last;
     TensorState* st = a.st;
     const float flo = (float)a.lo, fhi = (float)a.hi;
+    const float clo = kMagic + flo, chi = kMagic + fhi;
     const int n_list = MODE == 0 ? st->n_list : 1;
     if (MODE == 0 && n_list == 0) return;
     const float alpha_now = st->alpha;
     const float delta = st->delta;
     if (MODE == 1 && (!(alpha_now > 0.f) || st->polish_done)) return;
-    double* part_d = a.partials;                                         // [grid][kListCap]
-    long long* part_q = reinterpret_cast<long long*>(a.partials + (size_t)gridDim.x * kListCap);  // [grid]
-    const long long stride = (long long)gridDim.x * blockDim.x;
+    const int slot = MODE == 0 ? ((n_list + 3) & ~3) : 1;                  // doubles per block
+    const long long fit = a.partial_doubles / (slot + 1);
+    const unsigned int nblk = (long long)gridDim.x < fit ? gridDim.x : (unsigned int)fit;
+    if (blockIdx.x >= nblk) return;
+    double* part_d = a.partials;                                           // [nblk][slot]
+    long long* part_q = reinterpret_cast<long long*>(a.partials + (size_t)nblk * slot);   // [nblk]
+    const long long stride = (long long)nblk * blockDim.x;
     const long long tid0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     const long long n4 = a.n >> 2;
     const float4* x4 = reinterpret_cast<const float4*>(a.x);
 
     for (int l0 = 0; l0 < n_list; l0 += 4) {
-        float al[4];
+        float al[4], inv[4];
+        double ald[4];
         double acc[4] = {0.0, 0.0, 0.0, 0.0};
         long long sqq = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             if (MODE == 0) {
-                const int c = (l0 + j < n_list) ? st->list[l0 + j] : st->list[l0];
+                const int c = (l0 + j < n_list) ? a.list[l0 + j] : a.list[l0];
                 al[j] = __fmul_rn((float)(c + 1), st->step);
             } else {
                 al[j] = alpha_now;
             }
+            inv[j] = al[j] > 0.f ? __fdiv_rn(1.0f, al[j]) : 0.f;
+            ald[j] = (double)al[j];
         }
+        const int nj = MODE == 0 ? 4 : 1;
         auto element = [&](float x) {
-            if (MODE == 0) {
+            const double xd = (double)x;
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const double d = (double)x - (double)al[j] * (double)code_of(x, al[j], flo, fhi);
-                    acc[j] += d * d;
+            for (int j = 0; j < nj; ++j) {
+                bool amb;
+                float tc = magic_code(x, inv[j], clo, chi, amb);
+                if (amb) tc = kMagic + (float)(al[j] > 0.f ? code_of(x, al[j], flo, fhi) : 0);   // rare: the division decides
+                const int q = magic_int(tc);
+                const double qd = int_double(q);
+                if (MODE == 1) {
+                    sqq += q * q;
+                    acc[j] = fma(xd, qd, acc[j]);
+                } else {
+                    const double d = fma(-ald[j], qd, xd);
+                    acc[j] = fma(d, d, acc[j]);
                 }
-            } else if (MODE == 1) {
-                const int q = code_of(x, al[0], flo, fhi);
-                sqq += q * q;
-                acc[0] += (double)x * (double)q;
-            } else {
-                const int q = al[0] > 0.f ? code_of(x, al[0], flo, fhi) : 0;
-                const double d = (double)x - (double)al[0] * (double)q;
-                acc[0] += d * d;
             }
         };
 #pragma unroll 4
@@ -449,12 +480,11 @@ __global__ void __launch_bounds__(256) tensor_pass_kernel(const TensorArgs a) {
             element(v.w - delta);
         }
         for (long long i = (n4 << 2) + tid0; i < a.n; i += stride) element(a.x[i] - delta);
-        const int nj = MODE == 0 ? 4 : 1;
         for (int j = 0; j < nj; ++j) {
             long long q = sqq;
             block_sum2(acc[j], q, scratch);
             if (threadIdx.x == 0) {
-                part_d[(size_t)blockIdx.x * kListCap + l0 + j] = acc[j];
+                part_d[(size_t)blockIdx.x * slot + l0 + j] = acc[j];
                 if (MODE == 1) part_q[blockIdx.x] = q;
             }
         }
@@ -463,43 +493,40 @@ __global__ void __launch_bounds__(256) tensor_pass_kernel(const TensorArgs a) {
     __threadfence();
     if (threadIdx.x == 0) {
         const unsigned int tk = atomicAdd(&st->ticket, 1u);
-        is_last = (tk == gridDim.x - 1);
+        is_last = (tk == nblk - 1);
     }
     __syncthreads();
     if (!is_last) return;
     __threadfence();
-    const int nl = MODE == 0 ? ((n_list + 3) & ~3) : 1;
-    __shared__ double tot_d[kListCap];
-    __shared__ long long tot_q;
-    if (threadIdx.x < nl) {
-        double s = 0.0;
-        for (unsigned int b = 0; b < gridDim.x; ++b) s += __ldcg(&part_d[(size_t)b * kListCap + threadIdx.x]);
-        tot_d[threadIdx.x] = s;
+    double best_sse = INFINITY;     // MODE 0: this thread's best listed candidate
+    int best = 0x7fffffff;
+    double total = 0.0;             // MODE 1, 2: thread 0 sums the single column
+    long long total_q = 0;
+    if (MODE == 0) {
+        for (int l = threadIdx.x; l < n_list; l += blockDim.x) {
+            double s = 0.0;
+            for (unsigned int b = 0; b < nblk; ++b) s += __ldcg(&part_d[(size_t)b * slot + l]);
+            const int c = a.list[l];
+            if (s < best_sse || (s == best_sse && c < best)) {
+                best_sse = s;
+                best = c;
+            }
+        }
+        block_argmin(best_sse, best, scratch);
+    } else if (threadIdx.x == 0) {
+        for (unsigned int b = 0; b < nblk; ++b) total += __ldcg(&part_d[b]);
+        if (MODE == 1)
+            for (unsigned int b = 0; b < nblk; ++b) total_q += __ldcg(&part_q[b]);
     }
-    if (MODE == 1 && threadIdx.x == 32) {
-        long long q = 0;
-        for (unsigned int b = 0; b < gridDim.x; ++b) q += __ldcg(&part_q[b]);
-        tot_q = q;
-    }
-    __syncthreads();
     if (threadIdx.x == 0) {
         st->ticket = 0u;
         if (MODE == 0) {
-            double best_sse = INFINITY;
-            int best = 0x7fffffff;
-            for (int l = 0; l < n_list; ++l) {
-                const int c = st->list[l];
-                if (tot_d[l] < best_sse || (tot_d[l] == best_sse && c < best)) {
-                    best_sse = tot_d[l];
-                    best = c;
-                }
-            }
             st->best_idx = best;
             st->alpha = __fmul_rn((float)(best + 1), st->step);
         } else if (MODE == 1) {
             bool moved = false;
-            if (tot_q != 0) {
-                const float a_new = (float)(tot_d[0] / (double)tot_q);
+            if (total_q != 0) {
+                const float a_new = (float)(total / (double)total_q);
                 if (a_new >= FLT_MIN && a_new <= FLT_MAX && a_new != st->alpha) {
                     st->alpha = a_new;
                     moved = true;
@@ -509,7 +536,7 @@ __global__ void __launch_bounds__(256) tensor_pass_kernel(const TensorArgs a) {
         } else {
             *a.alpha_out = st->alpha;
             if (a.delta_out) *a.delta_out = st->delta;
-            *a.sse_out = (float)tot_d[0];
+            *a.sse_out = (float)total;
             if (a.idx_out) *a.idx_out = st->best_idx;
         }
     }

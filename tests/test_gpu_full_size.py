@@ -55,24 +55,31 @@ def test_resnet50_weight_set_every_row(gpu):
     assert gpu.ctx().omse_last_device_status() == 0
 
 
-@pytest.mark.parametrize("k,bits", [(27, 4), (25088, 2)])
-def test_sweep_cells_at_64m_elements_sampled_rows(gpu, k, bits):
+@pytest.mark.parametrize("k", [27, 576, 4608, 25088])
+def test_sweep_cells_at_64m_elements_sampled_rows(gpu, k):
+    """configs[4]: every (kernel length, bit width) cell at 2^26 elements, in the launch shape the benchmark
+    times; 2 % of the rows (first, last and the row holding the maximum included) checked against the oracle.
+    One generated tensor per kernel length serves the four bit widths."""
     w = synth.sweep_tensor(k, seed=5)
-    assert w.size > 67_000_000
-    alpha, sse, idx, q, pk = gpu.quantize_weights(w, bits, True, 1024, 1.0, 3, want_codes=True, want_packed=True)
-    assert np.array_equal(pk, orc.pack_int4(q))
-    rows = _sample_rows(w, 0.02 if k > 100 else 0.005, seed=k)
-    st = check_rows(w, alpha, sse, idx, q, None, bits, True, 1024, 1.0, 3, rows=rows)
-    assert st["idx_diff"] <= max(1, st["rows"] // 100) and st["alpha_bitwise"] >= 0.99, st
-    assert np.all(alpha > 0) and np.all(np.isfinite(sse))
-    lo, hi = -(1 << (bits - 1)), (1 << (bits - 1)) - 1
-    assert q.min() >= lo and q.max() <= hi
+    assert w.size > 67_000_000 and w.shape[0] == (1 << 26) // k
+    rows = _sample_rows(w, 0.02, seed=k)
+    for bits in (2, 3, 4, 8):
+        packed = bits <= 4
+        alpha, sse, idx, q, pk = gpu.quantize_weights(w, bits, True, 1024, 1.0, 3, want_codes=True, want_packed=packed)
+        if packed:
+            assert np.array_equal(pk, orc.pack_int4(q))
+        st = check_rows(w, alpha, sse, idx, q, None, bits, True, 1024, 1.0, 3, rows=rows)
+        assert st["idx_diff"] <= max(1, st["rows"] // 100) and st["alpha_bitwise"] >= 0.99, (bits, st)
+        assert np.all(alpha > 0) and np.all(np.isfinite(sse))
+        lo, hi = -(1 << (bits - 1)), (1 << (bits - 1)) - 1
+        assert q.min() >= lo and q.max() <= hi
+        del alpha, sse, idx, q, pk
 
 
 @pytest.mark.parametrize("k", [27, 576, 4608, 25088])
 @pytest.mark.parametrize("bits", [2, 3, 4, 8])
 def test_sweep_cells_reduced(gpu, k, bits):
-    s = {27: 20001, 576: 1201, 4608: 151, 25088: 21}[k]
+    s = {27: 20001, 576: 2401, 4608: 151, 25088: 21}[k]   # 576: enough rows for the batched short-row path
     w = synth.sweep_tensor(k, seed=5, n_kernels=s)
     alpha, sse, idx, q, pk = gpu.quantize_weights(w, bits, True, 1024, 1.0, 3, want_codes=True, want_packed=bits <= 4)
     rows = _sample_rows(w, 0.1 if k < 100 else 0.25, seed=bits)
@@ -101,23 +108,17 @@ def test_fc6_residual_two_tensors_sampled_rows(gpu):
     assert sse[1].sum() < 0.5 * sse[0].sum()        # a second tensor shrinks the error substantially
 
 
-def test_activation_tensor_51m_sampled_candidates(gpu):
-    """configs[2]: 64x256x56x56 post-ReLU tensor, unsigned 4-bit, 2048 candidates, one scale."""
+def test_activation_tensor_51m_full_curve(gpu):
+    """configs[2]: 64x256x56x56 post-ReLU tensor, unsigned 4-bit, 2048 candidates, one scale.  The oracle runs the
+    whole search (every candidate on every element); the library's curve, index, scale and error are compared."""
     x = synth.activation_tensor(seed=3)
     assert x.size == 51_380_224
     alpha, sse, idx, curve = gpu.activation_scale(x, 4, False, 2048, 1.0, 3)
-    m = float(x.max())
-    assert int(np.argmin(curve)) == idx                      # the argmin is a function of the curve ...
-    picks = sorted({0, 1, 7, 100, 511, 1024, 2047, idx, max(idx - 1, 0), min(idx + 1, 2047), max(idx - 2, 0),
-                    min(idx + 2, 2047)})
-    for c in picks:                                          # ... and the curve is the oracle's, point by point
-        ref = orc.sse_at(x, orc.candidate(m, 1.0, 2048, c), 4, False)
-        assert curve[c] == pytest.approx(ref, rel=2e-6), c
-    # no sampled neighbour beats the winner in the oracle's own arithmetic by more than a tie
-    best_ref = orc.sse_at(x, orc.candidate(m, 1.0, 2048, idx), 4, False)
-    for c in (idx - 2, idx - 1, idx + 1, idx + 2):
-        if 0 <= c < 2048:
-            assert orc.sse_at(x, orc.candidate(m, 1.0, 2048, c), 4, False) >= best_ref * (1 - 1e-6)
-    ref = orc.phi(x, 4, False, 2048, 1.0, 3, start_idx=idx, want_codes=False)
+    ref = orc.activation_scale(x, 4, False, 2048, 1.0, 3)
+    assert np.all(np.isfinite(ref.sse_curve)) and np.all(np.isfinite(curve))
+    np.testing.assert_allclose(curve, ref.sse_curve, rtol=2e-6)
+    if idx != ref.best_idx:          # another index only where the oracle's own errors tie to 1e-6
+        assert abs(ref.sse_curve[idx] - ref.sse_curve[ref.best_idx]) <= 1e-6 * ref.sse_curve[ref.best_idx]
+        ref = orc.phi(x, 4, False, 2048, 1.0, 3, start_idx=idx, want_codes=False)
     assert alpha == pytest.approx(ref.alpha, rel=RTOL)
     assert sse == pytest.approx(ref.sse, rel=RTOL)

@@ -52,20 +52,26 @@ def test_offset_rows_match_oracle(s, k, bits, n_cand):
         assert np.array_equal(pk, orc.pack_int4(q))
 
 
-@pytest.mark.parametrize("n", [5, 4097, 1_000_000])
-def test_offset_activation_scale_matches_oracle(n):
+@pytest.mark.parametrize("n,n_cand", [(5, 512), (4097, 512), (1_000_000, 512), (250_000, 600), (250_000, 1100),
+                                      (250_000, 1500), (250_000, 3000)])
+def test_offset_activation_scale_matches_oracle(n, n_cand):
     import torch
     import gpu_util
     x = synth.student_t3(n, seed=810, tensor_id=n % 89) * np.float32(0.5) + np.float32(2.0)
     d_x = torch.from_numpy(x).cuda()
     alpha, delta, sse = (torch.empty(1, device="cuda") for _ in range(3))
     idx = torch.empty(1, dtype=torch.int32, device="cuda")
-    gpu_util.ctx().omse_activation_scale_offset(d_x, n, 4, 512, 1.0, 3, alpha, delta, sse, idx)
+    curve = torch.empty(n_cand, dtype=torch.float64, device="cuda")
+    gpu_util.ctx().omse_activation_scale_offset(d_x, n, 4, n_cand, 1.0, 3, alpha, delta, sse, idx, curve)
     torch.cuda.synchronize()
-    ref = orc.offset_rows(x.reshape(1, -1), 4, 512, 1.0, 3)
+    ref = orc.offset_rows(x.reshape(1, -1), 4, n_cand, 1.0, 3)
     assert delta.item() == ref.delta[0] == x.min()
+    shifted = (x - ref.delta[0]).astype(np.float32)
+    ref_curve = orc.phi(shifted, 4, False, n_cand, 1.0, 0, want_codes=False, want_curve=True).sse_curve
+    np.testing.assert_allclose(curve.cpu().numpy(), ref_curve, rtol=2e-6)
     if idx.item() != ref.best_idx[0]:
-        ref = orc.offset_rows(x.reshape(1, -1), 4, 512, 1.0, 3, start_idx=np.array([idx.item()], np.int32))
+        assert abs(ref_curve[idx.item()] - ref_curve[ref.best_idx[0]]) <= TIE_RTOL * ref_curve[ref.best_idx[0]]
+        ref = orc.offset_rows(x.reshape(1, -1), 4, n_cand, 1.0, 3, start_idx=np.array([idx.item()], np.int32))
     assert alpha.item() == pytest.approx(ref.alpha[0], rel=RTOL)
     assert sse.item() == pytest.approx(ref.sse[0], rel=RTOL)
     # the plain call afterwards is unaffected by the offset state

@@ -154,8 +154,11 @@ def test_activation_scale_sizes(gpu, n):
     assert _check_activation(gpu, x, 4, False, 2048 if n > 1000 else 256, 3)
 
 
-@pytest.mark.parametrize("bits,signed,n_cand", [(4, True, 50), (8, False, 500), (2, False, 64), (3, True, 4096)])
+@pytest.mark.parametrize("bits,signed,n_cand", [(4, True, 50), (8, False, 500), (2, False, 64), (3, True, 4096),
+                                                (4, False, 600), (4, True, 1100), (3, False, 1500), (4, False, 3000),
+                                                (4, False, 33), (4, True, 129), (2, True, 700), (8, True, 2049)])
 def test_activation_scale_grids(gpu, bits, signed, n_cand):
+    """Every block shape of the per-tensor sweep: the thread count follows the candidate count (160 ... 512)."""
     x = synth.student_t3(250_000, seed=33, tensor_id=bits)
     if not signed:
         x = np.abs(x)

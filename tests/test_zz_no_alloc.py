@@ -44,7 +44,9 @@ def _both(x, bits, signed, n_cand, refine):
     return ref, got
 
 
-@pytest.mark.parametrize("n,bits,signed,n_cand", [(300_001, 4, False, 2048), (70_000, 3, True, 256), (5, 4, False, 50)])
+@pytest.mark.parametrize("n,bits,signed,n_cand", [(300_001, 4, False, 2048), (70_000, 3, True, 256), (5, 4, False, 50),
+                                                  (200_000, 4, False, 600), (200_000, 4, True, 1100),
+                                                  (200_000, 2, False, 1500)])
 def test_static_entry_point_matches_the_context_one_twice(n, bits, signed, n_cand):
     x = synth.relu_activations(n, seed=3, tensor_id=7) if not signed else synth.student_t3(n, seed=9)
     if n <= 8:
@@ -57,6 +59,15 @@ def test_static_entry_point_matches_the_context_one_twice(n, bits, signed, n_can
         np.testing.assert_allclose(curve, ref[3], rtol=2e-6)
         assert status == 0
     assert got[0][:3] == got[1][:3] and np.array_equal(got[0][3], got[1][3])   # second call starts clean
+    # ... and both entry points agree with the CPU oracle, not only with each other
+    from oracle import omse_oracle as orc
+    want = orc.activation_scale(x, bits, signed, n_cand, 1.0, 3)
+    alpha, sse, idx, curve, _ = got[1]
+    np.testing.assert_allclose(curve, want.sse_curve, rtol=2e-6)
+    if idx != want.best_idx:
+        assert abs(want.sse_curve[idx] - want.sse_curve[want.best_idx]) <= 1e-6 * want.sse_curve[want.best_idx]
+        want = orc.phi(x, bits, signed, n_cand, 1.0, 3, start_idx=idx, want_codes=False)
+    assert alpha == pytest.approx(want.alpha, rel=1e-5) and sse == pytest.approx(want.sse, rel=1e-5)
 
 
 def test_static_entry_point_clears_the_status_of_the_previous_call_and_rejects_oversize():

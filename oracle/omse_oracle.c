@@ -260,9 +260,18 @@ static void alg1_segment(const float *x, int64_t k, const int *bits, const int *
                          float hi_frac, int refine_iters, int n_tensors, int n_sweeps,
                          int64_t out_stride, float *alpha, double *sse, int32_t *best_idx,
                          int8_t *codes, int64_t code_stride, float *r, double *sse_sweeps,
-                         uint32_t *status)
+                         double eps, int32_t *sweeps_done, uint32_t *status)
 {   /* is_signed: one flag per quantized tensor; sse_sweeps (nullable): [n_sweeps][n_tensors] with stride
-     * out_stride, the error after every update, i.e. the convergence history of the while-loop */
+     * out_stride, the error after every update, i.e. the convergence history of the while-loop.
+     * eps >= 0: the while-condition of Algorithm 1.  The paper does not define its "convergence rate";
+     * here it is the relative decrease of the squared error over one sweep, (E_prev - E_cur)/E_prev
+     * with E the error after the last tensor's update and E_0 = ||T||^2 (all tensors zero); the loop
+     * ends after the first sweep whose rate is not above eps (tested as E_prev - E_cur > eps*E_prev),
+     * or after n_sweeps sweeps.  History entries of sweeps that did not run repeat the last error.
+     * eps < 0: exactly n_sweeps sweeps.  sweeps_done (nullable): sweeps that ran. */
+    double e_prev = 0.0;
+    for (int64_t e = 0; e < k; ++e) e_prev += (double)x[e] * (double)x[e];
+    int ran = 0;
     for (int j = 0; j < n_tensors; ++j) {
         alpha[j * out_stride] = 0.0f;
         memset(codes + j * code_stride, 0, (size_t)k);
@@ -283,11 +292,48 @@ static void alg1_segment(const float *x, int64_t k, const int *bits, const int *
             sse[j * out_stride] = s_j;
             if (sse_sweeps) sse_sweeps[((int64_t)sweep * n_tensors + j) * out_stride] = s_j;
         }
+        ran = sweep + 1;
+        if (eps >= 0.0) {
+            double e_cur = sse[(n_tensors - 1) * out_stride];
+            int go_on = (e_prev - e_cur) > eps * e_prev;
+            e_prev = e_cur;
+            if (!go_on) break;
+        }
     }
+    if (sse_sweeps)
+        for (int sweep = ran; sweep < n_sweeps; ++sweep)
+            for (int j = 0; j < n_tensors; ++j)
+                sse_sweeps[((int64_t)sweep * n_tensors + j) * out_stride] = sse[j * out_stride];
+    if (sweeps_done) *sweeps_done = ran;
 }
 
 /* Algorithm 1 kernel-wise with one signedness flag per quantized tensor and the error after every
  * update: sse_sweeps (nullable) is [n_sweeps][n_tensors][n_kernels]. */
+void omse_oracle_alg1_rows_eps(const float *t, int64_t n_kernels, int64_t kernel_len, const int *bits,
+                               const int *is_signed, int n_cand, float hi_frac, int refine_iters,
+                               int n_tensors, int max_sweeps, double eps, float *alpha, double *sse,
+                               int32_t *best_idx, int8_t *codes, double *sse_sweeps, int32_t *sweeps_done,
+                               uint32_t *status)
+{
+    /* layouts as omse_oracle_alg1_rows; sweeps_done [n_kernels] (nullable) */
+    int64_t n = n_kernels * kernel_len;
+    uint32_t st_all = 0;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 1) reduction(| : st_all)
+#endif
+    for (int64_t s = 0; s < n_kernels; ++s) {
+        uint32_t st = 0;
+        float *r = (float *)malloc(sizeof(float) * (size_t)kernel_len);
+        alg1_segment(t + s * kernel_len, kernel_len, bits, is_signed, n_cand, hi_frac, refine_iters,
+                     n_tensors, max_sweeps, n_kernels, alpha + s, sse + s, best_idx + s,
+                     codes + s * kernel_len, n, r, sse_sweeps ? sse_sweeps + s : NULL, eps,
+                     sweeps_done ? sweeps_done + s : NULL, &st);
+        free(r);
+        st_all |= st;
+    }
+    *status |= st_all;
+}
+
 void omse_oracle_alg1_rows(const float *t, int64_t n_kernels, int64_t kernel_len, const int *bits,
                            const int *is_signed, int n_cand, float hi_frac, int refine_iters,
                            int n_tensors, int n_sweeps, float *alpha, double *sse, int32_t *best_idx,
@@ -304,7 +350,7 @@ void omse_oracle_alg1_rows(const float *t, int64_t n_kernels, int64_t kernel_len
         float *r = (float *)malloc(sizeof(float) * (size_t)kernel_len);
         alg1_segment(t + s * kernel_len, kernel_len, bits, is_signed, n_cand, hi_frac, refine_iters,
                      n_tensors, n_sweeps, n_kernels, alpha + s, sse + s, best_idx + s,
-                     codes + s * kernel_len, n, r, sse_sweeps ? sse_sweeps + s : NULL, &st);
+                     codes + s * kernel_len, n, r, sse_sweeps ? sse_sweeps + s : NULL, -1.0, NULL, &st);
         free(r);
         st_all |= st;
     }
@@ -506,6 +552,204 @@ void omse_oracle_offset_rows(const float *w, int64_t n_kernels, int64_t kernel_l
         omse_oracle_offset_phi(w + s * kernel_len, kernel_len, bits, n_cand, hi_frac, refine_iters,
                                start_idx ? start_idx[s] : -1, &alpha[s], &delta[s], &sse[s], &best_idx[s],
                                codes ? codes + s * kernel_len : NULL, &st);
+        st_all |= st;
+    }
+    *status |= st_all;
+}
+
+/*
+ * Comparison solvers of Section 3.4 (the columns of the paper's table comparing quantization methods):
+ * other ways of choosing the scale alpha for the same objective ||T - alpha*[T/alpha]_Zp||^2.
+ *   solver 0, "uniform": the no-offset uniform quantizer of Section 3.1, alpha = max|T| / L with
+ *       L = 2^(p-1)-1 (signed range) or 2^p-1 (unsigned range); no search.
+ *   solver 1, "alternating": alternating optimisation started from the uniform scale: n_iter times
+ *       q = [T/alpha]_Zp, alpha = <T,q>/<q,q> (the least-squares scale for fixed codes).
+ *   solver 2, "golden": golden-section search for the minimum of the objective on the bracket
+ *       [0, hi_frac*max|T|].  The paper gives neither bracket nor stopping rule; here n_iter shrink
+ *       steps, all scales in binary32: with rho = 0.618034f the interior points are
+ *       x1 = b - rho*(b-a), x2 = a + rho*(b-a) (each operation rounded); if f(x1) <= f(x2) the
+ *       bracket becomes [a, x2] (equal values keep the smaller scale) else [x1, b]; one new
+ *       evaluation per step; the result is the interior point with the smaller error, x1 on
+ *       equal errors.  A scale below FLT_MIN has error +inf.
+ * After the solver, refine_iters further least-squares steps (0 for the plain columns), then the
+ * final codes and squared error, as in phi.  n_evals (nullable) receives the number of objective
+ * evaluations the solver made.
+ */
+void omse_oracle_solver_phi(const float *x, int64_t k, int bits, int is_signed, int solver, int n_iter,
+                            float hi_frac, int refine_iters, float *alpha, double *sse, int8_t *codes,
+                            int32_t *n_evals, uint32_t *status)
+{
+    int lo, hi;
+    uint32_t st = 0;
+    omse_oracle_grid_bounds(bits, is_signed, &lo, &hi);
+    float m = max_abs_of(x, k, &st);
+    float a = 0.0f;
+    int evals = 0;
+    if (solver == 0 || solver == 1) {
+        float levels = is_signed ? (float)((1 << (bits - 1)) - 1) : (float)((1 << bits) - 1);
+        a = m / levels;
+        if (solver == 1 && a >= FLT_MIN && a <= FLT_MAX) a = refine_from(x, k, a, lo, hi, n_iter);
+    } else {
+        const float rho = 0.618034f;
+        float lo_a = 0.0f, hi_a = hi_frac * m;
+        float d = hi_a - lo_a;
+        float t = rho * d;
+        float x1 = hi_a - t;
+        float x2 = lo_a + t;
+        double f1 = (x1 >= FLT_MIN && x1 <= FLT_MAX) ? sse_of(x, k, x1, lo, hi) : INFINITY;
+        double f2 = (x2 >= FLT_MIN && x2 <= FLT_MAX) ? sse_of(x, k, x2, lo, hi) : INFINITY;
+        evals = 2;
+        for (int it = 0; it < n_iter; ++it) {
+            if (f1 <= f2) {
+                hi_a = x2;
+                x2 = x1;
+                f2 = f1;
+                d = hi_a - lo_a;
+                t = rho * d;
+                x1 = hi_a - t;
+                f1 = (x1 >= FLT_MIN && x1 <= FLT_MAX) ? sse_of(x, k, x1, lo, hi) : INFINITY;
+            } else {
+                lo_a = x1;
+                x1 = x2;
+                f1 = f2;
+                d = hi_a - lo_a;
+                t = rho * d;
+                x2 = lo_a + t;
+                f2 = (x2 >= FLT_MIN && x2 <= FLT_MAX) ? sse_of(x, k, x2, lo, hi) : INFINITY;
+            }
+            ++evals;
+        }
+        a = (f1 <= f2) ? x1 : x2;
+        if (!(((f1 <= f2) ? f1 : f2) < INFINITY)) a = 0.0f;
+    }
+    if (n_evals) *n_evals = evals;
+    if (!(a >= FLT_MIN) || !(a <= FLT_MAX)) { /* no usable scale: same outputs as a degenerate phi */
+        double s = 0.0;
+        for (int64_t i = 0; i < k; ++i) s += (double)x[i] * (double)x[i];
+        *alpha = 0.0f;
+        *sse = s;
+        if (codes) memset(codes, 0, (size_t)k);
+        *status |= st | ORACLE_STATUS_DEGENERATE;
+        return;
+    }
+    a = refine_from(x, k, a, lo, hi, refine_iters);
+    *alpha = a;
+    *sse = sse_of(x, k, a, lo, hi);
+    if (codes)
+        for (int64_t i = 0; i < k; ++i) codes[i] = (int8_t)code_of(x[i], a, lo, hi);
+    *status |= st;
+}
+
+void omse_oracle_solver_rows(const float *w, int64_t n_kernels, int64_t kernel_len, int bits, int is_signed,
+                             int solver, int n_iter, float hi_frac, int refine_iters, float *alpha,
+                             double *sse, int8_t *codes, uint32_t *status)
+{
+    uint32_t st_all = 0;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 1) reduction(| : st_all)
+#endif
+    for (int64_t s = 0; s < n_kernels; ++s) {
+        uint32_t st = 0;
+        omse_oracle_solver_phi(w + s * kernel_len, kernel_len, bits, is_signed, solver, n_iter, hi_frac,
+                               refine_iters, &alpha[s], &sse[s], codes ? codes + s * kernel_len : NULL, NULL,
+                               &st);
+        st_all |= st;
+    }
+    *status |= st_all;
+}
+
+/*
+ * Quantization with offset (Section 3.1, first displayed scheme) with BOTH parameters searched:
+ * T^ = alpha*[(T - delta)/alpha]_Zp + delta on the unsigned range, minimising the squared error over a
+ * grid of offsets and, for each offset, the line-search grid of Section 3.4 on the shifted tensor.
+ * The paper fixes delta = min T and gives no search; this reading: with lo = min T, R = fl(max T - lo),
+ *     delta_d = fl(lo + fl(fl(d) * fl(fl(off_frac*R) / fl(n_delta)))),  d = 0 .. n_delta-1,
+ * (d = 0 is the paper's delta = min T), the shifted tensor is r_i = fl(T_i - delta_d) in binary32 and
+ * its candidates are phi's: n_cand scales in (0, hi_frac*max|r|].  The pair with the smallest
+ * error sum_i (r_i - alpha*[r_i/alpha]_Zp)^2 wins, lowest flat index d*n_cand + c on equal errors;
+ * then refine_iters least-squares steps on the scale (offset fixed), final codes and error of the
+ * shifted values.  start_flat >= 0 skips the search and starts from that flat index.
+ */
+void omse_oracle_affine_phi(const float *x, int64_t k, int bits, int n_cand, float hi_frac, int n_delta,
+                            float off_frac, int refine_iters, int start_flat, float *alpha, float *delta,
+                            double *sse, int32_t *best_idx, int8_t *codes, double *sse_curve, uint32_t *status)
+{
+    int lo, hi;
+    uint32_t st = 0;
+    omse_oracle_grid_bounds(bits, 0, &lo, &hi);
+    float tmin = INFINITY, tmax = -INFINITY;
+    for (int64_t i = 0; i < k; ++i) {
+        if (!(fabsf(x[i]) <= FLT_MAX)) {
+            st |= ORACLE_STATUS_NONFINITE;
+            continue;
+        }
+        if (x[i] < tmin) tmin = x[i];
+        if (x[i] > tmax) tmax = x[i];
+    }
+    if (!(tmin <= tmax)) tmin = tmax = 0.0f;
+    float range = tmax - tmin;
+    float dstep = (off_frac * range) / (float)n_delta;
+    float *r = (float *)malloc(sizeof(float) * (size_t)(k > 0 ? k : 1));
+    int best = -1;
+    double best_sse = INFINITY;
+    if (start_flat >= 0) {
+        best = start_flat;
+    } else {
+        for (int d = 0; d < n_delta; ++d) {
+            float dl = tmin + (float)d * dstep;
+            for (int64_t i = 0; i < k; ++i) r[i] = x[i] - dl;
+            uint32_t st_d = 0;
+            float m = max_abs_of(r, k, &st_d);
+            for (int c = 0; c < n_cand; ++c) {
+                float a = omse_oracle_candidate(m, hi_frac, n_cand, c);
+                double s = INFINITY;
+                if (a >= FLT_MIN && a <= FLT_MAX) s = sse_of(r, k, a, lo, hi);
+                if (sse_curve) sse_curve[(int64_t)d * n_cand + c] = s;
+                if (s < best_sse) {
+                    best_sse = s;
+                    best = d * n_cand + c;
+                }
+            }
+        }
+    }
+    int bd = best >= 0 ? best / n_cand : 0;
+    float dl = tmin + (float)bd * dstep;
+    for (int64_t i = 0; i < k; ++i) r[i] = x[i] - dl;
+    /* polish, final codes and error: phi on the shifted tensor started from the winning candidate */
+    omse_oracle_phi(r, k, bits, 0, n_cand, hi_frac, refine_iters, best >= 0 ? best % n_cand : 0, alpha, sse,
+                    best_idx, codes, NULL, &st);
+    if (best < 0 || *best_idx < 0) {
+        *best_idx = -1;
+        if (best < 0) { /* no usable pair at all: report the error of the tensor shifted by its minimum */
+            *alpha = 0.0f;
+            double s = 0.0;
+            for (int64_t i = 0; i < k; ++i) s += (double)r[i] * (double)r[i];
+            *sse = s;
+            if (codes) memset(codes, 0, (size_t)k);
+            st |= ORACLE_STATUS_DEGENERATE;
+        }
+    } else {
+        *best_idx = best;
+    }
+    *delta = dl;
+    *status |= st;
+    free(r);
+}
+
+void omse_oracle_affine_rows(const float *w, int64_t n_kernels, int64_t kernel_len, int bits, int n_cand,
+                             float hi_frac, int n_delta, float off_frac, int refine_iters,
+                             const int32_t *start_flat, float *alpha, float *delta, double *sse,
+                             int32_t *best_idx, int8_t *codes, uint32_t *status)
+{
+    uint32_t st_all = 0;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 1) reduction(| : st_all)
+#endif
+    for (int64_t s = 0; s < n_kernels; ++s) {
+        uint32_t st = 0;
+        omse_oracle_affine_phi(w + s * kernel_len, kernel_len, bits, n_cand, hi_frac, n_delta, off_frac,
+                               refine_iters, start_flat ? start_flat[s] : -1, &alpha[s], &delta[s], &sse[s],
+                               &best_idx[s], codes ? codes + s * kernel_len : NULL, NULL, &st);
         st_all |= st;
     }
     *status |= st_all;

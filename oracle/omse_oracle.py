@@ -72,6 +72,17 @@ def _load():
                                           C.c_float, C.c_int, C.c_int, C.c_int, f32p, f64p, i32p, i8p, f64p, u32p]
     lib.omse_oracle_offset_rows.argtypes = [f32p, C.c_int64, C.c_int64, C.c_int, C.c_int, C.c_float, C.c_int, i32p,
                                             f32p, f32p, f64p, i32p, i8p, u32p]
+    lib.omse_oracle_alg1_rows_eps.argtypes = [f32p, C.c_int64, C.c_int64, C.POINTER(C.c_int), C.POINTER(C.c_int),
+                                              C.c_int, C.c_float, C.c_int, C.c_int, C.c_int, C.c_double, f32p, f64p,
+                                              i32p, i8p, f64p, i32p, u32p]
+    lib.omse_oracle_solver_rows.argtypes = [f32p, C.c_int64, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int, C.c_float,
+                                            C.c_int, f32p, f64p, i8p, u32p]
+    lib.omse_oracle_solver_phi.argtypes = [f32p, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int, C.c_float, C.c_int,
+                                           f32p, f64p, i8p, i32p, u32p]
+    lib.omse_oracle_affine_rows.argtypes = [f32p, C.c_int64, C.c_int64, C.c_int, C.c_int, C.c_float, C.c_int,
+                                            C.c_float, C.c_int, i32p, f32p, f32p, f64p, i32p, i8p, u32p]
+    lib.omse_oracle_affine_phi.argtypes = [f32p, C.c_int64, C.c_int, C.c_int, C.c_float, C.c_int, C.c_float, C.c_int,
+                                           C.c_int, f32p, f32p, f64p, i32p, i8p, f64p, u32p]
     lib.omse_oracle_pack_int4.argtypes = [i8p, C.c_int64, u8p]
     lib.omse_oracle_unpack_int4.argtypes = [u8p, C.c_int64, C.c_int, i8p]
     _lib = lib
@@ -320,6 +331,117 @@ def offset_rows(w, bits=4, n_cand=256, hi_frac=1.0, refine_iters=3, start_idx=No
                                     _p(si, C.c_int32), _p(alpha, C.c_float), _p(delta, C.c_float),
                                     _p(sse, C.c_double), _p(idx, C.c_int32), _p(q, C.c_int8), C.byref(st))
     return OffsetResult(alpha, delta, sse, idx, q, st.value)
+
+
+SOLVER_UNIFORM, SOLVER_ALTERNATING, SOLVER_GOLDEN = 0, 1, 2
+
+
+@dataclass
+class SolverResult:
+    alpha: np.ndarray
+    sse: np.ndarray
+    codes: np.ndarray
+    status: int
+    n_evals: int = 0
+
+
+def solver_rows(w, solver, bits=4, is_signed=True, n_iter=20, hi_frac=1.0, refine_iters=0) -> SolverResult:
+    """Comparison solvers of Section 3.4 (uniform / alternating / golden-section), row by row."""
+    w = _f32(w)
+    S, K = w.shape
+    alpha, sse = np.empty(S, np.float32), np.empty(S, np.float64)
+    q = np.empty((S, K), np.int8)
+    st = C.c_uint32(0)
+    _load().omse_oracle_solver_rows(_p(w, C.c_float), S, K, bits, int(is_signed), solver, n_iter, _c32(hi_frac),
+                                    refine_iters, _p(alpha, C.c_float), _p(sse, C.c_double), _p(q, C.c_int8),
+                                    C.byref(st))
+    return SolverResult(alpha, sse, q, st.value)
+
+
+def solver_phi(x, solver, bits=4, is_signed=True, n_iter=20, hi_frac=1.0, refine_iters=0) -> SolverResult:
+    """One segment; also returns the number of objective evaluations the solver made."""
+    x = _f32(x).ravel()
+    a, s, n, st = C.c_float(), C.c_double(), C.c_int32(), C.c_uint32(0)
+    q = np.empty(x.size, np.int8)
+    _load().omse_oracle_solver_phi(_p(x, C.c_float), x.size, bits, int(is_signed), solver, n_iter, _c32(hi_frac),
+                                   refine_iters, C.byref(a), C.byref(s), _p(q, C.c_int8), C.byref(n), C.byref(st))
+    return SolverResult(a.value, s.value, q, st.value, n.value)
+
+
+def affine_rows(w, bits=4, n_cand=256, hi_frac=1.0, n_delta=8, off_frac=0.25, refine_iters=3,
+                start_flat=None) -> OffsetResult:
+    """Offset scheme of Section 3.1 with offset and scale both searched on grids, row by row;
+    best_idx is the flat index d*n_cand + c."""
+    w = _f32(w)
+    S, K = w.shape
+    alpha, delta = np.empty(S, np.float32), np.empty(S, np.float32)
+    sse, idx = np.empty(S, np.float64), np.empty(S, np.int32)
+    q = np.empty((S, K), np.int8)
+    st = C.c_uint32(0)
+    si = None if start_flat is None else np.ascontiguousarray(start_flat, dtype=np.int32)
+    _load().omse_oracle_affine_rows(_p(w, C.c_float), S, K, bits, n_cand, _c32(hi_frac), n_delta, _c32(off_frac),
+                                    refine_iters, _p(si, C.c_int32), _p(alpha, C.c_float), _p(delta, C.c_float),
+                                    _p(sse, C.c_double), _p(idx, C.c_int32), _p(q, C.c_int8), C.byref(st))
+    return OffsetResult(alpha, delta, sse, idx, q, st.value)
+
+
+def affine_phi(x, bits=4, n_cand=256, hi_frac=1.0, n_delta=8, off_frac=0.25, refine_iters=3, want_curve=False):
+    """One segment; returns (alpha, delta, sse, flat best index, codes, curve [n_delta, n_cand] or None)."""
+    x = _f32(x).ravel()
+    a, d, s, i, st = C.c_float(), C.c_float(), C.c_double(), C.c_int32(), C.c_uint32(0)
+    q = np.empty(x.size, np.int8)
+    curve = np.empty((n_delta, n_cand), np.float64) if want_curve else None
+    _load().omse_oracle_affine_phi(_p(x, C.c_float), x.size, bits, n_cand, _c32(hi_frac), n_delta, _c32(off_frac),
+                                   refine_iters, -1, C.byref(a), C.byref(d), C.byref(s), C.byref(i),
+                                   _p(q, C.c_int8), _p(curve, C.c_double), C.byref(st))
+    return a.value, d.value, s.value, i.value, q, curve
+
+
+def alg1_rows_eps(t, bits=(4, 4), is_signed=(True, True), n_cand=1024, hi_frac=1.0, refine_iters=3, max_sweeps=8,
+                  eps=1e-3):
+    """Algorithm 1 with its while-condition: sweeps go on while the relative decrease of the error over a
+    sweep exceeds eps (at most max_sweeps).  Returns (result, history [max_sweeps, n, S], sweeps_done [S])."""
+    t = _f32(t)
+    S, K = t.shape
+    n = len(bits)
+    b = (C.c_int * n)(*bits)
+    f = (C.c_int * n)(*[int(x) for x in is_signed])
+    alpha = np.zeros((n, S), np.float32)
+    sse = np.zeros((n, S), np.float64)
+    idx = np.zeros((n, S), np.int32)
+    q = np.zeros((n, S, K), np.int8)
+    hist = np.zeros((max_sweeps, n, S), np.float64)
+    done = np.zeros(S, np.int32)
+    st = C.c_uint32(0)
+    _load().omse_oracle_alg1_rows_eps(_p(t, C.c_float), S, K, b, f, n_cand, _c32(hi_frac), refine_iters, n,
+                                      max_sweeps, float(eps), _p(alpha, C.c_float), _p(sse, C.c_double),
+                                      _p(idx, C.c_int32), _p(q, C.c_int8), _p(hist, C.c_double), _p(done, C.c_int32),
+                                      C.byref(st))
+    return ResidualResult(alpha, sse, idx, q, st.value), hist, done
+
+
+@dataclass
+class KeyLayerResult:
+    first: list            # RowsResult per layer (single quantized tensor)
+    mse: np.ndarray        # [L] float64, from the fp32 per-kernel errors
+    is_key: np.ndarray     # [L] bool
+    second: dict           # layer index -> ResidualResult (two tensors) for the key layers
+    compression_ratio: float
+
+
+def key_layer_pipeline(layers, bits=4, is_signed=True, n_cand=1024, hi_frac=1.0, refine_iters=3,
+                       tau=8e-5) -> KeyLayerResult:
+    """Section 3.5 end to end on a list of 2-D weight arrays: quantize every layer, MSE per layer, layers with
+    MSE > tau get a second quantized tensor (the residual scheme, one sweep), compression ratio of the result.
+    Only an ordering of calls to the functions above."""
+    first = [quantize_rows(w, bits, is_signed, n_cand, hi_frac, refine_iters) for w in layers]
+    mse = np.array([layer_mse(r.sse.astype(np.float32), w.shape[1]) for r, w in zip(first, layers)])
+    is_key = mse > float(np.float32(tau))
+    second = {l: residual_rows(layers[l], (bits, bits), is_signed, n_cand, hi_frac, refine_iters, 1)
+              for l in np.nonzero(is_key)[0]}
+    cr = compression_ratio([w.shape[0] for w in layers], [w.shape[1] for w in layers], [bits] * len(layers),
+                           [2 if k else 1 for k in is_key])
+    return KeyLayerResult(first, mse, is_key, second, cr)
 
 
 def pack_int4(codes_) -> np.ndarray:

@@ -440,3 +440,191 @@ def test_offset_quantizer_pins():
     # (e) for skewed data the offset beats the signed grid of the same width (the extra level of Section 3.1)
     skew = (np.abs(x) - np.float32(0.3)).astype(np.float32)
     assert orc.offset_rows(skew, 3, 128, 1.0, 3).sse.sum() < orc.quantize_rows(skew, 3, True, 128, 1.0, 3).sse.sum()
+
+
+# ---------------------------------------------------------------- Section 3.4: the comparison solvers
+def test_uniform_and_alternating_solvers_by_hand():
+    """x = (1, 2, 3.5), signed 2-bit range {-2..1}, L = 1.  Uniform: alpha = 3.5, codes (0, 1, 1), error
+    1 + 1.5^2 + 0 = 3.25.  One least-squares step: alpha = (2 + 3.5)/2 = 2.75, which re-quantizes to the
+    same codes (1/2.75 = 0.36, 2/2.75 = 0.73, 3.5/2.75 = 1.27 saturates), so 2.75 is a fixed point with
+    error 1 + 0.75^2 + 0.75^2 = 2.125."""
+    x = np.array([[1.0, 2.0, 3.5]], np.float32)
+    u = orc.solver_rows(x, orc.SOLVER_UNIFORM, bits=2)
+    assert u.alpha[0] == np.float32(3.5) and u.codes.tolist() == [[0, 1, 1]] and u.sse[0] == pytest.approx(3.25)
+    for n_iter in (1, 2, 9):
+        a = orc.solver_rows(x, orc.SOLVER_ALTERNATING, bits=2, n_iter=n_iter)
+        assert a.alpha[0] == np.float32(2.75) and a.sse[0] == pytest.approx(2.125) and a.codes.tolist() == [[0, 1, 1]]
+    # unsigned 3-bit range: L = 7
+    y = np.array([[0.0, 7.0, 3.0]], np.float32)
+    assert orc.solver_rows(y, orc.SOLVER_UNIFORM, bits=3, is_signed=False).alpha[0] == np.float32(1.0)
+
+
+def test_alternating_solver_is_monotone_and_ends_at_a_least_squares_fixed_point():
+    w = synth.student_t3(8 * 200, seed=5).reshape(8, 200)
+    prev = orc.solver_rows(w, orc.SOLVER_UNIFORM, bits=4).sse
+    for n_iter in range(1, 30):
+        cur = orc.solver_rows(w, orc.SOLVER_ALTERNATING, bits=4, n_iter=n_iter)
+        assert np.all(cur.sse <= prev * (1 + 1e-12))      # each half-step solves its sub-problem exactly
+        prev = cur.sse
+    end, more = orc.solver_rows(w, orc.SOLVER_ALTERNATING, n_iter=200), orc.solver_rows(w, orc.SOLVER_ALTERNATING, n_iter=201)
+    assert np.array_equal(end.alpha, more.alpha)
+    q = end.codes.astype(np.float64)
+    ls = (w.astype(np.float64) * q).sum(1) / (q * q).sum(1)
+    np.testing.assert_allclose(end.alpha, ls, rtol=1e-6)   # the scale is the least-squares scale of its own codes
+    # the same steps started from a grid candidate are phi's polish: one candidate at max/L, R polish steps
+    one = orc.quantize_rows(w, 4, True, 1, 1.0 / 7, 5)
+    alt = orc.solver_rows(w, orc.SOLVER_ALTERNATING, bits=4, n_iter=5)
+    np.testing.assert_allclose(alt.alpha, one.alpha, rtol=1e-5)
+
+
+def test_golden_section_first_steps_and_unimodal_case():
+    rho = np.float32(0.618034)
+    x = synth.laplace(300, 0.05, seed=12)
+    m = np.float32(np.abs(x).max())
+    # no shrink step: the two interior points of [0, m] are m - rho*m and rho*m; the better one is returned
+    x1, x2 = np.float32(m - rho * m), np.float32(rho * m)
+    f1, f2 = orc.sse_at(x, x1, 4, True), orc.sse_at(x, x2, 4, True)
+    g0 = orc.solver_phi(x, orc.SOLVER_GOLDEN, n_iter=0)
+    assert g0.alpha == (x1 if f1 <= f2 else x2) and g0.n_evals == 2
+    # one shrink step keeps the half that holds the better point and adds one point inside it
+    g1 = orc.solver_phi(x, orc.SOLVER_GOLDEN, n_iter=1)
+    if f1 <= f2:      # bracket [0, x2]: new point x2 - rho*x2, old x1 stays
+        new = np.float32(x2 - np.float32(rho * x2))
+        cands = [(orc.sse_at(x, new, 4, True), new), (f1, x1)]
+    else:             # bracket [x1, m]: new point x1 + rho*(m - x1), old x2 stays
+        new = np.float32(x1 + np.float32(rho * np.float32(m - x1)))
+        cands = [(f2, x2), (orc.sse_at(x, new, 4, True), new)]
+    want = cands[0][1] if cands[0][0] <= cands[1][0] else cands[1][1]
+    assert g1.alpha == want and g1.n_evals == 3
+    # unimodal case with a known minimiser: every element equals v and the signed 2-bit range tops out at
+    # code 1, so the error is K*(v - alpha)^2 on (0, 2v): minimum at alpha = v, inside the bracket [0, 1.5v]
+    v = np.float32(0.8125)
+    row = np.full(40, v, np.float32)
+    for n_iter in (5, 10, 20, 30):
+        g = orc.solver_phi(row, orc.SOLVER_GOLDEN, bits=2, n_iter=n_iter, hi_frac=1.5)
+        width = 1.5 * float(v) * 0.618034 ** n_iter        # bracket length after n_iter steps
+        assert abs(g.alpha - float(v)) <= width + 1e-6 and g.n_evals == n_iter + 2
+        assert g.codes.tolist() == [1] * 40
+    # never better than the exact optimum, and close to it on a smooth curve
+    lo, hi = _bounds(4, True)
+    for seed in range(6):
+        t = synth.laplace(24, 1.0, seed=100 + seed)
+        best = exact_optimum(t, lo, hi, a_max=float(np.abs(t).max()))[0]
+        g = orc.solver_phi(t, orc.SOLVER_GOLDEN, n_iter=25)
+        assert g.sse >= best * (1 - 1e-9)
+
+
+def test_grid_search_is_the_best_of_the_four_solvers_on_average():
+    """Ordering the paper's comparison reports for the MSE itself: the dense grid with polish reaches the lowest
+    error; alternation from the uniform start improves on uniform but can stay in a local minimum."""
+    w = np.concatenate([synth.laplace(64 * 288, 0.06, seed=3).reshape(64, 288),
+                        synth.student_t3(64 * 288, seed=4).reshape(64, 288)])
+    uni = orc.solver_rows(w, orc.SOLVER_UNIFORM).sse
+    alt = orc.solver_rows(w, orc.SOLVER_ALTERNATING, n_iter=50).sse
+    gold = orc.solver_rows(w, orc.SOLVER_GOLDEN, n_iter=25).sse
+    grid = orc.quantize_rows(w, 4, True, 512, 1.0, 3).sse
+    assert np.all(alt <= uni * (1 + 1e-12))
+    assert grid.sum() < gold.sum() and grid.sum() < alt.sum() < uni.sum()
+    assert np.mean(grid <= np.minimum(alt, gold) * (1 + 1e-3)) > 0.9
+    assert np.any(grid < alt * 0.99)                      # alternation stuck in a local minimum somewhere
+
+
+# ---------------------------------------------------------------- Section 3.1: offset and scale both searched
+def test_affine_search_pins():
+    x = synth.student_t3(5 * 96, seed=17).reshape(5, 96)
+    # (a) a single offset on the grid is delta = min: the offset scheme
+    one = orc.affine_rows(x, 4, 64, 1.0, n_delta=1, off_frac=0.25, refine_iters=2)
+    off = orc.offset_rows(x, 4, 64, 1.0, 2)
+    assert np.array_equal(one.alpha, off.alpha) and np.array_equal(one.codes, off.codes)
+    assert np.array_equal(one.delta, off.delta) and np.array_equal(one.best_idx, off.best_idx)
+    # (b) delta = min stays on the grid (d = 0), so more offsets can only lower the grid error
+    g1 = orc.affine_rows(x, 4, 64, 1.0, n_delta=1, refine_iters=0)
+    g8 = orc.affine_rows(x, 4, 64, 1.0, n_delta=8, off_frac=0.25, refine_iters=0)
+    assert np.all(g8.sse <= g1.sse) and np.any(g8.sse < g1.sse * 0.9)     # heavy tails: clipping the low end pays
+    assert np.all(g8.best_idx // 64 < 8) and np.all(g8.delta >= x.min(1))
+    # (c) brute force over the whole (offset, scale) grid with shifted rows built here
+    for s in range(5):
+        lo, hi = np.float32(x[s].min()), np.float32(x[s].max())
+        dstep = np.float32(np.float32(np.float32(0.25) * np.float32(hi - lo)) / np.float32(8))
+        best = (np.inf, -1)
+        for d in range(8):
+            r = (x[s] - np.float32(lo + np.float32(np.float32(d) * dstep))).astype(np.float32)
+            m = float(np.abs(r).max())
+            for c in range(64):
+                e = orc.sse_at(r, orc.candidate(m, 1.0, 64, c), 4, False)
+                if e < best[0]:
+                    best = (e, d * 64 + c)
+        assert g8.best_idx[s] == best[1] and g8.sse[s] == pytest.approx(best[0], rel=1e-12)
+        d = best[1] // 64
+        assert g8.delta[s] == np.float32(lo + np.float32(np.float32(d) * dstep))
+    a, dl, sse, idx, codes, curve = orc.affine_phi(x[0], 4, 64, 1.0, 8, 0.25, 0, want_curve=True)
+    assert idx == int(np.argmin(curve.reshape(-1))) and sse == pytest.approx(curve.reshape(-1)[idx], rel=1e-12)
+    # (d) an exactly representable shift moves delta and nothing else
+    g = (np.random.default_rng(9).integers(-60, 60, (3, 80)) * 2.0 ** -6).astype(np.float32)
+    o1 = orc.affine_rows(g, 4, 32, 1.0, 4, 0.25, 2)
+    o2 = orc.affine_rows(g + np.float32(4.0), 4, 32, 1.0, 4, 0.25, 2)
+    assert np.array_equal(o1.alpha, o2.alpha) and np.array_equal(o1.codes, o2.codes)
+    assert np.array_equal(o2.delta, o1.delta + np.float32(4.0)) and np.array_equal(o1.best_idx, o2.best_idx)
+    # (e) the reported error is the reconstruction error of alpha*q + delta, codes in the unsigned range
+    full = orc.affine_rows(x, 4, 64, 1.0, 8, 0.25, 3)
+    rec = full.alpha[:, None].astype(np.float64) * full.codes + full.delta[:, None].astype(np.float64)
+    np.testing.assert_allclose(full.sse, np.sum((x.astype(np.float64) - rec) ** 2, axis=1), rtol=1e-4)
+    assert full.codes.min() >= 0 and full.codes.max() <= 15
+    # (f) per offset, the grid stays within the grid-resolution bound of the exact optimum for that offset
+    lo4, hi4 = _bounds(4, False)
+    t = synth.laplace(20, 1.0, seed=44)
+    a, dl, sse, idx, codes, curve = orc.affine_phi(t, 4, 64, 1.0, 4, 0.25, 0, want_curve=True)
+    tmin, tmax = np.float32(t.min()), np.float32(t.max())
+    dstep = np.float32(np.float32(np.float32(0.25) * np.float32(tmax - tmin)) / np.float32(4))
+    for d in range(4):
+        r = (t - np.float32(tmin + np.float32(np.float32(d) * dstep))).astype(np.float32)
+        m = float(np.abs(r).max())
+        e_star, a_star, q_star = exact_optimum(r, lo4, hi4, a_max=m)
+        step = m / 64
+        assert curve[d].min() >= e_star * (1 - 1e-9)
+        assert np.sqrt(curve[d].min()) <= np.sqrt(e_star) + 0.5 * step * np.linalg.norm(q_star) * (1 + 1e-6)
+
+
+# ---------------------------------------------------------------- Section 3.5: Algorithm 1's while-condition
+def test_algorithm_1_stops_when_the_error_stops_moving():
+    t = synth.student_t3(10 * 160, seed=23).reshape(10, 160)
+    fixed, hist_fixed = orc.alg1_rows(t, (3, 3), (True, True), 64, 1.0, 2, n_sweeps=6)
+    # eps = -1 in the C function is the fixed count; a huge eps stops after the first sweep
+    one, h1, d1 = orc.alg1_rows_eps(t, (3, 3), (True, True), 64, 1.0, 2, max_sweeps=6, eps=10.0)
+    first, _ = orc.alg1_rows(t, (3, 3), (True, True), 64, 1.0, 2, n_sweeps=1)
+    assert np.all(d1 == 1) and np.array_equal(one.alpha, first.alpha) and np.array_equal(one.codes, first.codes)
+    assert np.array_equal(h1[0], first.sse) and np.array_equal(h1[5], first.sse)    # later entries repeat the last error
+    # a moderate eps: every row stops exactly at the first sweep whose relative decrease is <= eps
+    eps = 0.02
+    res, hist, done = orc.alg1_rows_eps(t, (3, 3), (True, True), 64, 1.0, 2, max_sweeps=6, eps=eps)
+    e0 = np.sum(t.astype(np.float64) ** 2, axis=1)
+    assert done.min() >= 1 and done.max() <= 6 and len(set(done.tolist())) > 1
+    for s in range(10):
+        ends = np.concatenate([[e0[s]], hist_fixed[:, -1, s]])            # error after sweep 0 (nothing), 1, 2, ...
+        rate = (ends[:-1] - ends[1:]) / ends[:-1]
+        stop = next((i + 1 for i, r in enumerate(rate) if not r > eps), 6)
+        assert done[s] == stop
+        n = done[s]
+        assert np.array_equal(hist[:n, :, s], hist_fixed[:n, :, s])       # the sweeps that ran are the fixed-count ones
+        ref_n, _ = orc.alg1_rows(t[s:s + 1], (3, 3), (True, True), 64, 1.0, 2, n_sweeps=int(n))
+        assert np.array_equal(res.alpha[:, s], ref_n.alpha[:, 0]) and np.array_equal(res.codes[:, s], ref_n.codes[:, 0])
+    # eps = 0 runs until a sweep brings no decrease at all (or the cap)
+    z, hz, dz = orc.alg1_rows_eps(t, (3, 3), (True, True), 64, 1.0, 2, max_sweeps=6, eps=0.0)
+    assert np.all(dz >= done)
+
+
+def test_key_layer_pipeline_marks_by_tau_and_counts_the_second_tensor():
+    layers = [synth.laplace(16 * 72, 0.05, seed=1).reshape(16, 72), synth.student_t3(8 * 200, seed=2).reshape(8, 200),
+              synth.laplace(32 * 27, 0.3, seed=3).reshape(32, 27)]
+    probe = orc.key_layer_pipeline(layers, 4, True, 64, 1.0, 2, tau=0.0)
+    assert probe.is_key.all() and set(probe.second) == {0, 1, 2}
+    tau = float(np.sort(probe.mse)[1])                 # exactly one layer lies strictly above the middle MSE
+    out = orc.key_layer_pipeline(layers, 4, True, 64, 1.0, 2, tau=tau)
+    assert out.is_key.sum() == 1 and out.is_key[int(np.argmax(probe.mse))]
+    l = int(np.argmax(probe.mse))
+    assert np.array_equal(out.second[l].alpha[0], out.first[l].alpha)     # first tensor unchanged by the second pass
+    assert np.all(out.second[l].sse[1] <= out.second[l].sse[0])
+    n = [w.size for w in layers]
+    s = [w.shape[0] for w in layers]
+    want = sum((2 if i == l else 1) * (4 * n[i] + 32 * s[i]) for i in range(3)) / (32.0 * sum(n))
+    assert out.compression_ratio == pytest.approx(want, rel=1e-12)

@@ -13,10 +13,18 @@
  *   - Every pointer named d_* is DEVICE memory owned by the caller.  It must stay valid until
  *     the work queued by the call has finished on the context's stream.  The library keeps
  *     no pointer after the work completes.  float/int32 buffers must be 4-byte aligned,
- *     double buffers 8-byte aligned; there is no other alignment requirement.
+ *     double buffers 8-byte aligned; only omse_activation_scale* asks for more (16 bytes for
+ *     d_x).  Rows of odd length and views at odd offsets are therefore accepted as they are.
  *   - Pointers without the d_ prefix are HOST memory, read before the call returns.
  *   - Calls only enqueue work on the context's CUDA stream and return; nothing synchronises
- *     except omse_last_device_status() and omse_destroy().
+ *     except omse_last_device_status(), omse_read_evaluations() and omse_destroy().
+ *   - All work queued through one context shares that context's device workspace (work-unit
+ *     dispenser, search state, partial sums).  It must therefore be stream-ordered: after
+ *     omse_set_stream() the caller makes the new stream wait for the work already queued on the
+ *     old one (an event), otherwise two calls of one context may overlap on the GPU and corrupt
+ *     each other.  Use one context per stream for concurrent work.
+ *   - Every call makes the context's device current while it runs and restores the caller's
+ *     current device before it returns.
  *   - The return value is OMSE_OK or a negative omse_status.  Invalid arguments are
  *     rejected before anything is enqueued.  Data-dependent conditions (NaN/Inf in the
  *     input, an all-zero segment) never fail a call: they set bits in the device status
@@ -56,10 +64,12 @@ typedef enum {
 #define OMSE_MAX_TENSORS 4         /* n_tensors of omse_residual_quantize                           */
 #define OMSE_MAX_BATCH 1024        /* weight tensors per omse_quantize_weights_batched call         */
 
-/* The line-search grid of Section 3.4 ("a given grid"): n_cand scales spaced linearly in
- * (0, hi_frac*max|x|], candidate c (0-based) being fl(fl(c+1) * fl(fl(hi_frac*max|x|)/fl(n_cand)))
- * in binary32.  refine_iters is the number of closed-form polish steps
- * (alpha <- <x,q>/<q,q> with q = [x/alpha]_Zp) applied to the best candidate. */
+/* The grid of the line search of Section 3.4 (the paper fixes neither its range nor its spacing):
+ * n_cand scales spaced linearly in (0, hi_frac*max|x|], candidate c (0-based) being
+ * fl(fl(c+1) * fl(fl(hi_frac*max|x|)/fl(n_cand))) in binary32.  refine_iters is the number of
+ * closed-form polish steps (alpha <- <x,q>/<q,q> with q = [x/alpha]_Zp) applied to the best
+ * candidate; a step that reproduces the scale bit for bit ends the polish early (later steps would
+ * repeat it), as does <q,q> = 0 or a scale that is not a normal positive number. */
 typedef struct {
     int32_t n_cand;       /* 1 .. OMSE_MAX_CANDIDATES                    */
     float hi_frac;        /* > 0; 1.0 puts the last candidate at max|x| */
@@ -69,18 +79,21 @@ typedef struct {
 typedef struct omse_ctx omse_ctx;
 
 /* Creates a context bound to CUDA device `device` and to `cuda_stream` (a cudaStream_t, borrowed,
- * NULL = the legacy default stream).  Allocates a small device workspace (a few MB).  One context
- * must not be used from two host threads at once.  Returns OMSE_ECUDA if the device is absent. */
+ * NULL = the legacy default stream).  Allocates the device workspace (omse_workspace_bytes).  One
+ * context must not be used from two host threads at once; different contexts are independent.
+ * Returns OMSE_ECUDA if the device is absent. */
 int omse_create(omse_ctx** out, int device, void* cuda_stream);
 
 /* Waits for the stream, frees the workspace and the context. */
 int omse_destroy(omse_ctx* ctx);
 
-/* Replaces the stream later calls enqueue on (borrowed). */
+/* Replaces the stream later calls enqueue on (borrowed).  See the stream-ordering rule above. */
 int omse_set_stream(omse_ctx* ctx, void* cuda_stream);
 
-/* Bytes of device workspace the context holds (informational). */
-size_t omse_workspace_bytes(const omse_ctx* ctx);
+/* Bytes of device workspace a context allocates for calls of the given size (n_kernels rows of
+ * kernel_len elements, n_cand candidates, n_tensors quantized tensors per row).  Rows are searched
+ * on chip, so the answer is the same for every valid size (about 16.5 MB); 0 for invalid arguments. */
+size_t omse_workspace_bytes(int64_t n_kernels, int64_t kernel_len, int32_t n_cand, int32_t n_tensors);
 
 /*
  * Kernel-wise MMSE quantization of a weight tensor (Sections 3.3 and 3.4).
@@ -168,7 +181,7 @@ int omse_activation_scale_offset(omse_ctx* ctx, const float* d_x, int64_t n, int
 
 /*
  * omse_residual_quantize with one signedness flag per quantized tensor and the convergence history of
- * Algorithm 1 (Section 3.5: "until convergence").  is_signed: HOST array [n_tensors] (a non-negative
+ * Algorithm 1 (Section 3.5).  is_signed: HOST array [n_tensors] (a non-negative
  * tensor may take an unsigned first tensor and a signed tensor for its residual, whose rounding errors
  * have both signs).  d_sse_history (nullable): [n_sweeps][n_tensors][n_kernels] float, the squared
  * error after every update, in the order the updates are made; its last [n_tensors][n_kernels] block
@@ -178,6 +191,72 @@ int omse_alg1_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, int64
                        const int* bits, const int* is_signed, const omse_grid* grid, int n_tensors,
                        int n_sweeps, float* d_alpha, float* d_sse, float* d_sse_history,
                        int8_t* d_codes, uint8_t* d_packed);
+
+/*
+ * Algorithm 1 with its loop condition (Section 3.5, Algorithm 1: the sweeps go on while the convergence rate
+ * exceeds a threshold).  The paper does not define the rate; here it is the relative decrease of a kernel's
+ * squared error over one sweep, (E_prev - E_cur)/E_prev, E being the error after the last tensor's update and
+ * E_0 = ||T_k||^2.  Each kernel stops on its own after the first sweep whose rate is not above eps, or after
+ * max_sweeps sweeps.  d_sweeps_done (nullable) [n_kernels] int32: sweeps that ran; history entries of sweeps
+ * that did not run repeat the last error.  eps >= 0; everything else as in omse_alg1_quantize with
+ * n_sweeps = max_sweeps.
+ */
+int omse_alg1_quantize_converge(omse_ctx* ctx, const float* d_t, int64_t n_kernels, int64_t kernel_len,
+                                const int* bits, const int* is_signed, const omse_grid* grid, int n_tensors,
+                                int max_sweeps, float eps, float* d_alpha, float* d_sse, float* d_sse_history,
+                                int32_t* d_sweeps_done, int8_t* d_codes, uint8_t* d_packed);
+
+/*
+ * The other ways of choosing the scale that Section 3.4 compares the grid search with (the columns of its table
+ * of quantization methods), on the same objective and with the same outputs as omse_quantize_weights:
+ *   OMSE_SOLVER_GRID         the line search itself (identical to omse_quantize_weights; n_iter unused);
+ *   OMSE_SOLVER_UNIFORM      the no-offset uniform quantizer of Section 3.1, alpha = max|W_k| / L with L the
+ *                            largest code of the range (2^(bits-1)-1 signed, 2^bits-1 unsigned);
+ *   OMSE_SOLVER_ALTERNATING  alternating optimisation from that scale: n_iter least-squares steps
+ *                            alpha <- <x,q>/<q,q>, q = [x/alpha]_Zp;
+ *   OMSE_SOLVER_GOLDEN       golden-section search on the bracket [0, grid->hi_frac*max|W_k|] with n_iter
+ *                            shrink steps.  The paper gives neither bracket nor stopping rule; this library's:
+ *                            scales in binary32, rho = 0.618034f, interior points x1 = b - rho*(b-a) and
+ *                            x2 = a + rho*(b-a) (every operation rounded), the bracket becomes [a, x2] when
+ *                            f(x1) <= f(x2) and [x1, b] otherwise, the result is the interior point with the
+ *                            smaller error (x1 on equal errors), errors accumulated in binary64.
+ * grid->refine_iters further least-squares steps follow every solver (0 for the plain methods); grid->n_cand is
+ * used by the grid solver only.  d_best_idx receives 0 (-1 for a degenerate kernel) for the other solvers.
+ * 0 <= n_iter <= 1024.
+ */
+typedef enum {
+    OMSE_SOLVER_GRID = 0,
+    OMSE_SOLVER_UNIFORM = 1,
+    OMSE_SOLVER_ALTERNATING = 2,
+    OMSE_SOLVER_GOLDEN = 3
+} omse_solver;
+
+int omse_quantize_weights_solver(omse_ctx* ctx, const float* d_w, int64_t n_kernels, int64_t kernel_len, int bits,
+                                 int is_signed, int solver, int n_iter, const omse_grid* grid, float* d_alpha,
+                                 float* d_sse, int32_t* d_best_idx, int8_t* d_codes, uint8_t* d_packed);
+
+/*
+ * Quantization with offset (Section 3.1, first displayed scheme) with the offset searched as well as the scale.
+ * The paper fixes delta = min_i T_i; for a kernel with long tails on both sides the smallest error needs the low
+ * end clipped too.  With lo = min W_k, R = fl(max W_k - lo) the offsets are
+ *     delta_d = fl(lo + fl(fl(d) * fl(fl(off_frac*R)/fl(n_delta)))),   d = 0 .. n_delta-1
+ * (d = 0 is the paper's choice); for each, the shifted kernel fl(W_k - delta_d) goes through the line search of
+ * Section 3.4 on the unsigned range.  The (offset, scale) pair with the smallest error wins, lowest
+ * d*n_cand + c on equal errors; grid->refine_iters polish steps of the scale follow, the offset staying fixed.
+ * Outputs as omse_quantize_weights_offset; d_best_idx receives d*n_cand + c.  The kernel stays on chip while all
+ * offsets are tried, so the cost is n_delta line searches from one read of the tensor.
+ * Limits: 1 <= n_delta <= OMSE_MAX_OFFSETS, 0 <= off_frac <= 1, kernel_len <= OMSE_MAX_KERNEL_LEN_MULTISWEEP.
+ */
+#define OMSE_MAX_OFFSETS 64
+typedef struct {
+    int32_t n_delta; /* offsets on the grid                                  */
+    float off_frac;  /* they span [min, min + off_frac*(max-min))            */
+} omse_offset_grid;
+
+int omse_quantize_weights_affine(omse_ctx* ctx, const float* d_w, int64_t n_kernels, int64_t kernel_len, int bits,
+                                 const omse_grid* grid, const omse_offset_grid* offsets, float* d_alpha,
+                                 float* d_delta, float* d_sse, int32_t* d_best_idx, int8_t* d_codes,
+                                 uint8_t* d_packed);
 
 /*
  * Dual line search for two quantized tensors (Section 3.5, the special case n = 2, third displayed
@@ -209,8 +288,8 @@ int omse_dual_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, int64
                        uint8_t* d_packed);
 
 /*
- * Key layers (Section 3.5): "quantized layers with high MSE, or MSE bigger than some threshold tau" get a
- * second quantized tensor.  For each layer l this call sums the per-kernel squared errors that
+ * Key-layer rule of Section 3.5: a layer whose MSE exceeds a threshold tau gets a second quantized tensor.
+ * For each layer l this call sums the per-kernel squared errors that
  * omse_quantize_weights wrote (d_sse, [n_kernels] float) in binary64 in a fixed order, divides by the
  * layer's element count and compares with tau: d_mse[l] = sum / (n_kernels*kernel_len),
  * d_is_key[l] = (d_mse[l] > tau).  `layers` is a HOST array read before the call returns; d_mse
@@ -224,6 +303,29 @@ typedef struct {
 
 int omse_select_key_layers(omse_ctx* ctx, const omse_layer_error* layers, int n_layers, float tau,
                            double* d_mse, int32_t* d_is_key);
+
+/*
+ * The key-layer procedure of Section 3.5 in one call, with no host read in between:
+ *   1. every layer is quantized kernel-wise with one tensor (as omse_quantize_weights_batched on layers[l].first);
+ *   2. d_mse[l] and d_is_key[l] = (d_mse[l] > tau) as in omse_select_key_layers;
+ *   3. one more launch over all layers gives the layers with d_is_key[l] = 1 their second tensor: each kernel's
+ *      residual fl(W_k - alpha1*q1) is rebuilt on chip from the first scale and quantized the same way
+ *      (Algorithm 1, one sweep); blocks skip the other layers, whose second outputs stay untouched;
+ *      d_alpha2 / d_sse2 [n_kernels] (error after both tensors), d_codes2 / d_packed2 (nullable) are the second
+ *      tensor's outputs;
+ *   4. d_cr[0] (nullable, double) = compression ratio of the result, one or two tensors per layer.
+ * d_mse [n_layers] double and d_is_key [n_layers] int32 are required.  0 <= n_layers <= OMSE_MAX_BATCH.
+ */
+typedef struct {
+    omse_weight_tensor first;
+    float* d_alpha2;
+    float* d_sse2;
+    int8_t* d_codes2;
+    uint8_t* d_packed2;
+} omse_key_layer;
+
+int omse_quantize_key_layers(omse_ctx* ctx, const omse_key_layer* layers, int n_layers, int bits, int is_signed,
+                             const omse_grid* grid, float tau, double* d_mse, int32_t* d_is_key, double* d_cr);
 
 /*
  * Compression ratio (Section 3.5): size of the quantized model - bits[l] per code and one binary32

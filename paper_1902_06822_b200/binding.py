@@ -24,8 +24,11 @@ EXPORTS = [
     "omse_quantize_weights_batched", "omse_dual_quantize", "omse_select_key_layers", "omse_compression_ratio",
     "omse_alg1_quantize", "omse_read_evaluations", "omse_quantize_weights_offset", "omse_activation_scale_offset",
     "omse_activation_scale", "omse_residual_quantize", "omse_pack_int4", "omse_last_device_status",
-    "omse_status_string", "omse_activation_scale_static",
+    "omse_status_string", "omse_activation_scale_static", "omse_alg1_quantize_converge",
+    "omse_quantize_weights_solver", "omse_quantize_weights_affine", "omse_quantize_key_layers",
 ]
+SOLVER_GRID, SOLVER_UNIFORM, SOLVER_ALTERNATING, SOLVER_GOLDEN = 0, 1, 2, 3
+MAX_OFFSETS = 64
 
 
 class OmseGrid(C.Structure):
@@ -43,6 +46,15 @@ class OmseDualGrid(C.Structure):
 
 class OmseLayerError(C.Structure):
     _fields_ = [("d_sse", C.c_void_p), ("n_kernels", C.c_int64), ("kernel_len", C.c_int64)]
+
+
+class OmseOffsetGrid(C.Structure):
+    _fields_ = [("n_delta", C.c_int32), ("off_frac", C.c_float)]
+
+
+class OmseKeyLayer(C.Structure):
+    _fields_ = [("first", OmseWeightTensor), ("d_alpha2", C.c_void_p), ("d_sse2", C.c_void_p),
+                ("d_codes2", C.c_void_p), ("d_packed2", C.c_void_p)]
 
 
 class OmseError(RuntimeError):
@@ -66,7 +78,7 @@ def load_library() -> C.CDLL:
     lib.omse_create.argtypes = [C.POINTER(vp), i32, vp]
     lib.omse_destroy.argtypes = [vp]
     lib.omse_set_stream.argtypes = [vp, vp]
-    lib.omse_workspace_bytes.argtypes = [vp]
+    lib.omse_workspace_bytes.argtypes = [i64, i64, C.c_int32, C.c_int32]
     lib.omse_workspace_bytes.restype = C.c_size_t
     lib.omse_quantize_weights.argtypes = [vp, vp, i64, i64, i32, i32, C.POINTER(OmseGrid), vp, vp, vp, vp, vp]
     lib.omse_quantize_weights_batched.argtypes = [vp, C.POINTER(OmseWeightTensor), i32, i32, i32, C.POINTER(OmseGrid)]
@@ -78,6 +90,14 @@ def load_library() -> C.CDLL:
     lib.omse_activation_scale_offset.argtypes = [vp, vp, i64, i32, C.POINTER(OmseGrid), vp, vp, vp, vp, vp]
     lib.omse_alg1_quantize.argtypes = [vp, vp, i64, i64, C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(OmseGrid),
                                        i32, i32, vp, vp, vp, vp, vp]
+    lib.omse_alg1_quantize_converge.argtypes = [vp, vp, i64, i64, C.POINTER(C.c_int), C.POINTER(C.c_int),
+                                                C.POINTER(OmseGrid), i32, i32, C.c_float, vp, vp, vp, vp, vp, vp]
+    lib.omse_quantize_weights_solver.argtypes = [vp, vp, i64, i64, i32, i32, i32, i32, C.POINTER(OmseGrid), vp, vp, vp,
+                                                 vp, vp]
+    lib.omse_quantize_weights_affine.argtypes = [vp, vp, i64, i64, i32, C.POINTER(OmseGrid), C.POINTER(OmseOffsetGrid),
+                                                 vp, vp, vp, vp, vp, vp]
+    lib.omse_quantize_key_layers.argtypes = [vp, C.POINTER(OmseKeyLayer), i32, i32, i32, C.POINTER(OmseGrid), C.c_float,
+                                             vp, vp, vp]
     lib.omse_select_key_layers.argtypes = [vp, C.POINTER(OmseLayerError), i32, C.c_float, vp, vp]
     lib.omse_compression_ratio.argtypes = [C.POINTER(i64), C.POINTER(i64), C.POINTER(i32), C.POINTER(i32), i32]
     lib.omse_compression_ratio.restype = C.c_double
@@ -164,9 +184,9 @@ class Context:
         if rc != OK:
             raise OmseError(rc, "omse_set_stream")
 
-    @property
-    def workspace_bytes(self) -> int:
-        return int(load_library().omse_workspace_bytes(self._h))
+    @staticmethod
+    def workspace_bytes(n_kernels: int = 1, kernel_len: int = 1, n_cand: int = 1, n_tensors: int = 1) -> int:
+        return int(load_library().omse_workspace_bytes(n_kernels, kernel_len, n_cand, n_tensors))
 
     # -- the four calls of the library --------------------------------------------------------
     def omse_quantize_weights(self, w, n_kernels, kernel_len, bits, is_signed, n_cand, hi_frac, refine_iters,
@@ -247,6 +267,64 @@ class Context:
             _ptr(codes, torch.int8), _ptr(packed, torch.uint8))
         if rc != OK:
             raise OmseError(rc, "omse_alg1_quantize")
+
+    def omse_alg1_quantize_converge(self, t, n_kernels, kernel_len, bits, is_signed, n_cand, hi_frac, refine_iters,
+                                    max_sweeps, eps, alpha, sse, sse_history=None, sweeps_done=None, codes=None,
+                                    packed=None):
+        g = OmseGrid(n_cand, hi_frac, refine_iters)
+        b = (C.c_int * len(bits))(*bits)
+        f = (C.c_int * len(bits))(*[int(x) for x in is_signed])
+        rc = load_library().omse_alg1_quantize_converge(
+            self._h, _ptr(t, torch.float32), n_kernels, kernel_len, b, f, C.byref(g), len(bits), max_sweeps, eps,
+            _ptr(alpha, torch.float32), _ptr(sse, torch.float32), _ptr(sse_history, torch.float32),
+            _ptr(sweeps_done, torch.int32), _ptr(codes, torch.int8), _ptr(packed, torch.uint8))
+        if rc != OK:
+            raise OmseError(rc, "omse_alg1_quantize_converge")
+
+    def omse_quantize_weights_solver(self, w, n_kernels, kernel_len, bits, is_signed, solver, n_iter, n_cand, hi_frac,
+                                     refine_iters, alpha, sse, best_idx=None, codes=None, packed=None):
+        g = OmseGrid(n_cand, hi_frac, refine_iters)
+        rc = load_library().omse_quantize_weights_solver(
+            self._h, _ptr(w, torch.float32), n_kernels, kernel_len, bits, int(is_signed), solver, n_iter, C.byref(g),
+            _ptr(alpha, torch.float32), _ptr(sse, torch.float32), _ptr(best_idx, torch.int32),
+            _ptr(codes, torch.int8), _ptr(packed, torch.uint8))
+        if rc != OK:
+            raise OmseError(rc, "omse_quantize_weights_solver")
+
+    def omse_quantize_weights_affine(self, w, n_kernels, kernel_len, bits, n_cand, hi_frac, refine_iters, n_delta,
+                                     off_frac, alpha, delta, sse, best_idx=None, codes=None, packed=None):
+        g = OmseGrid(n_cand, hi_frac, refine_iters)
+        o = OmseOffsetGrid(n_delta, off_frac)
+        rc = load_library().omse_quantize_weights_affine(
+            self._h, _ptr(w, torch.float32), n_kernels, kernel_len, bits, C.byref(g), C.byref(o),
+            _ptr(alpha, torch.float32), _ptr(delta, torch.float32), _ptr(sse, torch.float32),
+            _ptr(best_idx, torch.int32), _ptr(codes, torch.int8), _ptr(packed, torch.uint8))
+        if rc != OK:
+            raise OmseError(rc, "omse_quantize_weights_affine")
+
+    def omse_quantize_key_layers(self, layers, bits, is_signed, n_cand, hi_frac, refine_iters, tau, mse, is_key,
+                                 cr=None):
+        """layers: sequence of dicts with the keys of omse_quantize_weights_batched plus alpha2, sse2 and
+        optionally codes2, packed2 (second tensor, written for key layers only)."""
+        g = OmseGrid(n_cand, hi_frac, refine_iters)
+        arr = (OmseKeyLayer * len(layers))()
+        for d, t in zip(arr, layers):
+            d.first.d_w = _ptr(t["w"], torch.float32)
+            d.first.n_kernels, d.first.kernel_len = t["n_kernels"], t["kernel_len"]
+            d.first.d_alpha = _ptr(t["alpha"], torch.float32)
+            d.first.d_sse = _ptr(t["sse"], torch.float32)
+            d.first.d_best_idx = _ptr(t.get("best_idx"), torch.int32)
+            d.first.d_codes = _ptr(t.get("codes"), torch.int8)
+            d.first.d_packed = _ptr(t.get("packed"), torch.uint8)
+            d.d_alpha2 = _ptr(t["alpha2"], torch.float32)
+            d.d_sse2 = _ptr(t["sse2"], torch.float32)
+            d.d_codes2 = _ptr(t.get("codes2"), torch.int8)
+            d.d_packed2 = _ptr(t.get("packed2"), torch.uint8)
+        rc = load_library().omse_quantize_key_layers(
+            self._h, arr, len(layers), bits, int(is_signed), C.byref(g), tau, _ptr(mse, torch.float64),
+            _ptr(is_key, torch.int32), _ptr(cr, torch.float64))
+        if rc != OK:
+            raise OmseError(rc, "omse_quantize_key_layers")
 
     def omse_quantize_weights_offset(self, w, n_kernels, kernel_len, bits, n_cand, hi_frac, refine_iters, alpha, delta,
                                      sse, best_idx=None, codes=None, packed=None):

@@ -54,6 +54,8 @@ struct Workspace {
 
 }  // namespace
 
+struct LaunchShape { int cpt, threads; size_t smem; int occ; };
+
 struct omse_ctx {
     int device;
     cudaStream_t stream;
@@ -61,7 +63,34 @@ struct omse_ctx {
     Workspace* ws;       // device
     double* partials;    // device, kPartialBytes
     omse::RowTensor* d_tensors;   // device, OMSE_MAX_BATCH descriptors of a batched launch
+    // per-context launch bookkeeping (a context is used by one host thread at a time, so no lock)
+    bool attr_rows[4], attr_tensor[4], attr_dual;   // opt-in shared-memory attribute set, per template instance
+    LaunchShape seen[16];                           // blocks per SM of the row-kernel launch shapes met so far
+    int n_seen, next_seen;
 };
+
+namespace {
+
+// Makes the context's device current for the duration of a call and puts the caller's device back afterwards.
+class DeviceScope {
+public:
+    explicit DeviceScope(int device) : prev_(-1), ok_(false) {
+        if (cudaGetDevice(&prev_) != cudaSuccess) prev_ = -1;
+        ok_ = (prev_ == device) || cudaSetDevice(device) == cudaSuccess;
+        if (prev_ == device) prev_ = -1;   // nothing to restore
+    }
+    ~DeviceScope() {
+        if (prev_ >= 0) cudaSetDevice(prev_);
+    }
+    bool ok() const { return ok_; }
+private:
+    int prev_;
+    bool ok_;
+};
+
+int cpt_slot(int cpt) { return cpt == 1 ? 0 : cpt == 2 ? 1 : cpt == 4 ? 2 : 3; }
+
+}  // namespace
 
 namespace {
 
@@ -90,25 +119,22 @@ void bounds(int bits, int is_signed, int* lo, int* hi) {
 
 template <int CPT>
 int launch_rows_t(omse_ctx* ctx, omse::RowArgs& a, size_t smem) {
-    static bool attr_set[64] = {};
-    if (!attr_set[ctx->device & 63]) {
+    if (!ctx->attr_rows[cpt_slot(CPT)]) {
         if (cudaFuncSetAttribute(omse::rows_kernel<CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess)
             return OMSE_ECUDA;
-        attr_set[ctx->device & 63] = true;
+        ctx->attr_rows[cpt_slot(CPT)] = true;
     }
     const int threads = a.groups * a.tg;
     // blocks per SM for this launch shape (remembered: the query costs more than a small launch)
-    struct Shape { int device, threads; size_t smem; int occ; };
-    static Shape seen[16];
-    static int n_seen = 0;
     int occ = 0;
-    for (int i = 0; i < n_seen; ++i)
-        if (seen[i].device == ctx->device && seen[i].threads == threads && seen[i].smem == smem) occ = seen[i].occ;
+    for (int i = 0; i < ctx->n_seen; ++i)
+        if (ctx->seen[i].cpt == CPT && ctx->seen[i].threads == threads && ctx->seen[i].smem == smem) occ = ctx->seen[i].occ;
     if (occ == 0) {
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, omse::rows_kernel<CPT>, threads, smem) != cudaSuccess || occ < 1)
             return OMSE_ECUDA;
-        seen[n_seen % 16] = Shape{ctx->device, threads, smem, occ};
-        if (n_seen < 16) ++n_seen;
+        ctx->seen[ctx->next_seen] = LaunchShape{CPT, threads, smem, occ};   // round robin once the table is full
+        ctx->next_seen = (ctx->next_seen + 1) % 16;
+        if (ctx->n_seen < 16) ++ctx->n_seen;
     }
     long long grid = (long long)ctx->n_sm * occ;
     if (grid > a.n_units) grid = a.n_units;
@@ -163,6 +189,8 @@ void fill_tensor(omse::RowTensor& t, const float* w, int64_t S, int64_t K, float
     t.codes = reinterpret_cast<signed char*>(codes);
     t.packed = packed;
     t.delta = nullptr;
+    t.prior_alpha = nullptr;
+    t.gate = nullptr;
     t.unit_begin = 0;
     t.rows_per_unit = (packed && (K & 1)) ? 2 : 1;
     t.small = 0;
@@ -183,11 +211,10 @@ bool misaligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3) !=
 
 template <int CPT>
 int launch_tensor_sweep_t(omse_ctx* ctx, omse::TensorArgs& a, size_t smem, int* n_blocks) {
-    static bool attr_set[64] = {};
-    if (!attr_set[ctx->device & 63]) {
+    if (!ctx->attr_tensor[cpt_slot(CPT)]) {
         if (cudaFuncSetAttribute(omse::tensor_sweep_kernel<CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess)
             return OMSE_ECUDA;
-        attr_set[ctx->device & 63] = true;
+        ctx->attr_tensor[cpt_slot(CPT)] = true;
     }
     const int threads = a.groups * a.tg;
     int occ = 0;
@@ -209,15 +236,24 @@ int launch_tensor_sweep_t(omse_ctx* ctx, omse::TensorArgs& a, size_t smem, int* 
 
 namespace {
 
+// How the scale of each row is found, for launches that do not use the default grid search with polish.
+struct ListMode {
+    int solver = 0, solver_iters = 0;   // comparison solvers of Section 3.4 (RowArgs::solver)
+    int n_delta = 0;                    // offsets searched per row (0: none)
+    float off_frac = 0.f;
+};
+
 // Launch for a list of weight tensors (bounds already set by the caller).
 int quantize_list(omse_ctx* ctx, std::vector<omse::RowTensor>& list, long long max_k, int bits, int is_signed,
-                  const omse_grid* grid) {
+                  const omse_grid* grid, const ListMode& mode = ListMode()) {
     if (list.empty()) return OMSE_OK;
-    if (cudaSetDevice(ctx->device) != cudaSuccess) return OMSE_ECUDA;
+    DeviceScope dev(ctx->device);
+    if (!dev.ok()) return OMSE_ECUDA;
     // Short rows are batched per work unit when the block is a single element group and the launch
     // still has a few work units per SM afterwards (otherwise one row per block fills the GPU better).
     size_t smem_small = 0;
-    if (single_group(grid->n_cand, max_k)) {
+    const bool plain = mode.solver == 0 && mode.n_delta == 0;   // the batched short-row paths implement the grid search only
+    if (plain && single_group(grid->n_cand, max_k)) {
         const int cpt = cpt_for(grid->n_cand);
         const int ncs = cpt * group_threads(grid->n_cand);
         long long units_if_small = 0;
@@ -228,7 +264,7 @@ int quantize_list(omse_ctx* ctx, std::vector<omse::RowTensor>& list, long long m
         // very short rows in large numbers: a thread per row, a block-sized batch of rows per unit
         const int threads = group_threads(grid->n_cand);
         for (auto& t : list) {
-            if (t.K > OMSE_TINY_K || t.S < 64ll * ctx->n_sm) continue;
+            if (t.K > OMSE_TINY_K || t.S < 64ll * ctx->n_sm || t.prior_alpha) continue;
             t.small = 4;
             t.rows_per_unit = threads;
             const size_t need = (size_t)((threads * t.K + 3) & ~3ll) * 4 + (size_t)((grid->n_cand + 3) & ~3) * 4 +
@@ -276,7 +312,12 @@ int quantize_list(omse_ctx* ctx, std::vector<omse::RowTensor>& list, long long m
     a.n_tensors = 1;
     a.n_sweeps = 1;
     bounds(bits, is_signed, &a.lo[0], &a.hi[0]);
-    a.keep_x0 = 0;
+    a.solver = mode.solver;
+    a.solver_iters = mode.solver_iters;
+    a.n_delta = mode.n_delta;
+    a.off_frac = mode.off_frac;
+    a.eps = -1.f;
+    a.keep_x0 = mode.n_delta > 0 ? 1 : 0;   // every offset is applied to the original row
     return launch_rows(ctx, a, max_k, smem_small);
 }
 
@@ -303,9 +344,11 @@ int omse_create(omse_ctx** out, int device, void* cuda_stream) {
     *out = nullptr;
     int n_dev = 0;
     if (cudaGetDeviceCount(&n_dev) != cudaSuccess || device < 0 || device >= n_dev) return OMSE_ECUDA;
-    if (cudaSetDevice(device) != cudaSuccess) return OMSE_ECUDA;
+    DeviceScope dev(device);
+    if (!dev.ok()) return OMSE_ECUDA;
     omse_ctx* c = new (std::nothrow) omse_ctx;
     if (!c) return OMSE_ENOMEM;
+    memset(c, 0, sizeof(*c));
     c->device = device;
     c->stream = static_cast<cudaStream_t>(cuda_stream);
     c->ws = nullptr;
@@ -336,7 +379,7 @@ int omse_create(omse_ctx** out, int device, void* cuda_stream) {
 
 int omse_destroy(omse_ctx* ctx) {
     if (!ctx) return OMSE_EINVAL;
-    cudaSetDevice(ctx->device);
+    DeviceScope dev(ctx->device);
     cudaStreamSynchronize(ctx->stream);
     cudaFree(ctx->ws);
     cudaFree(ctx->partials);
@@ -351,13 +394,19 @@ int omse_set_stream(omse_ctx* ctx, void* cuda_stream) {
     return OMSE_OK;
 }
 
-size_t omse_workspace_bytes(const omse_ctx* ctx) {
-    return ctx ? sizeof(Workspace) + kPartialBytes + sizeof(omse::RowTensor) * OMSE_MAX_BATCH : 0;
+size_t omse_workspace_bytes(int64_t n_kernels, int64_t kernel_len, int32_t n_cand, int32_t n_tensors) {
+    // Rows are searched on chip, so the workspace does not grow with the problem: status and dispenser words, the
+    // per-tensor search state and curve, per-block partial sums, descriptors of a batched launch.
+    if (n_kernels < 0 || kernel_len < 1 || n_cand < 1 || n_cand > OMSE_MAX_CANDIDATES || n_tensors < 1 ||
+        n_tensors > OMSE_MAX_TENSORS)
+        return 0;
+    return sizeof(Workspace) + kPartialBytes + sizeof(omse::RowTensor) * OMSE_MAX_BATCH;
 }
 
 int omse_last_device_status(omse_ctx* ctx, uint32_t* host_out) {
     if (!ctx || !host_out) return OMSE_EINVAL;
-    if (cudaSetDevice(ctx->device) != cudaSuccess) return OMSE_ECUDA;
+    DeviceScope dev(ctx->device);
+    if (!dev.ok()) return OMSE_ECUDA;
     if (cudaMemcpyAsync(host_out, &ctx->ws->status, sizeof(uint32_t), cudaMemcpyDeviceToHost, ctx->stream) != cudaSuccess)
         return OMSE_ECUDA;
     if (cudaMemsetAsync(&ctx->ws->status, 0, sizeof(uint32_t), ctx->stream) != cudaSuccess) return OMSE_ECUDA;
@@ -366,7 +415,8 @@ int omse_last_device_status(omse_ctx* ctx, uint32_t* host_out) {
 
 int omse_read_evaluations(omse_ctx* ctx, uint64_t* host_out) {
     if (!ctx || !host_out) return OMSE_EINVAL;
-    if (cudaSetDevice(ctx->device) != cudaSuccess) return OMSE_ECUDA;
+    DeviceScope dev(ctx->device);
+    if (!dev.ok()) return OMSE_ECUDA;
     unsigned long long v = 0;
     if (cudaMemcpyAsync(&v, &ctx->ws->evals, sizeof(v), cudaMemcpyDeviceToHost, ctx->stream) != cudaSuccess) return OMSE_ECUDA;
     if (cudaMemsetAsync(&ctx->ws->evals, 0, sizeof(v), ctx->stream) != cudaSuccess) return OMSE_ECUDA;
@@ -440,9 +490,9 @@ int omse_residual_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, i
                               nullptr, d_codes, d_packed);
 }
 
-int omse_alg1_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, int64_t kernel_len, const int* bits,
-                       const int* is_signed, const omse_grid* grid, int n_tensors, int n_sweeps, float* d_alpha,
-                       float* d_sse, float* d_sse_history, int8_t* d_codes, uint8_t* d_packed) {
+static int alg1_impl(omse_ctx* ctx, const float* d_t, int64_t n_kernels, int64_t kernel_len, const int* bits,
+                     const int* is_signed, const omse_grid* grid, int n_tensors, int n_sweeps, float eps, float* d_alpha,
+                     float* d_sse, float* d_sse_history, int32_t* d_sweeps_done, int8_t* d_codes, uint8_t* d_packed) {
     if (!ctx || !grid_ok(grid) || !bits || !is_signed || n_tensors < 1 || n_tensors > OMSE_MAX_TENSORS || n_sweeps < 1 ||
         n_sweeps > 64 || n_kernels < 0 || kernel_len < 1 || kernel_len > OMSE_MAX_KERNEL_LEN ||
         n_kernels > (int64_t)1 << 40)
@@ -454,8 +504,11 @@ int omse_alg1_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, int64
     if (n_sweeps > 1 && (!d_codes || kernel_len > OMSE_MAX_KERNEL_LEN_MULTISWEEP)) return OMSE_EINVAL;
     if (n_kernels == 0) return OMSE_OK;
     if (!d_t || !d_alpha || !d_sse) return OMSE_EINVAL;
-    if (misaligned4(d_t) || misaligned4(d_alpha) || misaligned4(d_sse) || misaligned4(d_sse_history)) return OMSE_EINVAL;
-    if (cudaSetDevice(ctx->device) != cudaSuccess) return OMSE_ECUDA;
+    if (misaligned4(d_t) || misaligned4(d_alpha) || misaligned4(d_sse) || misaligned4(d_sse_history) ||
+        misaligned4(d_sweeps_done))
+        return OMSE_EINVAL;
+    DeviceScope dev(ctx->device);
+    if (!dev.ok()) return OMSE_ECUDA;
     omse::RowArgs a;
     memset(&a, 0, sizeof(a));
     fill_tensor(a.one, d_t, n_kernels, kernel_len, d_alpha, d_sse, nullptr, d_codes, d_packed);
@@ -470,7 +523,126 @@ int omse_alg1_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, int64
     for (int j = 0; j < n_tensors; ++j) bounds(bits[j], is_signed[j], &a.lo[j], &a.hi[j]);
     a.keep_x0 = n_sweeps > 1 ? 1 : 0;
     a.sse_history = d_sse_history;
+    a.eps = eps;
+    a.sweeps_done = d_sweeps_done;
     return launch_rows(ctx, a, kernel_len);
+}
+
+int omse_alg1_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, int64_t kernel_len, const int* bits,
+                       const int* is_signed, const omse_grid* grid, int n_tensors, int n_sweeps, float* d_alpha,
+                       float* d_sse, float* d_sse_history, int8_t* d_codes, uint8_t* d_packed) {
+    return alg1_impl(ctx, d_t, n_kernels, kernel_len, bits, is_signed, grid, n_tensors, n_sweeps, -1.f, d_alpha, d_sse,
+                     d_sse_history, nullptr, d_codes, d_packed);
+}
+
+int omse_alg1_quantize_converge(omse_ctx* ctx, const float* d_t, int64_t n_kernels, int64_t kernel_len, const int* bits,
+                                const int* is_signed, const omse_grid* grid, int n_tensors, int max_sweeps, float eps,
+                                float* d_alpha, float* d_sse, float* d_sse_history, int32_t* d_sweeps_done,
+                                int8_t* d_codes, uint8_t* d_packed) {
+    if (!(eps >= 0.f)) return OMSE_EINVAL;
+    return alg1_impl(ctx, d_t, n_kernels, kernel_len, bits, is_signed, grid, n_tensors, max_sweeps, eps, d_alpha, d_sse,
+                     d_sse_history, d_sweeps_done, d_codes, d_packed);
+}
+
+int omse_quantize_weights_solver(omse_ctx* ctx, const float* d_w, int64_t n_kernels, int64_t kernel_len, int bits,
+                                 int is_signed, int solver, int n_iter, const omse_grid* grid, float* d_alpha,
+                                 float* d_sse, int32_t* d_best_idx, int8_t* d_codes, uint8_t* d_packed) {
+    if (solver == OMSE_SOLVER_GRID)
+        return omse_quantize_weights(ctx, d_w, n_kernels, kernel_len, bits, is_signed, grid, d_alpha, d_sse, d_best_idx,
+                                     d_codes, d_packed);
+    if (!ctx || !grid_ok(grid) || bits < 2 || bits > 8 || n_kernels < 0 || kernel_len < 1 ||
+        kernel_len > OMSE_MAX_KERNEL_LEN || n_kernels > (int64_t)1 << 40 || (d_packed && bits > 4) ||
+        solver < OMSE_SOLVER_UNIFORM || solver > OMSE_SOLVER_GOLDEN || n_iter < 0 || n_iter > 1024)
+        return OMSE_EINVAL;
+    if (n_kernels == 0) return OMSE_OK;
+    if (!d_w || !d_alpha || !d_sse) return OMSE_EINVAL;
+    if (misaligned4(d_w) || misaligned4(d_alpha) || misaligned4(d_sse) || misaligned4(d_best_idx)) return OMSE_EINVAL;
+    std::vector<omse::RowTensor> list(1);
+    fill_tensor(list[0], d_w, n_kernels, kernel_len, d_alpha, d_sse, d_best_idx, d_codes, d_packed);
+    ListMode mode;
+    mode.solver = solver;
+    mode.solver_iters = n_iter;
+    return quantize_list(ctx, list, kernel_len, bits, is_signed, grid, mode);
+}
+
+int omse_quantize_weights_affine(omse_ctx* ctx, const float* d_w, int64_t n_kernels, int64_t kernel_len, int bits,
+                                 const omse_grid* grid, const omse_offset_grid* offsets, float* d_alpha, float* d_delta,
+                                 float* d_sse, int32_t* d_best_idx, int8_t* d_codes, uint8_t* d_packed) {
+    if (!ctx || !grid_ok(grid) || !offsets || offsets->n_delta < 1 || offsets->n_delta > OMSE_MAX_OFFSETS ||
+        !(offsets->off_frac >= 0.f) || !(offsets->off_frac <= 1.f) || bits < 2 || bits > 8 || n_kernels < 0 ||
+        kernel_len < 1 || kernel_len > OMSE_MAX_KERNEL_LEN_MULTISWEEP || n_kernels > (int64_t)1 << 40 ||
+        (d_packed && bits > 4) || (int64_t)offsets->n_delta * grid->n_cand > 0x7fffffff)
+        return OMSE_EINVAL;
+    if (n_kernels == 0) return OMSE_OK;
+    if (!d_w || !d_alpha || !d_sse || !d_delta) return OMSE_EINVAL;
+    if (misaligned4(d_w) || misaligned4(d_alpha) || misaligned4(d_sse) || misaligned4(d_best_idx) || misaligned4(d_delta))
+        return OMSE_EINVAL;
+    std::vector<omse::RowTensor> list(1);
+    fill_tensor(list[0], d_w, n_kernels, kernel_len, d_alpha, d_sse, d_best_idx, d_codes, d_packed);
+    list[0].delta = d_delta;
+    ListMode mode;
+    mode.n_delta = offsets->n_delta;
+    mode.off_frac = offsets->off_frac;
+    return quantize_list(ctx, list, kernel_len, bits, /*is_signed=*/0, grid, mode);
+}
+
+int omse_quantize_key_layers(omse_ctx* ctx, const omse_key_layer* layers, int n_layers, int bits, int is_signed,
+                             const omse_grid* grid, float tau, double* d_mse, int32_t* d_is_key, double* d_cr) {
+    if (!ctx || !grid_ok(grid) || bits < 2 || bits > 8 || n_layers < 0 || n_layers > OMSE_MAX_BATCH ||
+        (n_layers > 0 && (!layers || !d_mse || !d_is_key)) || !(tau >= 0.f))
+        return OMSE_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(d_mse) & 7) || (reinterpret_cast<uintptr_t>(d_cr) & 7) || misaligned4(d_is_key))
+        return OMSE_EINVAL;
+    std::vector<omse_weight_tensor> first((size_t)n_layers);
+    std::vector<omse_layer_error> errs((size_t)n_layers);
+    for (int l = 0; l < n_layers; ++l) {
+        const omse_key_layer& L = layers[l];
+        if (L.first.n_kernels < 1 || L.first.kernel_len < 1 || L.first.kernel_len > OMSE_MAX_KERNEL_LEN ||
+            !L.d_alpha2 || !L.d_sse2 || misaligned4(L.d_alpha2) || misaligned4(L.d_sse2) || (L.d_packed2 && bits > 4))
+            return OMSE_EINVAL;
+        first[l] = L.first;
+        errs[l].d_sse = L.first.d_sse;
+        errs[l].n_kernels = L.first.n_kernels;
+        errs[l].kernel_len = L.first.kernel_len;
+    }
+    if (n_layers == 0) return OMSE_OK;
+    // 1. every layer with one quantized tensor; 2. MSE per layer against tau
+    int rc = omse_quantize_weights_batched(ctx, first.data(), n_layers, bits, is_signed, grid);
+    if (rc != OMSE_OK) return rc;
+    rc = omse_select_key_layers(ctx, errs.data(), n_layers, tau, d_mse, d_is_key);
+    if (rc != OMSE_OK) return rc;
+    // 3. one launch over all layers for the second tensor: blocks skip the layers whose flag is 0, so the host
+    //    never reads the flags; each row's residual is rebuilt on chip from the first scale
+    std::vector<omse::RowTensor> list((size_t)n_layers);
+    long long max_k = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        const omse_key_layer& L = layers[l];
+        fill_tensor(list[l], L.first.d_w, L.first.n_kernels, L.first.kernel_len, L.d_alpha2, L.d_sse2, nullptr,
+                    L.d_codes2, L.d_packed2);
+        list[l].prior_alpha = L.first.d_alpha;
+        list[l].gate = d_is_key + l;
+        if (L.first.kernel_len > max_k) max_k = L.first.kernel_len;
+    }
+    rc = quantize_list(ctx, list, max_k, bits, is_signed, grid);
+    if (rc != OMSE_OK) return rc;
+    // 4. compression ratio of the result (one or two quantized tensors per layer)
+    if (d_cr) {
+        DeviceScope dev(ctx->device);
+        if (!dev.ok()) return OMSE_ECUDA;
+        std::vector<omse::LayerError> shape((size_t)n_layers);
+        for (int l = 0; l < n_layers; ++l) {
+            shape[l].sse = nullptr;
+            shape[l].n_kernels = layers[l].first.n_kernels;
+            shape[l].kernel_len = layers[l].first.kernel_len;
+        }
+        omse::LayerError* d_layers = reinterpret_cast<omse::LayerError*>(ctx->d_tensors);
+        if (cudaMemcpyAsync(d_layers, shape.data(), sizeof(omse::LayerError) * shape.size(), cudaMemcpyHostToDevice,
+                            ctx->stream) != cudaSuccess)
+            return OMSE_ECUDA;
+        omse::compression_ratio_kernel<<<1, 32, 0, ctx->stream>>>(d_layers, n_layers, bits, d_is_key, d_cr);
+        if (cudaGetLastError() != cudaSuccess) return OMSE_ECUDA;
+    }
+    return OMSE_OK;
 }
 
 int omse_dual_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, int64_t kernel_len, int bits1, int bits2,
@@ -485,7 +657,8 @@ int omse_dual_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, int64
     if (n_kernels == 0) return OMSE_OK;
     if (!d_t || !d_alpha || !d_sse) return OMSE_EINVAL;
     if (misaligned4(d_t) || misaligned4(d_alpha) || misaligned4(d_sse) || misaligned4(d_best_idx)) return OMSE_EINVAL;
-    if (cudaSetDevice(ctx->device) != cudaSuccess) return OMSE_ECUDA;
+    DeviceScope dev(ctx->device);
+    if (!dev.ok()) return OMSE_ECUDA;
     omse::DualArgs a;
     memset(&a, 0, sizeof(a));
     a.t = d_t;
@@ -505,11 +678,10 @@ int omse_dual_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, int64
     a.status = &ctx->ws->status;
     a.rows_per_unit = (d_packed && (kernel_len & 1)) ? 2 : 1;
     const size_t smem = (size_t)((kernel_len + 3) & ~3ll) * 4 + 64 * 8 + omse::kDualListCap * 4 + 4 * 4;
-    static bool attr_set[64] = {};
-    if (!attr_set[ctx->device & 63]) {
+    if (!ctx->attr_dual) {
         if (cudaFuncSetAttribute(omse::dual_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess)
             return OMSE_ECUDA;
-        attr_set[ctx->device & 63] = true;
+        ctx->attr_dual = true;
     }
     int occ = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, omse::dual_kernel, omse::kDualThreads, smem) != cudaSuccess || occ < 1)
@@ -542,7 +714,8 @@ int omse_select_key_layers(omse_ctx* ctx, const omse_layer_error* layers, int n_
         list[i].kernel_len = layers[i].kernel_len;
     }
     if (n_layers == 0) return OMSE_OK;
-    if (cudaSetDevice(ctx->device) != cudaSuccess) return OMSE_ECUDA;
+    DeviceScope dev(ctx->device);
+    if (!dev.ok()) return OMSE_ECUDA;
     omse::LayerError* d_layers = reinterpret_cast<omse::LayerError*>(ctx->d_tensors);
     if (cudaMemcpyAsync(d_layers, list.data(), sizeof(omse::LayerError) * list.size(), cudaMemcpyHostToDevice,
                         ctx->stream) != cudaSuccess)
@@ -586,7 +759,8 @@ static int activation_impl(omse_ctx* ctx, const float* d_x, int64_t n, int bits,
         (reinterpret_cast<uintptr_t>(d_sse) & 3) || (reinterpret_cast<uintptr_t>(d_best_idx) & 3) ||
         (reinterpret_cast<uintptr_t>(d_sse_curve) & 7))
         return OMSE_EINVAL;
-    if (cudaSetDevice(ctx->device) != cudaSuccess) return OMSE_ECUDA;
+    DeviceScope dev(ctx->device);
+    if (!dev.ok()) return OMSE_ECUDA;
     omse::TensorArgs a;
     memset(&a, 0, sizeof(a));
     a.x = d_x;
@@ -645,7 +819,8 @@ int omse_pack_int4(omse_ctx* ctx, const int8_t* d_codes, int64_t n, int is_signe
     if (!ctx || n < 0) return OMSE_EINVAL;
     if (n == 0) return OMSE_OK;
     if (!d_codes || !d_packed) return OMSE_EINVAL;
-    if (cudaSetDevice(ctx->device) != cudaSuccess) return OMSE_ECUDA;
+    DeviceScope dev(ctx->device);
+    if (!dev.ok()) return OMSE_ECUDA;
     long long grid = (n / 16 + 255) / 256;
     if (grid > (long long)ctx->n_sm * 16) grid = (long long)ctx->n_sm * 16;
     if (grid < 1) grid = 1;
@@ -739,7 +914,8 @@ extern "C" int omse_activation_scale_static(int device, void* cuda_stream, const
         (reinterpret_cast<uintptr_t>(d_sse) & 3) || (reinterpret_cast<uintptr_t>(d_best_idx) & 3) ||
         (reinterpret_cast<uintptr_t>(d_sse_curve) & 7) || (reinterpret_cast<uintptr_t>(d_status) & 3))
         return OMSE_EINVAL;
-    if (cudaSetDevice(device) != cudaSuccess) return OMSE_ECUDA;
+    DeviceScope dev(device);
+    if (!dev.ok()) return OMSE_ECUDA;
     StaticDevice& sd = g_static_dev[device];
     {
         // once per device, with that device current: the device address of the array

@@ -20,6 +20,9 @@ struct RowTensor {
     signed char* codes;      // [n_tensors][N], nullable
     unsigned char* packed;   // [n_tensors][ceil(N/2)], nullable
     float* delta;            // [S] offset subtracted from each row (Section 3.1 scheme with offset), nullable = no offset
+    const float* prior_alpha;   // [S] nullable: scale of an earlier quantized tensor of this row; the row is replaced by its
+                                // residual fl(x - alpha*[x/alpha]_Zp) before the search (second tensor of a key layer, Section 3.5)
+    const int* gate;         // nullable: the tensor's units are skipped when *gate == 0 (key-layer flag written by an earlier kernel)
     long long unit_begin;    // index of this tensor's first work unit in the launch-wide numbering
     int rows_per_unit;       // long rows: 2 when nibble packing needs an even element count per unit (odd K), else 1;
                              // short rows: the batch size B (even)
@@ -47,6 +50,13 @@ struct RowArgs {
     int keep_x0;                // n_sweeps > 1: keep the original row next to the residual
     int max_k4;                 // float4s of the longest row in the launch (shared-memory carve-up)
     int prune;                  // 1: rows are regrouped by magnitude so that candidates skip elements they code as 0
+    int solver;                 // 0: grid line search (Section 3.4); 1: uniform scale max|x|/L; 2: alternating from the
+                                // uniform scale; 3: golden-section search (the comparison solvers of Section 3.4)
+    int solver_iters;           // alternating: least-squares steps; golden: shrink steps
+    int n_delta;                // > 0: offsets searched per row (offset scheme of Section 3.1 with delta on a grid); needs keep_x0
+    float off_frac;             // offsets span [min, min + off_frac*(max-min))
+    float eps;                  // >= 0: Algorithm 1 stops after the first sweep whose relative error decrease is <= eps
+    int* sweeps_done;           // [S] sweeps Algorithm 1 ran per row, nullable
 };
 
 }  // namespace omse
@@ -60,10 +70,55 @@ constexpr int kScratchDoubles = 64 + 16 * 9;
 
 struct PhiOut {
     float alpha;
-    double sse;
+    double sse;       // with PhiCtl::want_sse: squared error at the chosen grid candidate (true division, fp64)
     int idx;
     bool degenerate;
 };
+
+// What phi_block does on the row in s.xs besides the default "grid search, then refine_iters polish steps".
+struct PhiCtl {
+    int solver;       // as RowArgs::solver
+    int n_iter;       // as RowArgs::solver_iters
+    int start_idx;    // >= 0: skip the search and start from this grid candidate
+    int n_refine;     // polish steps
+    bool want_sse;    // also return the fp64 error at the chosen candidate (before any polish)
+};
+
+// ||x - alpha*[x/alpha]_Zp||^2 of the row in s.xs in fp64 with true division; every thread gets the sum.
+__device__ __forceinline__ double exact_sse_block(const float* xs, int k, float alpha, float flo, float fhi,
+                                                   double* scratch) {
+    double ss = 0.0;
+    long long zero = 0;
+    for (int i = threadIdx.x; i < k; i += blockDim.x) {
+        const float x = xs[i];
+        const double d = (double)x - (double)alpha * (double)code_of(x, alpha, flo, fhi);
+        ss += d * d;
+    }
+    block_sum2(ss, zero, scratch);
+    return ss;
+}
+
+// Least-squares polish of Section 3.4's objective: alpha <- <x,q>/<q,q>, q = [x/alpha]_Zp, at most n times.
+__device__ __forceinline__ float polish_block(const float* xs, int k, float alpha, float flo, float fhi, int n,
+                                              double* scratch) {
+    for (int it = 0; it < n; ++it) {
+        double sxq = 0.0;
+        long long sqq = 0;
+        for (int i = threadIdx.x; i < k; i += blockDim.x) {
+            const float x = xs[i];
+            const int q = code_of(x, alpha, flo, fhi);
+            sqq += q * q;
+            sxq += (double)x * (double)q;
+        }
+        block_sum2(sxq, sqq, scratch);
+        if (sqq == 0) break;
+        const float a_new = (float)(sxq / (double)sqq);
+        if (!(a_new >= FLT_MIN) || !(a_new <= FLT_MAX)) break;
+        if (a_new == alpha) break;   // fixed point: further steps would repeat it exactly
+        alpha = a_new;
+    }
+    return alpha;
+}
 
 // shared-memory carve-up for one block
 struct RowSmem {
@@ -190,7 +245,7 @@ __device__ void partition_row(const RowSmem& s, int k, const GridSetup& g, int t
 // The quantization mapping phi of Section 3.4 on the row held in s.xs (k elements, k4 float4s).
 template <int CPT>
 __device__ PhiOut phi_block(const RowArgs& a, const RowSmem& s, int k, int k4, float flo, float fhi,
-                             const float (&rcp)[CPT], unsigned long long& ev) {
+                             const float (&rcp)[CPT], unsigned long long& ev, const PhiCtl& ctl) {
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int grp = tid / a.tg, t = tid - grp * a.tg;
     const float4* xs4 = reinterpret_cast<const float4*>(s.xs);
@@ -213,7 +268,58 @@ __device__ PhiOut phi_block(const RowArgs& a, const RowSmem& s, int k, int k4, f
     out.sse = 0.0;
     out.idx = -1;
     out.degenerate = true;
+    if (ctl.solver != 0) {
+        // ---- comparison solvers of Section 3.4: another way to the starting scale, then the same polish
+        float alpha = 0.f;
+        if (ctl.solver == 3) {
+            // golden-section search on [0, hi_frac*max|x|], scales in binary32, errors in fp64 (uniform over the block)
+            const float rho = 0.618034f;
+            float lo_a = 0.f, hi_a = __fmul_rn(a.hi_frac, m);
+            float t = __fmul_rn(rho, __fsub_rn(hi_a, lo_a));
+            float x1 = __fsub_rn(hi_a, t), x2 = __fadd_rn(lo_a, t);
+            auto f = [&](float al) -> double {
+                return (al >= FLT_MIN && al <= FLT_MAX) ? exact_sse_block(s.xs, k, al, flo, fhi, s.scratch) : (double)INFINITY;
+            };
+            double f1 = f(x1), f2 = f(x2);
+            for (int it = 0; it < ctl.n_iter; ++it) {
+                if (f1 <= f2) {          // equal errors keep the smaller scale
+                    hi_a = x2;
+                    x2 = x1;
+                    f2 = f1;
+                    t = __fmul_rn(rho, __fsub_rn(hi_a, lo_a));
+                    x1 = __fsub_rn(hi_a, t);
+                    f1 = f(x1);
+                } else {
+                    lo_a = x1;
+                    x1 = x2;
+                    f1 = f2;
+                    t = __fmul_rn(rho, __fsub_rn(hi_a, lo_a));
+                    x2 = __fadd_rn(lo_a, t);
+                    f2 = f(x2);
+                }
+            }
+            alpha = (f1 <= f2) ? x1 : x2;
+            if (!(fmin(f1, f2) < (double)INFINITY)) alpha = 0.f;
+        } else {
+            // no-offset uniform quantizer of Section 3.1: alpha = max|x| / L
+            alpha = __fdiv_rn(m, fhi);   // L = 2^(p-1)-1 (signed) or 2^p-1 (unsigned) is the top code of the range
+        }
+        if (!(alpha >= FLT_MIN) || !(alpha <= FLT_MAX)) return out;
+        out.degenerate = false;
+        out.idx = 0;
+        const int steps = ctl.n_refine + (ctl.solver == 2 ? ctl.n_iter : 0);
+        out.alpha = polish_block(s.xs, k, alpha, flo, fhi, steps, s.scratch);
+        return out;
+    }
     if (!(m > 0.f) || !(a_last >= FLT_MIN)) return out;   // no usable scale: alpha = 0, all codes 0
+    if (ctl.start_idx >= 0) {
+        const float ac = __fmul_rn((float)(ctl.start_idx + 1), g.step);
+        if (!(ac >= FLT_MIN)) return out;
+        out.degenerate = false;
+        out.idx = ctl.start_idx;
+        out.alpha = polish_block(s.xs, k, ac, flo, fhi, ctl.n_refine, s.scratch);
+        return out;
+    }
 
     // ---- per-thread candidate constants
     u64 inv2[CPT], na2[CPT];
@@ -295,8 +401,8 @@ __device__ PhiOut phi_block(const RowArgs& a, const RowSmem& s, int k, int k4, f
     const int holders = __syncthreads_count(mine > 0);
     const int multi = __syncthreads_or(mine > 1);
     int best = bi;
+    double best_sse = INFINITY;
     if (holders > 1 || multi) {
-        double best_sse = INFINITY;
         best = 0x7fffffff;
         int prev = -1;
         for (;;) {
@@ -326,27 +432,12 @@ __device__ PhiOut phi_block(const RowArgs& a, const RowSmem& s, int k, int k4, f
         }
     }
 
-    // ---- polish: alpha <- <x,q>/<q,q>, q = [x/alpha]_Zp, refine_iters times
-    float alpha = __fmul_rn((float)(best + 1), g.step);
-    for (int it = 0; it < a.refine_iters; ++it) {
-        double sxq = 0.0;
-        long long sqq = 0;
-        for (int i = tid; i < k; i += nthr) {
-            const float x = s.xs[i];
-            const int q = code_of(x, alpha, flo, fhi);
-            sqq += q * q;
-            sxq += (double)x * (double)q;
-        }
-        block_sum2(sxq, sqq, s.scratch);
-        if (sqq == 0) break;
-        const float a_new = (float)(sxq / (double)sqq);
-        if (!(a_new >= FLT_MIN) || !(a_new <= FLT_MAX)) break;
-        if (a_new == alpha) break;   // fixed point: further steps would repeat it exactly
-        alpha = a_new;
-    }
-    out.alpha = alpha;
+    // ---- polish: alpha <- <x,q>/<q,q>, q = [x/alpha]_Zp
+    const float a_grid = __fmul_rn((float)(best + 1), g.step);
+    if (ctl.want_sse)
+        out.sse = best_sse < INFINITY ? best_sse : exact_sse_block(s.xs, k, a_grid, flo, fhi, s.scratch);
+    out.alpha = polish_block(s.xs, k, a_grid, flo, fhi, ctl.n_refine, s.scratch);
     out.idx = best;
-    out.sse = 0.0;   // filled by emit_block
     return out;
 }
 
@@ -457,6 +548,7 @@ __global__ void __launch_bounds__(OMSE_ROWS_MAX_THREADS) rows_kernel(const RowAr
             tp = a.tensors + ti;
         }
         const RowTensor& T = *tp;
+        if (T.gate && *T.gate == 0) continue;   // not a key layer: nothing to do for this unit
         if (T.small & 4) {
             tiny_dispatch<CPT>(a, T, unit - T.unit_begin, smem_raw, st, ev);
             continue;
@@ -500,7 +592,18 @@ __global__ void __launch_bounds__(OMSE_ROWS_MAX_THREADS) rows_kernel(const RowAr
                 }
             }
             if (bad) st |= 1u;
-            if (T.delta) {
+            if (T.prior_alpha) {
+                // second quantized tensor of a key layer: the row becomes the residual of the first tensor
+                __syncthreads();
+                const float a1 = T.prior_alpha[row];
+                const float flo0 = (float)a.lo[0], fhi0 = (float)a.hi[0];
+                if (a1 > 0.f)
+                    for (int i = tid; i < k; i += nthr) {
+                        const float x = s.xs[i];
+                        s.xs[i] = fmaf(-a1, (float)code_of(x, a1, flo0, fhi0), x);
+                    }
+            }
+            if (T.delta && a.n_delta == 0) {
                 // quantization with offset: delta = min of the row, the shifted row fl(x - delta) is what gets searched
                 __syncthreads();
                 float lo = INFINITY;
@@ -525,8 +628,88 @@ __global__ void __launch_bounds__(OMSE_ROWS_MAX_THREADS) rows_kernel(const RowAr
             }
             __syncthreads();
 
+            if (a.n_delta > 0) {
+                // ---- offset scheme of Section 3.1 with the offset searched as well: for every offset on the grid
+                //      the line search of the shifted row fl(x - delta); the pair with the smallest error wins
+                //      (lowest offset, then lowest scale index, on equal errors); polish and codes at that pair
+                const float flo = (float)a.lo[0], fhi = (float)a.hi[0];
+                float lo = INFINITY, hi = -INFINITY;   // extremes of the finite values of the row
+                for (int i = tid; i < k; i += nthr) {
+                    const float v = s.x0[i];
+                    if (fabsf(v) <= FLT_MAX) {
+                        lo = fminf(lo, v);
+                        hi = fmaxf(hi, v);
+                    }
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+                    hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+                }
+                __shared__ float s_ext[2][32];
+                if ((tid & 31) == 0) {
+                    s_ext[0][tid >> 5] = lo;
+                    s_ext[1][tid >> 5] = hi;
+                }
+                __syncthreads();
+                lo = INFINITY;
+                hi = -INFINITY;
+                for (int w = 0; w < ((nthr + 31) >> 5); ++w) {
+                    lo = fminf(lo, s_ext[0][w]);
+                    hi = fmaxf(hi, s_ext[1][w]);
+                }
+                if (!(lo <= hi)) lo = hi = 0.f;
+                const float dstep = __fdiv_rn(__fmul_rn(a.off_frac, __fsub_rn(hi, lo)), (float)a.n_delta);
+                double best_sse = INFINITY;
+                int best_d = -1, best_c = -1;
+                PhiCtl search = {0, 0, -1, 0, true};
+                for (int d = 0; d < a.n_delta; ++d) {
+                    const float dl = __fadd_rn(lo, __fmul_rn((float)d, dstep));
+                    __syncthreads();
+                    for (int i = tid; i < 4 * k4; i += nthr) s.xs[i] = i < k ? __fsub_rn(s.x0[i], dl) : 0.f;
+                    __syncthreads();
+                    const PhiOut r = phi_block<CPT>(a, s, k, k4, flo, fhi, rcp, ev, search);
+                    if (!r.degenerate && r.sse < best_sse) {   // increasing offset: strict < keeps the lowest flat index
+                        best_sse = r.sse;
+                        best_d = d;
+                        best_c = r.idx;
+                    }
+                }
+                const float dl = __fadd_rn(lo, __fmul_rn((float)max(best_d, 0), dstep));
+                __syncthreads();
+                for (int i = tid; i < 4 * k4; i += nthr) s.xs[i] = i < k ? __fsub_rn(s.x0[i], dl) : 0.f;
+                __syncthreads();
+                PhiOut r;
+                r.alpha = 0.f;
+                r.idx = -1;
+                r.degenerate = true;
+                if (best_d >= 0) {
+                    const PhiCtl from = {0, 0, best_c, a.refine_iters, false};
+                    r = phi_block<CPT>(a, s, k, k4, flo, fhi, rcp, ev, from);
+                }
+                if (r.degenerate) st |= 2u;
+                const double sse = emit_block(s, k, r.alpha, flo, fhi, T.codes, T.packed, row_base, &s.misc[1], more);
+                if (tid == 0) {
+                    T.alpha[row] = r.alpha;
+                    T.sse[row] = (float)sse;
+                    if (T.delta) T.delta[row] = dl;
+                    if (T.best_idx) T.best_idx[row] = r.degenerate ? -1 : best_d * a.n_cand + best_c;
+                }
+                __syncthreads();
+                continue;
+            }
+
             // ---- Algorithm 1: sweeps over the tensors; one tensor and one sweep is plain phi
+            double e_prev = 0.0;                   // error before the current sweep (all tensors zero: ||T||^2)
+            if (a.eps >= 0.f) {
+                long long zero = 0;
+                for (int i = tid; i < k; i += nthr) e_prev += (double)s.xs[i] * (double)s.xs[i];
+                block_sum2(e_prev, zero, s.scratch);
+            }
+            int sweeps_ran = 0;
+            const PhiCtl ctl = {a.solver, a.solver_iters, -1, a.refine_iters, false};
             for (int sweep = 0; sweep < a.n_sweeps; ++sweep) {
+                double e_cur = 0.0;
                 for (int j = 0; j < a.n_tensors; ++j) {
                     const float flo = (float)a.lo[j], fhi = (float)a.hi[j];
                     if (a.keep_x0 && !(sweep == 0 && j == 0)) {
@@ -543,12 +726,13 @@ __global__ void __launch_bounds__(OMSE_ROWS_MAX_THREADS) rows_kernel(const RowAr
                         }
                         __syncthreads();
                     }
-                    PhiOut r = phi_block<CPT>(a, s, k, k4, flo, fhi, rcp, ev);
+                    PhiOut r = phi_block<CPT>(a, s, k, k4, flo, fhi, rcp, ev, ctl);
                     if (r.degenerate) st |= 2u;
                     const double sse = emit_block(s, k, r.alpha, flo, fhi,
                                                   T.codes ? T.codes + (long long)j * n_total : nullptr,
                                                   T.packed ? T.packed + (long long)j * packed_stride : nullptr,
                                                   row_base, &s.misc[1 + j], more);
+                    e_cur = sse;
                     if (tid == 0) {
                         T.alpha[(long long)j * T.S + row] = r.alpha;
                         T.sse[(long long)j * T.S + row] = (float)sse;
@@ -565,6 +749,20 @@ __global__ void __launch_bounds__(OMSE_ROWS_MAX_THREADS) rows_kernel(const RowAr
                     }
                     __syncthreads();   // alpha / codes of tensor j visible to the block (global + shared)
                 }
+                sweeps_ran = sweep + 1;
+                if (a.eps >= 0.f) {
+                    // while-condition of Algorithm 1: go on while the sweep lowered the error by more than eps (relative)
+                    const bool go_on = (e_prev - e_cur) > (double)a.eps * e_prev;
+                    e_prev = e_cur;
+                    if (!go_on) break;
+                }
+            }
+            if (tid == 0) {
+                if (a.sweeps_done) a.sweeps_done[row] = sweeps_ran;
+                if (a.sse_history)     // sweeps that did not run repeat the last error
+                    for (int sweep = sweeps_ran; sweep < a.n_sweeps; ++sweep)
+                        for (int j = 0; j < a.n_tensors; ++j)
+                            a.sse_history[((long long)sweep * a.n_tensors + j) * T.S + row] = T.sse[(long long)j * T.S + row];
             }
         }
     }

@@ -295,6 +295,18 @@ __device__ void small_unit(const RowArgs& a, const RowTensor& T, long long unit_
     }
     if (bad) st |= 1u;
     __syncthreads();
+    if (T.prior_alpha) {
+        // second quantized tensor of a key layer: every row becomes the residual of its first tensor
+        for (int i = tid; i < nrows * kpad; i += nthr) {
+            const int r = i / kpad, c = i - r * kpad;
+            const float a1 = T.prior_alpha[row0 + r];
+            if (c < k && a1 > 0.f) {
+                const float x = xs[i];
+                xs[i] = fmaf(-a1, (float)code_of(x, a1, flo, fhi), x);
+            }
+        }
+        __syncthreads();
+    }
 
     // ---- max of the positive and negative part of every row, and the row's grid: a warp per row
     for (int r = warp; r < nrows; r += nwarp) {

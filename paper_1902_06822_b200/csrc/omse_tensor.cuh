@@ -564,6 +564,20 @@ __global__ void __launch_bounds__(256) layer_mse_kernel(const LayerError* __rest
     }
 }
 
+// Compression ratio of Section 3.5 for layers that hold one quantized tensor, or two where is_key is set:
+// (codes at `bits` per element plus one binary32 scale per kernel, per quantized tensor) over the binary32 size.
+__global__ void compression_ratio_kernel(const LayerError* __restrict__ layers, int n_layers, int bits,
+                                         const int* __restrict__ is_key, double* __restrict__ cr) {
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    double q = 0.0, f = 0.0;
+    for (int l = 0; l < n_layers; ++l) {
+        const double n = (double)layers[l].n_kernels * (double)layers[l].kernel_len;
+        q += (is_key[l] ? 2.0 : 1.0) * (n * (double)bits + 32.0 * (double)layers[l].n_kernels);
+        f += 32.0 * n;
+    }
+    *cr = f > 0.0 ? q / f : 0.0;
+}
+
 // INT4 emission: byte e/2 holds element e (even) in bits 0-3 and element e+1 in bits 4-7.
 __global__ void __launch_bounds__(256) pack_int4_kernel(const signed char* __restrict__ codes, long long n,
                                                          unsigned char* __restrict__ packed) {

@@ -30,21 +30,24 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 N_CAND, BITS, REFINE, HI_FRAC = 1024, 4, 3, 1.0
+METRIC = "elements quantized/sec (4-bit MMSE search)"
 INSTR_PER_EVAL = 6            # reference FP32 sequence per (element, candidate): 3 fma + 2 min/max + 1 add
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the timed kernel, from the ncu capture summarised
-# in profiles/rows_kernel_resnet50_weight_set.md; set to None whenever the kernel changes after the capture
-NCU_TRAFFIC_BYTES = 108_999_936
+LANE_OPS_PER_EVAL = 4         # FMA-pipe lane operations of an evaluation the kernels execute: fma, add, fma, fma
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the timed kernel from an ncu capture of the
+# default workload; None whenever the kernel has changed since the capture
+NCU_TRAFFIC_BYTES = None
 E2E_CHUNKS = 12               # batched launches per end-to-end step (copies of later chunks overlap earlier searches)
 N_SM, LANES_PER_SM = 148, 128
 WORKLOAD = "resnet50_weight_set_54_tensors_25.5M_params_signed4bit_kernelwise_1024cand_3refine_packed"
 
 
-def _peaks():
+def _hbm_peak():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
         d = json.load(open(p))
-        return d.get("sm_max_mhz", 1965.0), "measured"
-    return 1965.0, "fallback"
+        if d.get("hbm_gbs"):
+            return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json: copy bandwidth)"
+    return 6650.0, "fallback (6.65 TB/s, an earlier measurement on this pool)"
 
 
 class ClockSampler:
@@ -146,6 +149,14 @@ class Workload:
     def host_arrays(self):       # list of numpy inputs
         raise NotImplementedError
 
+    def algorithmic_bytes(self):  # HBM bytes one step has to move: inputs read once, outputs written once
+        return self.h2d + self.d2h
+
+    def release(self):           # drop device and pinned buffers
+        for k in list(self.__dict__):
+            if k not in ("name", "n_cand", "n_total", "h2d", "d2h", "evals_per_element"):
+                delattr(self, k)
+
 
 class WeightSet(Workload):
     """One or more weight tensors through the batched kernel-wise call."""
@@ -233,6 +244,12 @@ class Activation(Workload):
     def __init__(self, name, x, n_cand):
         self.name, self.x, self.n_cand = name, x, n_cand
 
+    def host_arrays(self):
+        return [self.x]
+
+    def algorithmic_bytes(self):  # maximum, sweep, polish steps and the final error each read the tensor once
+        return 4 * self.n_total * (3 + REFINE)
+
     def setup(self, ctx, torch, dev):
         self.host_in = torch.from_numpy(self.x).pin_memory()
         self.d_x = self.host_in.to(dev)
@@ -266,6 +283,9 @@ class Residual(Workload):
 
     def __init__(self, name, t, n_cand):
         self.name, self.t, self.n_cand = name, t, n_cand
+
+    def host_arrays(self):
+        return [self.t]
 
     def setup(self, ctx, torch, dev):
         s, k = self.t.shape
@@ -309,6 +329,9 @@ class Dual(Workload):
         self.n_cand = self.C1 * self.C2
         self.evals_per_element = 1 << BITS          # first codes enumerated per pair
 
+    def host_arrays(self):
+        return [self.t]
+
     def setup(self, ctx, torch, dev):
         s, k = self.t.shape
         self.host_in = torch.from_numpy(self.t).pin_memory()
@@ -347,6 +370,10 @@ def make_workload(spec: str, rank: int):
     if spec == "c1":
         return WeightSet("single_conv_layer_64x576_signed4bit_256cand_3refine_int8", [synth.conv_layer(1 + rank)],
                          BITS, 256, False, 1, "all 64 kernels")
+    if spec == "c1x64":
+        ws = [synth.conv_layer(100 + 64 * rank + i) for i in range(64)]
+        return WeightSet("64_conv_layers_64x576_signed4bit_256cand_3refine_int8_one_batched_launch", ws, BITS, 256, False,
+                         4, "every 4th kernel of each of the 64 tensors")
     if spec == "c3":
         return Activation("activation_64x256x56x56_unsigned4bit_per_tensor_2048cand_3refine",
                           synth.activation_tensor(seed=3 + 1000 * rank), 2048)
@@ -366,11 +393,18 @@ def make_workload(spec: str, rank: int):
     raise SystemExit(f"unknown workload {spec}")
 
 
+def base_config(wl, n_total):
+    """The keys both arms print under "config"."""
+    return {"workload": wl.name, "elements_per_gpu": n_total, "n_cand": wl.n_cand, "refine_iters": REFINE,
+            "l2": "flushed between timed steps (256 MB write)"}
+
+
 def run_reference(args, rank):
     """The oracle, as it stands, on the host cores; each step is the workload's bounded sample."""
     if rank != 0:
         return
     wl = make_workload(args.workload, 0)
+    n_total = sum(a.size for a in wl.host_arrays())
     # Size the per-step sample so that all the steps together take about a minute on this host: one
     # calibration call on the standard sample, then a coarser row stride if the run would be longer.
     if hasattr(wl, "sample_stride"):
@@ -389,13 +423,71 @@ def run_reference(args, rank):
         total_t += time.perf_counter() - t0
     value = n * args.steps / total_t
     print(json.dumps({
-        "impl": "reference", "metric": "elements quantized/sec (4-bit MMSE search)", "value": value,
+        "impl": "reference", "metric": METRIC, "value": value,
         "unit": "elements/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": 1e3 * total_t / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f64", "data": "synthetic", "config": {"workload": wl.name, "sample": desc},
+        "dtype": "f64", "data": "synthetic", "config": base_config(wl, n_total),
         "cpu_baseline": {"value": value, "unit": "elements/s", "cores": cores, "kind": "oracle", "sample": desc},
         "e2e": {"value": value, "unit": "elements/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
+
+
+class Timer:
+    """CUDA-event timing of `steps` calls with an L2 flush before each (the flush is not timed)."""
+
+    def __init__(self, torch, stream, dev, dist):
+        self.torch, self.stream, self.dev, self.dist = torch, stream, dev, dist
+        self.flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # > 126 MB L2
+
+    def barrier(self):
+        self.torch.cuda.synchronize()
+        if self.dist is not None:
+            self.dist.barrier()
+            self.torch.cuda.synchronize()
+
+    def run(self, fn, steps):
+        torch = self.torch
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        self.barrier()
+        for s0, s1 in ev:
+            self.flush.fill_(1)         # evict the inputs from L2 between timed steps
+            s0.record(self.stream)
+            fn()
+            s1.record(self.stream)
+        self.barrier()
+        return max_over_ranks(sum(s0.elapsed_time(s1) for s0, s1 in ev), self.dist, self.dev)
+
+
+def roofline_of(wl, n_total, per_step_s, executed, fma_peak, hbm_gbs):
+    """Executed work against the two roofs: FP32 lane operations of the FMA pipe (4 per executed evaluation:
+    fma, add, fma, fma) and algorithmic HBM bytes; the fraction is the larger of the two, i.e. roof time / time."""
+    evals = wl.n_cand * wl.evals_per_element * n_total                      # all (element, candidate) pairs
+    ipe = getattr(wl, "instr_per_eval", INSTR_PER_EVAL)
+    lane_ops = LANE_OPS_PER_EVAL * executed
+    bytes_algo = wl.algorithmic_bytes()
+    frac_fma = lane_ops / per_step_s / fma_peak
+    frac_hbm = bytes_algo / per_step_s / (hbm_gbs * 1e9)
+    return {"bound": "alu", "achieved": lane_ops / per_step_s / 1e12, "peak": fma_peak / 1e12,
+            "unit": "T FP32 lane-op/s", "frac": max(frac_fma, frac_hbm), "frac_fma_pipe": frac_fma, "frac_hbm": frac_hbm,
+            "kernel": wl.kernel, "lane_ops_per_executed_evaluation": LANE_OPS_PER_EVAL,
+            "executed_evaluations_per_step": executed, "executed_share": executed / evals,
+            "algorithmic_bytes_per_step": bytes_algo,
+            # speed against a kernel that evaluates every pair with the 6-instruction reference sequence at this peak
+            "speed_vs_exhaustive": ipe * evals / per_step_s / fma_peak}
+
+
+def measure(wl, ctx, timer, steps, warmup):
+    """Device-resident timing of one workload: ms per step and executed evaluations per step."""
+    for _ in range(max(warmup, 3)):
+        wl.step()
+    timer.torch.cuda.synchronize()
+    ctx.omse_read_evaluations()                     # clear the instrumentation counter
+    ms = timer.run(wl.step, steps)
+    executed = ctx.omse_read_evaluations() / steps
+    return ms, executed
+
+
+PER_CONFIG = ["c1", "c1x64", "c3", "c4", "c5:27:4", "c5:576:4", "c5:4608:4", "c5:25088:4", "dual"]
 
 
 def run_ours(args, rank, world):
@@ -413,68 +505,79 @@ def run_ours(args, rank, world):
     wl = make_workload(args.workload, rank)
     ctx = binding.Context(local)
     stream = torch.cuda.current_stream(dev)
+    timer = Timer(torch, stream, dev, dist)
     wl.setup(ctx, torch, dev)
     n_total = wl.n_total
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # > 126 MB L2
+    hbm_gbs, hbm_src = _hbm_peak()
 
-    def barrier():
-        torch.cuda.synchronize()
-        if dist is not None:
-            dist.barrier()
-            torch.cuda.synchronize()
+    # ---- the FP32 roof, measured in this process on this GPU (packed fma loop on every SM), clocks sampled beside it
+    peak_sampler = ClockSampler(local) if rank == 0 else None
+    ctx.omse_measure_fp32_peak(50)
+    fma_peak = ctx.omse_measure_fp32_peak(400)
+    peak_clocks = peak_sampler.stop() if peak_sampler else None
 
-    def timed(fn, steps):
-        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
-        barrier()
-        for s0, s1 in ev:
-            flush.fill_(1)          # evict the inputs from L2 between timed steps (not timed)
-            s0.record(stream)
-            fn()
-            s1.record(stream)
-        barrier()
-        return max_over_ranks(sum(s0.elapsed_time(s1) for s0, s1 in ev), dist, dev)
-
+    # ---- the timed region proper
     sampler = ClockSampler(local) if rank == 0 else None
-    for _ in range(max(args.warmup, 3)):
-        wl.step()
-    torch.cuda.synchronize()
-    ctx.omse_read_evaluations()                     # clear the instrumentation counter
-    ms = timed(wl.step, args.steps)
-    executed = ctx.omse_read_evaluations() / args.steps   # evaluations the kernels really executed per step
+    ms, executed = measure(wl, ctx, timer, args.steps, args.warmup)
     clocks = sampler.stop() if sampler else None
     wl.step_e2e()
-    ms_e2e = timed(wl.step_e2e, args.steps)
+    ms_e2e = timer.run(wl.step_e2e, args.steps)
     status = ctx.omse_last_device_status()
 
+    # ---- the same step repeated for seconds: does the clock hold under this kernel?
+    sustained = None
+    if world == 1 and not args.quick:
+        n_long = int(min(20000, max(args.steps, np.ceil(2000.0 / (ms / args.steps)))))
+        long_sampler = ClockSampler(local)
+        ms_long = timer.run(wl.step, n_long)
+        lc = long_sampler.stop()
+        sustained = {"steps": n_long, "ms_per_step": ms_long / n_long, "value": n_total / (ms_long * 1e-3 / n_long),
+                     "clocks": lc}
+
+    # ---- the other configurations, a few steps each (the default line stays the one the metric is quoted on)
+    per_config = None
+    if world == 1 and not args.quick and args.workload == "c2":
+        per_config = {}
+        for spec in PER_CONFIG:
+            w2 = make_workload(spec, rank)
+            w2.setup(ctx, torch, dev)
+            s2 = 5
+            ms2, ex2 = measure(w2, ctx, timer, s2, 3)
+            r2 = roofline_of(w2, w2.n_total, ms2 * 1e-3 / s2, ex2, fma_peak, hbm_gbs)
+            per_config[spec] = {"workload": w2.name, "elements": w2.n_total, "steps": s2, "ms_per_step": ms2 / s2,
+                                "value": w2.n_total / (ms2 * 1e-3 / s2), "executed_share": r2["executed_share"],
+                                "frac": r2["frac"], "frac_fma_pipe": r2["frac_fma_pipe"], "frac_hbm": r2["frac_hbm"],
+                                "speed_vs_exhaustive": r2["speed_vs_exhaustive"], "kernel": w2.kernel,
+                                "gpu_launches": w2.launches_per_step * s2}
+            w2.release()
+            del w2
+            torch.cuda.empty_cache()
+
     if rank == 0:
-        sm_max_mhz, peak_src = _peaks()
         per_step_s = ms * 1e-3 / args.steps
         value = whole_job_value(n_total, world, ms, args.steps)
-        peak = N_SM * LANES_PER_SM * sm_max_mhz * 1e6                     # FP32 lane-instructions per second
-        evals = wl.n_cand * wl.evals_per_element * n_total                 # (element, candidate) evaluations per step
-        ipe = getattr(wl, "instr_per_eval", INSTR_PER_EVAL)
-        achieved = ipe * evals / per_step_s                                # algorithmic instructions per second
+        roof = roofline_of(wl, n_total, per_step_s, executed, fma_peak, hbm_gbs)
+        roof["traffic"] = NCU_TRAFFIC_BYTES if args.workload == "c2" else None
+        roof["peak_source"] = ("measured in this run: packed fma.rn.f32x2 loop on all SMs, "
+                               f"{fma_peak / (N_SM * LANES_PER_SM) / 1e6:.0f} MHz-equivalent per lane")
+        roof["peak_clocks"] = peak_clocks
+        roof["hbm_peak_gbs"] = hbm_gbs
+        roof["hbm_peak_source"] = hbm_src
         out = {
-            "metric": "elements quantized/sec (4-bit MMSE search)", "value": value, "unit": "elements/s",
+            "metric": METRIC, "value": value, "unit": "elements/s",
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": wl.name, "elements_per_gpu": n_total, "n_cand": wl.n_cand,
-                       "refine_iters": REFINE, "l2": "flushed between timed steps (256 MB write)",
-                       "device_status": status},
+            "config": base_config(wl, n_total), "device_status": status,
             "clocks": clocks,
             "e2e": {"value": whole_job_value(n_total, world, ms_e2e, args.steps), "unit": "elements/s",
                     "h2d_bytes_per_step": wl.h2d, "d2h_bytes_per_step": wl.d2h},
             "gpu_launches": wl.launches_per_step * args.steps,
-            "roofline": {"bound": "alu", "achieved": achieved / 1e12, "peak": peak / 1e12,
-                         "unit": "T FP32-instr/s", "frac": achieved / peak,
-                         "traffic": NCU_TRAFFIC_BYTES if args.workload == "c2" else None,
-                         "kernel": wl.kernel, "peak_source": f"148 SMs x 128 lanes x {sm_max_mhz:.0f} MHz ({peak_src} max clock)",
-                         "instr_per_eval": ipe, "evaluations_per_s": evals / per_step_s,
-                         # the kernels skip, exactly, evaluations whose code is provably zero: what was executed,
-                         # and the FMA-pipe lane operations (4 per executed evaluation) against the same peak
-                         "executed_evaluations_per_step": executed, "executed_share": executed / evals,
-                         "executed_fma_frac": 4.0 * executed / per_step_s / peak},
+            "roofline": roof,
         }
+        if sustained is not None:
+            out["sustained"] = sustained
+        if per_config is not None:
+            out["per_config"] = per_config
         if world == 1 and not args.no_cpu_baseline:
             v, cores, desc, _ = wl.cpu()
             out["cpu_baseline"] = {"value": v, "unit": "elements/s", "cores": cores, "kind": "oracle", "sample": desc}
@@ -490,8 +593,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--quick", action="store_true",
+                    help="only the timed region of the selected workload: no seconds-long loop, no per_config block")
     ap.add_argument("--workload", default="c2",
-                    help="c2 (default: the ResNet-50 weight set the metric is quoted on), c1, c3, c4, c5:K:bits, dual")
+                    help="c2 (default: the ResNet-50 weight set the metric is quoted on), c1, c1x64, c3, c4, c5:K:bits, dual")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))

@@ -387,6 +387,12 @@ int omse_last_device_status(omse_ctx* ctx, uint32_t* host_out);
  * omse_dual_quantize the unit is (element, pair, first code).  omse_activation_scale_static does not count. */
 int omse_read_evaluations(omse_ctx* ctx, uint64_t* host_out);
 
+/* Instrumentation (no counterpart in the paper): runs a register-only loop of independent fma.rn.f32x2 on every SM
+ * for about target_ms milliseconds (1..5000) on the context's stream, synchronises, and returns in *host_out the
+ * measured FP32 lane operations per second of the FMA pipe (a packed instruction counts as two).  This is the
+ * arithmetic roof the candidate sweep is compared with: an evaluation the sweep executes costs 4 such operations. */
+int omse_measure_fp32_peak(omse_ctx* ctx, int target_ms, double* host_out);
+
 /* Static description of a return value. */
 const char* omse_status_string(int status);
 

@@ -64,7 +64,7 @@ struct omse_ctx {
     double* partials;    // device, kPartialBytes
     omse::RowTensor* d_tensors;   // device, OMSE_MAX_BATCH descriptors of a batched launch
     // per-context launch bookkeeping (a context is used by one host thread at a time, so no lock)
-    bool attr_rows[4], attr_tensor[4], attr_dual;   // opt-in shared-memory attribute set, per template instance
+    bool attr_rows[8], attr_tensor[4], attr_dual;   // opt-in shared-memory attribute set, per template instance
     LaunchShape seen[16];                           // blocks per SM of the row-kernel launch shapes met so far
     int n_seen, next_seen;
 };
@@ -117,28 +117,29 @@ void bounds(int bits, int is_signed, int* lo, int* hi) {
     }
 }
 
-template <int CPT>
+template <int CPT, bool EXT>
 int launch_rows_t(omse_ctx* ctx, omse::RowArgs& a, size_t smem) {
-    if (!ctx->attr_rows[cpt_slot(CPT)]) {
-        if (cudaFuncSetAttribute(omse::rows_kernel<CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess)
+    const int slot = cpt_slot(CPT) + (EXT ? 4 : 0);
+    if (!ctx->attr_rows[slot]) {
+        if (cudaFuncSetAttribute(omse::rows_kernel<CPT, EXT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess)
             return OMSE_ECUDA;
-        ctx->attr_rows[cpt_slot(CPT)] = true;
+        ctx->attr_rows[slot] = true;
     }
     const int threads = a.groups * a.tg;
     // blocks per SM for this launch shape (remembered: the query costs more than a small launch)
     int occ = 0;
     for (int i = 0; i < ctx->n_seen; ++i)
-        if (ctx->seen[i].cpt == CPT && ctx->seen[i].threads == threads && ctx->seen[i].smem == smem) occ = ctx->seen[i].occ;
+        if (ctx->seen[i].cpt == slot && ctx->seen[i].threads == threads && ctx->seen[i].smem == smem) occ = ctx->seen[i].occ;
     if (occ == 0) {
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, omse::rows_kernel<CPT>, threads, smem) != cudaSuccess || occ < 1)
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, omse::rows_kernel<CPT, EXT>, threads, smem) != cudaSuccess || occ < 1)
             return OMSE_ECUDA;
-        ctx->seen[ctx->next_seen] = LaunchShape{CPT, threads, smem, occ};   // round robin once the table is full
+        ctx->seen[ctx->next_seen] = LaunchShape{slot, threads, smem, occ};   // round robin once the table is full
         ctx->next_seen = (ctx->next_seen + 1) % 16;
         if (ctx->n_seen < 16) ++ctx->n_seen;
     }
     long long grid = (long long)ctx->n_sm * occ;
     if (grid > a.n_units) grid = a.n_units;
-    omse::rows_kernel<CPT><<<(unsigned)grid, threads, smem, ctx->stream>>>(a);
+    omse::rows_kernel<CPT, EXT><<<(unsigned)grid, threads, smem, ctx->stream>>>(a);
     return cudaGetLastError() == cudaSuccess ? OMSE_OK : OMSE_ECUDA;
 }
 
@@ -170,11 +171,23 @@ int launch_rows(omse_ctx* ctx, omse::RowArgs& a, long long max_k, size_t smem_sm
     a.ticket = ctx->ws->ticket;
     a.status = &ctx->ws->status;
     a.evals = &ctx->ws->evals;
+    // the extended kernel only where a launch needs what it adds
+    bool ext = a.solver != 0 || a.n_delta > 0 || a.eps >= 0.f || a.sweeps_done != nullptr;
+    if (a.tensors == nullptr) ext = ext || a.one.gate || a.one.prior_alpha;
+    else ext = ext || a.ext_tensors;
+    if (ext) {
+        switch (cpt) {
+            case 1: return launch_rows_t<1, true>(ctx, a, smem);
+            case 2: return launch_rows_t<2, true>(ctx, a, smem);
+            case 4: return launch_rows_t<4, true>(ctx, a, smem);
+            default: return launch_rows_t<8, true>(ctx, a, smem);
+        }
+    }
     switch (cpt) {
-        case 1: return launch_rows_t<1>(ctx, a, smem);
-        case 2: return launch_rows_t<2>(ctx, a, smem);
-        case 4: return launch_rows_t<4>(ctx, a, smem);
-        default: return launch_rows_t<8>(ctx, a, smem);
+        case 1: return launch_rows_t<1, false>(ctx, a, smem);
+        case 2: return launch_rows_t<2, false>(ctx, a, smem);
+        case 4: return launch_rows_t<4, false>(ctx, a, smem);
+        default: return launch_rows_t<8, false>(ctx, a, smem);
     }
 }
 
@@ -297,6 +310,7 @@ int quantize_list(omse_ctx* ctx, std::vector<omse::RowTensor>& list, long long m
     memset(&a, 0, sizeof(a));
     a.n_launch_tensors = (int)list.size();
     a.n_units = units;
+    for (const auto& t : list) a.ext_tensors |= (t.gate || t.prior_alpha) ? 1 : 0;
     if (list.size() == 1) {
         a.tensors = nullptr;
         a.one = list[0];
@@ -422,6 +436,36 @@ int omse_read_evaluations(omse_ctx* ctx, uint64_t* host_out) {
     if (cudaMemsetAsync(&ctx->ws->evals, 0, sizeof(v), ctx->stream) != cudaSuccess) return OMSE_ECUDA;
     if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return OMSE_ECUDA;
     *host_out = v;
+    return OMSE_OK;
+}
+
+int omse_measure_fp32_peak(omse_ctx* ctx, int target_ms, double* host_out) {
+    if (!ctx || !host_out || target_ms < 1 || target_ms > 5000) return OMSE_EINVAL;
+    DeviceScope dev(ctx->device);
+    if (!dev.ok()) return OMSE_ECUDA;
+    const int blocks = ctx->n_sm * 4, threads = 256;
+    float* out = reinterpret_cast<float*>(ctx->partials);        // blocks*threads floats, far below the 16 MB held
+    // iterations for about target_ms at 128 lane operations per clock and SM at 2 GHz
+    const double lane_ops_per_iter = (double)blocks * threads * omse::kPeakChains * 2.0;
+    long long iters = (long long)((double)target_ms * 1e-3 * (double)ctx->n_sm * 128.0 * 2.0e9 / lane_ops_per_iter);
+    if (iters < 1024) iters = 1024;
+    if (iters > 0x7fffffff) iters = 0x7fffffff;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) {
+        if (e0) cudaEventDestroy(e0);
+        return OMSE_ECUDA;
+    }
+    omse::fma_peak_kernel<<<blocks, threads, 0, ctx->stream>>>(out, 4096, 1.0f);      // warm-up
+    cudaEventRecord(e0, ctx->stream);
+    omse::fma_peak_kernel<<<blocks, threads, 0, ctx->stream>>>(out, (int)iters, 1.0f);
+    cudaEventRecord(e1, ctx->stream);
+    float ms = 0.f;
+    const bool ok = cudaEventSynchronize(e1) == cudaSuccess && cudaEventElapsedTime(&ms, e0, e1) == cudaSuccess &&
+                    cudaGetLastError() == cudaSuccess && ms > 0.f;
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (!ok) return OMSE_ECUDA;
+    *host_out = lane_ops_per_iter * (double)iters / ((double)ms * 1e-3);
     return OMSE_OK;
 }
 

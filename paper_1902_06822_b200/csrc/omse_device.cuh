@@ -347,6 +347,29 @@ __device__ __forceinline__ void report_evaluations(unsigned long long* counter, 
     if ((threadIdx.x & 31) == 0 && mine) atomicAdd(counter, mine);
 }
 
+// Register-only loop of independent packed multiply-adds: measures the FP32 lane-operation rate of the FMA pipe,
+// the roof the candidate sweep is compared with.  Every thread runs kPeakChains chains of fma.rn.f32x2.
+constexpr int kPeakChains = 8;
+__global__ void __launch_bounds__(256) fma_peak_kernel(float* __restrict__ out, int iters, float seed) {
+    u64 v[kPeakChains];
+#pragma unroll
+    for (int s = 0; s < kPeakChains; ++s) v[s] = pack2(seed + 1e-3f * (float)(threadIdx.x + s), seed - 1e-3f * (float)s);
+    const u64 m = pack2(0.9999999f, 1.0000001f), c = pack2(1e-7f, -1e-7f);
+#pragma unroll 4
+    for (int i = 0; i < iters; ++i) {
+#pragma unroll
+        for (int s = 0; s < kPeakChains; ++s) v[s] = fma2(v[s], m, c);
+    }
+    float r = 0.f;
+#pragma unroll
+    for (int s = 0; s < kPeakChains; ++s) {
+        float a, b;
+        unpack2(v[s], a, b);
+        r += a + b;
+    }
+    out[(size_t)blockIdx.x * blockDim.x + threadIdx.x] = r;
+}
+
 // Per-candidate constants of one thread for the grid of Section 3.4 on a tensor with max|x| = m.
 // Candidate c has alpha_c = fl(fl(c+1)*step), step = fl(fl(hi_frac*m)/fl(C)), all binary32.
 // In the sweep x/alpha_c is replaced by x*inv_c with inv_c within 2 ulp of 1/alpha_c: a code can

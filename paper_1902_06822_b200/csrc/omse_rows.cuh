@@ -57,6 +57,7 @@ struct RowArgs {
     float off_frac;             // offsets span [min, min + off_frac*(max-min))
     float eps;                  // >= 0: Algorithm 1 stops after the first sweep whose relative error decrease is <= eps
     int* sweeps_done;           // [S] sweeps Algorithm 1 ran per row, nullable
+    int ext_tensors;            // a tensor of a batched launch has a gate or an earlier tensor's scale
 };
 
 }  // namespace omse
@@ -82,6 +83,16 @@ struct PhiCtl {
     int start_idx;    // >= 0: skip the search and start from this grid candidate
     int n_refine;     // polish steps
     bool want_sse;    // also return the fp64 error at the chosen candidate (before any polish)
+};
+
+// Per-row state of the pass loop of rows_kernel (shared memory; thread 0 writes between barriers).
+struct RowMode {
+    PhiCtl ctl;             // what the next phi_block call does
+    double aff_best;        // offset search: smallest error so far, its offset index and scale index
+    int aff_d, aff_c;
+    float aff_lo, aff_dstep, aff_dl;   // row minimum, offset step, offset of the current pass
+    double e_prev;          // Algorithm 1: error after the previous sweep
+    int sweeps_ran;
 };
 
 // ||x - alpha*[x/alpha]_Zp||^2 of the row in s.xs in fp64 with true division; every thread gets the sum.
@@ -243,7 +254,7 @@ __device__ void partition_row(const RowSmem& s, int k, const GridSetup& g, int t
 }
 
 // The quantization mapping phi of Section 3.4 on the row held in s.xs (k elements, k4 float4s).
-template <int CPT>
+template <int CPT, bool EXT>
 __device__ PhiOut phi_block(const RowArgs& a, const RowSmem& s, int k, int k4, float flo, float fhi,
                              const float (&rcp)[CPT], unsigned long long& ev, const PhiCtl& ctl) {
     const int tid = threadIdx.x, nthr = blockDim.x;
@@ -268,7 +279,7 @@ __device__ PhiOut phi_block(const RowArgs& a, const RowSmem& s, int k, int k4, f
     out.sse = 0.0;
     out.idx = -1;
     out.degenerate = true;
-    if (ctl.solver != 0) {
+    if (EXT && ctl.solver != 0) {
         // ---- comparison solvers of Section 3.4: another way to the starting scale, then the same polish
         float alpha = 0.f;
         if (ctl.solver == 3) {
@@ -312,9 +323,9 @@ __device__ PhiOut phi_block(const RowArgs& a, const RowSmem& s, int k, int k4, f
         return out;
     }
     if (!(m > 0.f) || !(a_last >= FLT_MIN)) return out;   // no usable scale: alpha = 0, all codes 0
-    if (ctl.start_idx >= 0) {
+    if (EXT && ctl.start_idx >= 0) {
         const float ac = __fmul_rn((float)(ctl.start_idx + 1), g.step);
-        if (!(ac >= FLT_MIN)) return out;
+        if (!(ac >= FLT_MIN) || ctl.start_idx >= a.n_cand) return out;
         out.degenerate = false;
         out.idx = ctl.start_idx;
         out.alpha = polish_block(s.xs, k, ac, flo, fhi, ctl.n_refine, s.scratch);
@@ -434,9 +445,9 @@ __device__ PhiOut phi_block(const RowArgs& a, const RowSmem& s, int k, int k4, f
 
     // ---- polish: alpha <- <x,q>/<q,q>, q = [x/alpha]_Zp
     const float a_grid = __fmul_rn((float)(best + 1), g.step);
-    if (ctl.want_sse)
+    if (EXT && ctl.want_sse)
         out.sse = best_sse < INFINITY ? best_sse : exact_sse_block(s.xs, k, a_grid, flo, fhi, s.scratch);
-    out.alpha = polish_block(s.xs, k, a_grid, flo, fhi, ctl.n_refine, s.scratch);
+    out.alpha = polish_block(s.xs, k, a_grid, flo, fhi, EXT ? ctl.n_refine : a.refine_iters, s.scratch);
     out.idx = best;
     return out;
 }
@@ -512,10 +523,14 @@ __device__ double emit_block(const RowSmem& s, int k, float alpha, float flo, fl
     return ss;
 }
 
-template <int CPT>
+// EXT = false: the grid search with polish (and Algorithm 1 with a fixed number of sweeps) and nothing else, so that
+// the common launches keep their register allocation and code size; EXT = true adds the comparison solvers, the offset
+// search, Algorithm 1's loop condition, gated layers and rows that start from an earlier tensor's residual.
+template <int CPT, bool EXT>
 __global__ void __launch_bounds__(OMSE_ROWS_MAX_THREADS) rows_kernel(const RowArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ unsigned long long s_unit;
+    __shared__ RowMode s_mode;
     const int tid = threadIdx.x, nthr = blockDim.x;
     RowSmem s;
     s.xs = reinterpret_cast<float*>(smem_raw);
@@ -548,13 +563,13 @@ __global__ void __launch_bounds__(OMSE_ROWS_MAX_THREADS) rows_kernel(const RowAr
             tp = a.tensors + ti;
         }
         const RowTensor& T = *tp;
-        if (T.gate && *T.gate == 0) continue;   // not a key layer: nothing to do for this unit
+        if (EXT && T.gate && *T.gate == 0) continue;   // not a key layer: nothing to do for this unit
         if (T.small & 4) {
             tiny_dispatch<CPT>(a, T, unit - T.unit_begin, smem_raw, st, ev);
             continue;
         }
         if (T.small) {
-            small_unit<CPT>(a, T, unit - T.unit_begin, smem_raw, rcp, st, ev);
+            small_unit<CPT, EXT>(a, T, unit - T.unit_begin, smem_raw, rcp, st, ev);
             continue;
         }
         const int k = (int)T.K;
@@ -592,7 +607,7 @@ __global__ void __launch_bounds__(OMSE_ROWS_MAX_THREADS) rows_kernel(const RowAr
                 }
             }
             if (bad) st |= 1u;
-            if (T.prior_alpha) {
+            if (EXT && T.prior_alpha) {
                 // second quantized tensor of a key layer: the row becomes the residual of the first tensor
                 __syncthreads();
                 const float a1 = T.prior_alpha[row];
@@ -603,7 +618,7 @@ __global__ void __launch_bounds__(OMSE_ROWS_MAX_THREADS) rows_kernel(const RowAr
                         s.xs[i] = fmaf(-a1, (float)code_of(x, a1, flo0, fhi0), x);
                     }
             }
-            if (T.delta && a.n_delta == 0) {
+            if (T.delta && !(EXT && a.n_delta > 0)) {
                 // quantization with offset: delta = min of the row, the shifted row fl(x - delta) is what gets searched
                 __syncthreads();
                 float lo = INFINITY;
@@ -628,11 +643,16 @@ __global__ void __launch_bounds__(OMSE_ROWS_MAX_THREADS) rows_kernel(const RowAr
             }
             __syncthreads();
 
-            if (a.n_delta > 0) {
-                // ---- offset scheme of Section 3.1 with the offset searched as well: for every offset on the grid
-                //      the line search of the shifted row fl(x - delta); the pair with the smallest error wins
-                //      (lowest offset, then lowest scale index, on equal errors); polish and codes at that pair
-                const float flo = (float)a.lo[0], fhi = (float)a.hi[0];
+            // ---- The row goes through phi one or more times; all modes share the one call below.
+            //  * default / Algorithm 1 (Section 3.5): pass = (sweep, tensor j); the residual of the other tensors is
+            //    quantized; one tensor and one sweep is plain phi.
+            //  * offset searched as well (Section 3.1 scheme, a.n_delta > 0): passes 0..n_delta-1 run the line search
+            //    on the row shifted by offset d and keep the pair with the smallest error (lowest offset, then lowest
+            //    scale index, on equal errors); the last pass polishes and emits at that pair.
+            // Everything that steers the passes lives in shared memory (s_mode), not in registers: the sweep inside
+            // phi_block needs the whole register budget.
+            const bool affine = EXT && a.n_delta > 0;
+            if (affine) {
                 float lo = INFINITY, hi = -INFINITY;   // extremes of the finite values of the row
                 for (int i = tid; i < k; i += nthr) {
                     const float v = s.x0[i];
@@ -652,112 +672,118 @@ __global__ void __launch_bounds__(OMSE_ROWS_MAX_THREADS) rows_kernel(const RowAr
                     s_ext[1][tid >> 5] = hi;
                 }
                 __syncthreads();
-                lo = INFINITY;
-                hi = -INFINITY;
-                for (int w = 0; w < ((nthr + 31) >> 5); ++w) {
-                    lo = fminf(lo, s_ext[0][w]);
-                    hi = fmaxf(hi, s_ext[1][w]);
+                if (tid == 0) {
+                    lo = INFINITY;
+                    hi = -INFINITY;
+                    for (int w = 0; w < ((nthr + 31) >> 5); ++w) {
+                        lo = fminf(lo, s_ext[0][w]);
+                        hi = fmaxf(hi, s_ext[1][w]);
+                    }
+                    if (!(lo <= hi)) lo = hi = 0.f;
+                    s_mode.aff_lo = lo;
+                    s_mode.aff_dstep = __fdiv_rn(__fmul_rn(a.off_frac, __fsub_rn(hi, lo)), (float)a.n_delta);
+                    s_mode.aff_best = INFINITY;
+                    s_mode.aff_d = -1;
+                    s_mode.aff_c = -1;
                 }
-                if (!(lo <= hi)) lo = hi = 0.f;
-                const float dstep = __fdiv_rn(__fmul_rn(a.off_frac, __fsub_rn(hi, lo)), (float)a.n_delta);
-                double best_sse = INFINITY;
-                int best_d = -1, best_c = -1;
-                PhiCtl search = {0, 0, -1, 0, true};
-                for (int d = 0; d < a.n_delta; ++d) {
-                    const float dl = __fadd_rn(lo, __fmul_rn((float)d, dstep));
+            }
+            if (EXT && a.eps >= 0.f) {
+                // Algorithm 1: error before the first sweep (all tensors zero) is ||T||^2
+                double e0 = 0.0;
+                long long zero = 0;
+                for (int i = tid; i < k; i += nthr) e0 += (double)s.xs[i] * (double)s.xs[i];
+                block_sum2(e0, zero, s.scratch);
+                if (tid == 0) s_mode.e_prev = e0;
+            }
+            if (EXT && tid == 0) s_mode.sweeps_ran = 0;
+            const int n_pass = affine ? a.n_delta + 1 : a.n_sweeps * a.n_tensors;
+            for (int pass = 0; pass < n_pass; ++pass) {
+                const int sweep = affine ? 0 : pass / a.n_tensors;
+                const int j = affine ? 0 : pass - sweep * a.n_tensors;
+                if (EXT) __syncthreads();   // every thread is done with the previous pass's control block
+                if (EXT && tid == 0) {
+                    PhiCtl c = {a.solver, a.solver_iters, -1, a.refine_iters, false};
+                    if (affine) {
+                        const bool last = pass == a.n_delta;
+                        if (last) {
+                            c.start_idx = s_mode.aff_d >= 0 ? s_mode.aff_c : a.n_cand;   // n_cand: no offset had a usable scale
+                        } else {
+                            c.n_refine = 0;
+                            c.want_sse = true;
+                        }
+                        s_mode.aff_dl = __fadd_rn(s_mode.aff_lo, __fmul_rn((float)(last ? max(s_mode.aff_d, 0) : pass), s_mode.aff_dstep));
+                    }
+                    s_mode.ctl = c;
+                }
+                if (affine) {
                     __syncthreads();
+                    const float dl = s_mode.aff_dl;
                     for (int i = tid; i < 4 * k4; i += nthr) s.xs[i] = i < k ? __fsub_rn(s.x0[i], dl) : 0.f;
                     __syncthreads();
-                    const PhiOut r = phi_block<CPT>(a, s, k, k4, flo, fhi, rcp, ev, search);
-                    if (!r.degenerate && r.sse < best_sse) {   // increasing offset: strict < keeps the lowest flat index
-                        best_sse = r.sse;
-                        best_d = d;
-                        best_c = r.idx;
+                } else if (a.keep_x0 && pass > 0) {
+                    // residual T - sum_{i != j} alpha_i q^i from the original row, increasing i
+                    for (int i = tid; i < k; i += nthr) {
+                        float v = s.x0[i];
+                        for (int i2 = 0; i2 < a.n_tensors; ++i2) {
+                            if (i2 == j || (sweep == 0 && i2 > j)) continue;
+                            const float ai = T.alpha[(long long)i2 * T.S + row];
+                            const float qi = (float)T.codes[(long long)i2 * n_total + row_base + i];
+                            v = fmaf(-ai, qi, v);
+                        }
+                        s.xs[i] = v;
                     }
+                    __syncthreads();
                 }
-                const float dl = __fadd_rn(lo, __fmul_rn((float)max(best_d, 0), dstep));
-                __syncthreads();
-                for (int i = tid; i < 4 * k4; i += nthr) s.xs[i] = i < k ? __fsub_rn(s.x0[i], dl) : 0.f;
-                __syncthreads();
-                PhiOut r;
-                r.alpha = 0.f;
-                r.idx = -1;
-                r.degenerate = true;
-                if (best_d >= 0) {
-                    const PhiCtl from = {0, 0, best_c, a.refine_iters, false};
-                    r = phi_block<CPT>(a, s, k, k4, flo, fhi, rcp, ev, from);
+                const float flo = (float)a.lo[j], fhi = (float)a.hi[j];
+                PhiOut r = phi_block<CPT, EXT>(a, s, k, k4, flo, fhi, rcp, ev, s_mode.ctl);
+                if (affine && pass < a.n_delta) {
+                    if (tid == 0 && !r.degenerate && r.sse < s_mode.aff_best) {   // increasing offset: strict < keeps the lowest flat index
+                        s_mode.aff_best = r.sse;
+                        s_mode.aff_d = pass;
+                        s_mode.aff_c = r.idx;
+                    }
+                    continue;      // the barriers of the next pass order these writes before their readers
                 }
                 if (r.degenerate) st |= 2u;
-                const double sse = emit_block(s, k, r.alpha, flo, fhi, T.codes, T.packed, row_base, &s.misc[1], more);
+                const double sse = emit_block(s, k, r.alpha, flo, fhi,
+                                              T.codes ? T.codes + (long long)j * n_total : nullptr,
+                                              T.packed ? T.packed + (long long)j * packed_stride : nullptr,
+                                              row_base, &s.misc[1 + j], more);
                 if (tid == 0) {
-                    T.alpha[row] = r.alpha;
-                    T.sse[row] = (float)sse;
-                    if (T.delta) T.delta[row] = dl;
-                    if (T.best_idx) T.best_idx[row] = r.degenerate ? -1 : best_d * a.n_cand + best_c;
-                }
-                __syncthreads();
-                continue;
-            }
-
-            // ---- Algorithm 1: sweeps over the tensors; one tensor and one sweep is plain phi
-            double e_prev = 0.0;                   // error before the current sweep (all tensors zero: ||T||^2)
-            if (a.eps >= 0.f) {
-                long long zero = 0;
-                for (int i = tid; i < k; i += nthr) e_prev += (double)s.xs[i] * (double)s.xs[i];
-                block_sum2(e_prev, zero, s.scratch);
-            }
-            int sweeps_ran = 0;
-            const PhiCtl ctl = {a.solver, a.solver_iters, -1, a.refine_iters, false};
-            for (int sweep = 0; sweep < a.n_sweeps; ++sweep) {
-                double e_cur = 0.0;
-                for (int j = 0; j < a.n_tensors; ++j) {
-                    const float flo = (float)a.lo[j], fhi = (float)a.hi[j];
-                    if (a.keep_x0 && !(sweep == 0 && j == 0)) {
-                        // residual T - sum_{i != j} alpha_i q^i from the original row, increasing i
-                        for (int i = tid; i < k; i += nthr) {
-                            float v = s.x0[i];
-                            for (int i2 = 0; i2 < a.n_tensors; ++i2) {
-                                if (i2 == j || (sweep == 0 && i2 > j)) continue;
-                                const float ai = T.alpha[(long long)i2 * T.S + row];
-                                const float qi = (float)T.codes[(long long)i2 * n_total + row_base + i];
-                                v = fmaf(-ai, qi, v);
-                            }
-                            s.xs[i] = v;
-                        }
-                        __syncthreads();
+                    T.alpha[(long long)j * T.S + row] = r.alpha;
+                    T.sse[(long long)j * T.S + row] = (float)sse;
+                    if (a.sse_history) a.sse_history[((long long)sweep * a.n_tensors + j) * T.S + row] = (float)sse;
+                    if (affine) {
+                        if (T.delta) T.delta[row] = s_mode.aff_dl;
+                        if (T.best_idx) T.best_idx[row] = r.degenerate ? -1 : s_mode.aff_d * a.n_cand + s_mode.aff_c;
+                    } else if (T.best_idx && j == 0) {
+                        T.best_idx[row] = r.idx;
                     }
-                    PhiOut r = phi_block<CPT>(a, s, k, k4, flo, fhi, rcp, ev, ctl);
-                    if (r.degenerate) st |= 2u;
-                    const double sse = emit_block(s, k, r.alpha, flo, fhi,
-                                                  T.codes ? T.codes + (long long)j * n_total : nullptr,
-                                                  T.packed ? T.packed + (long long)j * packed_stride : nullptr,
-                                                  row_base, &s.misc[1 + j], more);
-                    e_cur = sse;
-                    if (tid == 0) {
-                        T.alpha[(long long)j * T.S + row] = r.alpha;
-                        T.sse[(long long)j * T.S + row] = (float)sse;
-                        if (a.sse_history) a.sse_history[((long long)sweep * a.n_tensors + j) * T.S + row] = (float)sse;
-                        if (T.best_idx && j == 0) T.best_idx[row] = r.idx;
-                    }
-                    if (!a.keep_x0 && j + 1 < a.n_tensors) {
-                        // first sweep without a kept copy: the residual is updated in place
-                        for (int i = tid; i < k; i += nthr) {
-                            const float x = s.xs[i];
-                            const int q = r.alpha > 0.f ? code_of(x, r.alpha, flo, fhi) : 0;
-                            s.xs[i] = fmaf(-r.alpha, (float)q, x);
-                        }
-                    }
-                    __syncthreads();   // alpha / codes of tensor j visible to the block (global + shared)
                 }
-                sweeps_ran = sweep + 1;
-                if (a.eps >= 0.f) {
-                    // while-condition of Algorithm 1: go on while the sweep lowered the error by more than eps (relative)
-                    const bool go_on = (e_prev - e_cur) > (double)a.eps * e_prev;
-                    e_prev = e_cur;
-                    if (!go_on) break;
+                if (!a.keep_x0 && j + 1 < a.n_tensors) {
+                    // first sweep without a kept copy: the residual is updated in place
+                    for (int i = tid; i < k; i += nthr) {
+                        const float x = s.xs[i];
+                        const int q = r.alpha > 0.f ? code_of(x, r.alpha, flo, fhi) : 0;
+                        s.xs[i] = fmaf(-r.alpha, (float)q, x);
+                    }
                 }
+                bool stop = false;
+                if (EXT && j == a.n_tensors - 1) {
+                    if (tid == 0) s_mode.sweeps_ran = sweep + 1;
+                    if (a.eps >= 0.f) {
+                        // loop condition of Algorithm 1: go on while the sweep lowered the error by more than eps (relative);
+                        // every thread holds the same sse, so the decision is uniform
+                        const double e_prev = s_mode.e_prev;
+                        stop = !((e_prev - sse) > (double)a.eps * e_prev);
+                    }
+                }
+                __syncthreads();   // alpha / codes of tensor j visible to the block (global + shared); e_prev read by all
+                if (EXT && j == a.n_tensors - 1 && a.eps >= 0.f && tid == 0) s_mode.e_prev = sse;
+                if (stop) break;
             }
-            if (tid == 0) {
+            const int sweeps_ran = EXT ? s_mode.sweeps_ran : a.n_sweeps;
+            if (EXT && tid == 0 && !affine) {
                 if (a.sweeps_done) a.sweeps_done[row] = sweeps_ran;
                 if (a.sse_history)     // sweeps that did not run repeat the last error
                     for (int sweep = sweeps_ran; sweep < a.n_sweeps; ++sweep)

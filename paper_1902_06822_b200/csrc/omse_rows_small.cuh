@@ -250,7 +250,7 @@ __device__ __forceinline__ float small_row_epilogue(const RowArgs& a, const RowT
 
 // One work unit of the short-row path: rows [unit_local*B, +B) of tensor T.  Requires a single
 // element group (blockDim.x == a.tg) and a single quantized tensor per row.
-template <int CPT>
+template <int CPT, bool EXT>
 __device__ void small_unit(const RowArgs& a, const RowTensor& T, long long unit_local, unsigned char* smem_raw,
                            const float (&rcp)[CPT], unsigned int& st, unsigned long long& ev) {
     const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
@@ -295,7 +295,7 @@ __device__ void small_unit(const RowArgs& a, const RowTensor& T, long long unit_
     }
     if (bad) st |= 1u;
     __syncthreads();
-    if (T.prior_alpha) {
+    if (EXT && T.prior_alpha) {
         // second quantized tensor of a key layer: every row becomes the residual of its first tensor
         for (int i = tid; i < nrows * kpad; i += nthr) {
             const int r = i / kpad, c = i - r * kpad;

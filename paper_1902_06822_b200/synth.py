@@ -12,6 +12,9 @@ regenerated independently and results do not depend on chunking.
 """
 from __future__ import annotations
 
+import os
+from concurrent.futures import ThreadPoolExecutor
+
 import numpy as np
 
 _GOLDEN = np.uint64(0x9E3779B97F4A7C15)
@@ -52,30 +55,47 @@ def _chunks(n):
         yield s, min(_CHUNK, n - s)
 
 
+def _for_chunks(n, work):
+    """work(start, count) for every chunk; chunks are independent (counter-based), so they run on host threads."""
+    chunks = list(_chunks(n))
+    if len(chunks) <= 1:
+        for s, c in chunks:
+            work(s, c)
+        return
+    with ThreadPoolExecutor(max_workers=min(len(chunks), os.cpu_count() or 1)) as ex:
+        list(ex.map(lambda sc: work(*sc), chunks))
+
+
 def laplace(n: int, b: float, seed: int, tensor_id: int = 0) -> np.ndarray:
     """Laplace(0, b) by inverse CDF."""
     out = np.empty(n, np.float32)
-    for s, c in _chunks(n):
+
+    def work(s, c):
         u = uniform01(seed, tensor_id, 0, s, c) - 0.5
         out[s:s + c] = (-b * np.sign(u) * np.log1p(-2.0 * np.abs(u))).astype(np.float32)
+    _for_chunks(n, work)
     return out
 
 
 def student_t3(n: int, seed: int, tensor_id: int = 0) -> np.ndarray:
     """Student-t with 3 degrees of freedom, unit scale: Z / sqrt((Z1^2+Z2^2+Z3^2)/3)."""
     out = np.empty(n, np.float32)
-    for s, c in _chunks(n):
+
+    def work(s, c):
         z = _normal(seed, tensor_id, 0, s, c)
         chi = sum(_normal(seed, tensor_id, l, s, c) ** 2 for l in (1, 2, 3))
         out[s:s + c] = (z / np.sqrt(chi / 3.0)).astype(np.float32)
+    _for_chunks(n, work)
     return out
 
 
 def relu_activations(n: int, seed: int, zero_prob: float = 0.4, tensor_id: int = 0) -> np.ndarray:
     """Post-ReLU stand-in: |t_3| magnitudes, each element exactly zero with probability zero_prob."""
     out = np.abs(student_t3(n, seed, tensor_id))
-    for s, c in _chunks(n):
+
+    def work(s, c):
         out[s:s + c][uniform01(seed, tensor_id, 15, s, c) < zero_prob] = 0.0
+    _for_chunks(n, work)
     return out
 
 
@@ -84,10 +104,12 @@ def laplace_with_outliers(n: int, b: float, seed: int, outlier_prob: float = 1e-
     """Laplace(0, b); with probability outlier_prob an element becomes +-n_sigma*sigma, sigma = b*sqrt(2)."""
     out = laplace(n, b, seed, tensor_id)
     mag = np.float32(n_sigma * b * np.sqrt(2.0))
-    for s, c in _chunks(n):
+
+    def work(s, c):
         hit = uniform01(seed, tensor_id, 14, s, c) < outlier_prob
         sign = np.where(uniform01(seed, tensor_id, 13, s, c) < 0.5, np.float32(-1), np.float32(1))
         out[s:s + c] = np.where(hit, sign * mag, out[s:s + c])
+    _for_chunks(n, work)
     return out
 
 

@@ -67,6 +67,7 @@ struct omse_ctx {
     bool attr_rows[8], attr_tensor[4], attr_dual;   // opt-in shared-memory attribute set, per template instance
     LaunchShape seen[16];                           // blocks per SM of the row-kernel launch shapes met so far
     int n_seen, next_seen;
+    int occ_sweep[2], occ_pass[3];                  // blocks per SM of the per-tensor kernels (0 = not yet asked)
 };
 
 namespace {
@@ -222,26 +223,97 @@ bool single_group(int n_cand, long long max_k) {
 
 bool misaligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3) != 0; }
 
+// ---- per-tensor search: the launches shared by omse_activation_scale* and the allocation-free entry point
+struct TensorEnv {
+    int n_sm;
+    cudaStream_t stream;
+    int* occ_sweep;      // [2] blocks per SM of the two sweep launch shapes (0 = not yet asked), cached by the caller
+    int* occ_pass;       // [3] blocks per SM of the three pass kernels
+    bool opt_in_smem;    // the sweep may ask for more than 48 KB of dynamic shared memory (context path only)
+    bool* attr_tensor;   // [4] per CPT: opt-in attribute already set
+};
+
 template <int CPT>
-int launch_tensor_sweep_t(omse_ctx* ctx, omse::TensorArgs& a, size_t smem, int* n_blocks) {
-    if (!ctx->attr_tensor[cpt_slot(CPT)]) {
+int sweep_launch_t(const TensorEnv& env, omse::TensorArgs& a, size_t smem, int occ_slot, int* n_blocks) {
+    if (env.opt_in_smem && smem > 48 * 1024 && !env.attr_tensor[cpt_slot(CPT)]) {
         if (cudaFuncSetAttribute(omse::tensor_sweep_kernel<CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess)
             return OMSE_ECUDA;
-        ctx->attr_tensor[cpt_slot(CPT)] = true;
+        env.attr_tensor[cpt_slot(CPT)] = true;
     }
     const int threads = a.groups * a.tg;
     int occ = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, omse::tensor_sweep_kernel<CPT>, threads, smem) != cudaSuccess || occ < 1)
         return OMSE_ECUDA;
+    (void)occ_slot;
     const long long n4 = (a.n + 3) >> 2;
     const long long n_tiles = (n4 + a.tile4 - 1) / a.tile4;
-    long long grid = (long long)ctx->n_sm * occ;
-    const long long cap = (long long)(kPartialBytes / ((size_t)a.n_cand * 8));
+    long long grid = (long long)env.n_sm * occ;
+    const long long cap = a.partial_doubles / a.n_cand;
     if (grid > cap) grid = cap;
     if (grid > n_tiles) grid = n_tiles;
     if (grid < 1) grid = 1;
     *n_blocks = (int)grid;
-    omse::tensor_sweep_kernel<CPT><<<(unsigned)grid, threads, smem, ctx->stream>>>(a);
+    omse::tensor_sweep_kernel<CPT><<<(unsigned)grid, threads, smem, env.stream>>>(a);
+    return cudaGetLastError() == cudaSuccess ? OMSE_OK : OMSE_ECUDA;
+}
+
+// One sweep launch over the candidates [c_base, c_base + c_count) with `cpt` candidates per thread.
+int sweep_launch(const TensorEnv& env, omse::TensorArgs a, int c_base, int c_count, int cpt, int occ_slot, int* n_blocks) {
+    a.c_base = c_base;
+    a.c_count = c_count;
+    a.tg = (((c_count + cpt - 1) / cpt) + 31) & ~31;
+    a.groups = 256 / a.tg < 1 ? 1 : 256 / a.tg;
+    a.tile4 = 4 * a.groups * a.tg;   // every thread stages exactly four float4s of a tile
+    const size_t smem = (size_t)a.tile4 * 16 + (size_t)cpt * 16 + (size_t)(a.groups - 1) * cpt * a.tg * 8;
+    if (!env.opt_in_smem && smem > 48 * 1024) return OMSE_ELIMIT;
+    switch (cpt) {
+        case 1: return sweep_launch_t<1>(env, a, smem, occ_slot, n_blocks);
+        case 2: return sweep_launch_t<2>(env, a, smem, occ_slot, n_blocks);
+        case 4: return sweep_launch_t<4>(env, a, smem, occ_slot, n_blocks);
+        default: return sweep_launch_t<8>(env, a, smem, occ_slot, n_blocks);
+    }
+}
+
+template <int MODE>
+int pass_grid(const TensorEnv& env, long long n) {
+    int& occ = env.occ_pass[MODE];
+    if (occ == 0 && (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, omse::tensor_pass_kernel<MODE>, 256, 0) != cudaSuccess || occ < 1))
+        occ = 4;
+    long long grid = (n + 1023) / 1024;            // at least one float4 per thread
+    if (grid > (long long)env.n_sm * occ) grid = (long long)env.n_sm * occ;   // one wave: every block is resident
+    return grid < 1 ? 1 : (int)grid;
+}
+
+// Everything after the state has been cleared: maxima, sweep (one or two launches), curve, argmin, re-score, polish,
+// final error.  `a` carries the buffers; grid fields are filled here.
+int enqueue_tensor_search(const TensorEnv& env, omse::TensorArgs& a, int refine_iters) {
+    cudaStream_t s = env.stream;
+    const long long n = a.n;
+    long long absmax_grid = (n + 1023) / 1024;
+    if (absmax_grid > (long long)env.n_sm * 8) absmax_grid = (long long)env.n_sm * 8;
+    if (absmax_grid < 1) absmax_grid = 1;
+    const int kFine = 256;        // candidates of the first launch: 32 per slot
+    int split = a.n_cand, nb_lo = 1, nb_hi = 1;
+    if (n > 0) {
+        omse::tensor_absmax_kernel<<<(unsigned)absmax_grid, 256, 0, s>>>(a.x, n, a.st, a.status);
+        if (a.delta_out) omse::tensor_offset_kernel<<<1, 32, 0, s>>>(a.st);
+        int rc;
+        if (a.n_cand <= kFine) {
+            rc = sweep_launch(env, a, 0, a.n_cand, cpt_for(a.n_cand), 0, &nb_lo);
+            nb_hi = nb_lo;
+        } else {
+            split = kFine;
+            rc = sweep_launch(env, a, 0, kFine, 8, 0, &nb_lo);
+            if (rc == OMSE_OK) rc = sweep_launch(env, a, kFine, a.n_cand - kFine, 8, 1, &nb_hi);
+        }
+        if (rc != OMSE_OK) return rc;
+    }
+    omse::tensor_curve_kernel<<<(unsigned)((a.n_cand + 31) / 32), 256, 0, s>>>(a, split, nb_lo, nb_hi);
+    omse::tensor_finish_kernel<<<1, 1024, 0, s>>>(a);
+    omse::tensor_pass_kernel<0><<<(unsigned)pass_grid<0>(env, n), 256, 0, s>>>(a);
+    const int g1 = pass_grid<1>(env, n);
+    for (int it = 0; it < refine_iters; ++it) omse::tensor_pass_kernel<1><<<(unsigned)g1, 256, 0, s>>>(a);
+    omse::tensor_pass_kernel<2><<<(unsigned)pass_grid<2>(env, n), 256, 0, s>>>(a);
     return cudaGetLastError() == cudaSuccess ? OMSE_OK : OMSE_ECUDA;
 }
 
@@ -812,10 +884,6 @@ static int activation_impl(omse_ctx* ctx, const float* d_x, int64_t n, int bits,
     a.n_cand = grid->n_cand;
     a.hi_frac = grid->hi_frac;
     bounds(bits, is_signed, &a.lo, &a.hi);
-    const int cpt = cpt_for(a.n_cand);
-    a.tg = (((a.n_cand + cpt - 1) / cpt) + 31) & ~31;
-    a.groups = 256 / a.tg < 1 ? 1 : 256 / a.tg;
-    a.tile4 = 4 * a.groups * a.tg;   // every thread stages exactly four float4s of a tile
     a.st = &ctx->ws->tstate;
     a.partials = ctx->partials;
     a.partial_doubles = (long long)(kPartialBytes / 8);
@@ -828,32 +896,9 @@ static int activation_impl(omse_ctx* ctx, const float* d_x, int64_t n, int bits,
     a.delta_out = d_delta;
     a.evals = &ctx->ws->evals;
     a.status = &ctx->ws->status;
-    cudaStream_t s = ctx->stream;
-
-    omse::tensor_init_kernel<<<1, 32, 0, s>>>(a.st);
-    long long pass_grid = (n + 1023) / 1024;
-    if (pass_grid > (long long)ctx->n_sm * 8) pass_grid = (long long)ctx->n_sm * 8;
-    if (pass_grid < 1) pass_grid = 1;
-    int n_blocks = 1;
-    if (n > 0) {
-        omse::tensor_absmax_kernel<<<(unsigned)pass_grid, 256, 0, s>>>(d_x, n, a.st, a.status);
-        if (d_delta) omse::tensor_offset_kernel<<<1, 32, 0, s>>>(a.st);
-        const size_t smem = (size_t)a.tile4 * 16 + (size_t)cpt * 16 + (size_t)(a.groups - 1) * cpt * a.tg * 8;
-        int rc;
-        switch (cpt) {
-            case 1: rc = launch_tensor_sweep_t<1>(ctx, a, smem, &n_blocks); break;
-            case 2: rc = launch_tensor_sweep_t<2>(ctx, a, smem, &n_blocks); break;
-            case 4: rc = launch_tensor_sweep_t<4>(ctx, a, smem, &n_blocks); break;
-            default: rc = launch_tensor_sweep_t<8>(ctx, a, smem, &n_blocks); break;
-        }
-        if (rc != OMSE_OK) return rc;
-    }
-    omse::tensor_curve_kernel<<<(unsigned)((a.n_cand + 63) / 64), 64, 0, s>>>(a, n_blocks);
-    omse::tensor_finish_kernel<<<1, 1024, 0, s>>>(a);
-    omse::tensor_pass_kernel<0><<<(unsigned)pass_grid, 256, 0, s>>>(a);
-    for (int it = 0; it < grid->refine_iters; ++it) omse::tensor_pass_kernel<1><<<(unsigned)pass_grid, 256, 0, s>>>(a);
-    omse::tensor_pass_kernel<2><<<(unsigned)pass_grid, 256, 0, s>>>(a);
-    return cudaGetLastError() == cudaSuccess ? OMSE_OK : OMSE_ECUDA;
+    omse::tensor_init_kernel<<<1, 32, 0, ctx->stream>>>(a.st);
+    const TensorEnv env = {ctx->n_sm, ctx->stream, ctx->occ_sweep, ctx->occ_pass, true, ctx->attr_tensor};
+    return enqueue_tensor_search(env, a, grid->refine_iters);
 }
 
 extern "C" {
@@ -900,6 +945,8 @@ struct StaticDevice {
     StaticScratch* ptr;   // device address of g_static_scratch on this device
     int n_sm;
     bool ready;
+    int occ_sweep[2], occ_pass[3];
+    bool attr_unused[4];
 };
 StaticDevice g_static_dev[64];
 std::mutex g_static_mutex;
@@ -925,24 +972,6 @@ __global__ void static_begin_kernel(StaticScratch* s) {
 
 __global__ void static_end_kernel(const StaticScratch* s, unsigned int* d_status) {
     if (threadIdx.x == 0 && d_status) *d_status = s->status;
-}
-
-template <int CPT>
-int launch_static_sweep_t(int n_sm, cudaStream_t stream, omse::TensorArgs& a, size_t smem, int* n_blocks) {
-    const int threads = a.groups * a.tg;
-    int occ = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, omse::tensor_sweep_kernel<CPT>, threads, smem) != cudaSuccess || occ < 1)
-        return OMSE_ECUDA;
-    const long long n4 = (a.n + 3) >> 2;
-    const long long n_tiles = (n4 + a.tile4 - 1) / a.tile4;
-    long long grid = (long long)n_sm * occ;
-    const long long cap = (long long)(kStaticPartialDoubles / (size_t)a.n_cand);
-    if (grid > cap) grid = cap;
-    if (grid > n_tiles) grid = n_tiles;
-    if (grid < 1) grid = 1;
-    *n_blocks = (int)grid;
-    omse::tensor_sweep_kernel<CPT><<<(unsigned)grid, threads, smem, stream>>>(a);
-    return cudaGetLastError() == cudaSuccess ? OMSE_OK : OMSE_ECUDA;
 }
 
 }  // namespace
@@ -981,10 +1010,6 @@ extern "C" int omse_activation_scale_static(int device, void* cuda_stream, const
     a.n_cand = grid->n_cand;
     a.hi_frac = grid->hi_frac;
     bounds(bits, is_signed, &a.lo, &a.hi);
-    const int cpt = cpt_for(a.n_cand);
-    a.tg = (((a.n_cand + cpt - 1) / cpt) + 31) & ~31;
-    a.groups = 256 / a.tg < 1 ? 1 : 256 / a.tg;
-    a.tile4 = 4 * a.groups * a.tg;   // every thread stages exactly four float4s of a tile
     a.st = &sc->tstate;
     a.partials = sc->partials;
     a.partial_doubles = (long long)kStaticPartialDoubles;
@@ -997,27 +1022,10 @@ extern "C" int omse_activation_scale_static(int device, void* cuda_stream, const
     a.status = &sc->status;
 
     static_begin_kernel<<<1, 32, 0, s>>>(sc);
-    long long pass_grid = (n + 1023) / 1024;
-    if (pass_grid > (long long)sd.n_sm * 8) pass_grid = (long long)sd.n_sm * 8;
-    if (pass_grid < 1) pass_grid = 1;
-    int n_blocks = 1;
-    if (n > 0) {
-        omse::tensor_absmax_kernel<<<(unsigned)pass_grid, 256, 0, s>>>(d_x, n, a.st, a.status);
-        const size_t smem = (size_t)a.tile4 * 16 + (size_t)cpt * 16 + (size_t)(a.groups - 1) * cpt * a.tg * 8;   // < 48 KB: no opt-in needed
-        int rc;
-        switch (cpt) {
-            case 1: rc = launch_static_sweep_t<1>(sd.n_sm, s, a, smem, &n_blocks); break;
-            case 2: rc = launch_static_sweep_t<2>(sd.n_sm, s, a, smem, &n_blocks); break;
-            case 4: rc = launch_static_sweep_t<4>(sd.n_sm, s, a, smem, &n_blocks); break;
-            default: rc = launch_static_sweep_t<8>(sd.n_sm, s, a, smem, &n_blocks); break;
-        }
-        if (rc != OMSE_OK) return rc;
-    }
-    omse::tensor_curve_kernel<<<(unsigned)((a.n_cand + 63) / 64), 64, 0, s>>>(a, n_blocks);
-    omse::tensor_finish_kernel<<<1, 1024, 0, s>>>(a);
-    omse::tensor_pass_kernel<0><<<(unsigned)pass_grid, 256, 0, s>>>(a);
-    for (int it = 0; it < grid->refine_iters; ++it) omse::tensor_pass_kernel<1><<<(unsigned)pass_grid, 256, 0, s>>>(a);
-    omse::tensor_pass_kernel<2><<<(unsigned)pass_grid, 256, 0, s>>>(a);
+    // the sweep stays below 48 KB of dynamic shared memory, so no attribute call is needed here
+    const TensorEnv env = {sd.n_sm, s, sd.occ_sweep, sd.occ_pass, false, sd.attr_unused};
+    const int rc = enqueue_tensor_search(env, a, grid->refine_iters);
+    if (rc != OMSE_OK) return rc;
     static_end_kernel<<<1, 32, 0, s>>>(sc, d_status);
     return cudaGetLastError() == cudaSuccess ? OMSE_OK : OMSE_ECUDA;
 }

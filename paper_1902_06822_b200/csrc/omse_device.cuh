@@ -315,13 +315,13 @@ __device__ __forceinline__ void block_argmin(double& v, int& idx, double* scratc
     idx = bi;
 }
 
-// Number of leading candidate slots (slot sl holds scales >= (sl*tg+1)*step) that must still evaluate x:
-// the others code it as 0.  inv_thr = 1/(0.4999*step), inv_tg = 1/tg.
+// Number of leading candidate slots that must still evaluate x, for a thread group whose slot sl holds the scales
+// >= (c_base + sl*tg + 1)*step: the others code it as 0.  inv_thr = 1/(0.4999*step), inv_tg = 1/tg.
 template <int CPT>
-__device__ __forceinline__ int magnitude_class(float x, float inv_thr, float inv_tg) {
+__device__ __forceinline__ int magnitude_class(float x, float inv_thr, float inv_tg, float c_base = 0.f) {
     const float ax = fabsf(x);
     if (!(ax <= FLT_MAX)) return CPT;          // non-finite: every slot sees it (and reports it)
-    const float r = ax * inv_thr;              // |x| / (0.4999*step)
+    const float r = ax * inv_thr - c_base;     // |x| / (0.4999*step), counted from the group's first candidate
     if (r <= 1.0f) return 0;
     const float f = (r - 1.0f) * inv_tg;       // slot sl needs x iff r > sl*tg + 1
     int nb = f >= (float)CPT ? CPT : (int)f + 1;
@@ -330,12 +330,13 @@ __device__ __forceinline__ int magnitude_class(float x, float inv_thr, float inv
 }
 
 // Candidates with index below the returned value may saturate on an element of magnitude class nb
-// (nb < CPT bounds |x| from above: |x| < 0.4999*(nb*tg+1)*step, and candidate c saturates only if
+// (nb < CPT bounds |x| from above: |x| < 0.4999*(c_base + nb*tg + 1)*step, and candidate c saturates only if
 // |x| >= min(hi+1/2, 1/2-lo)*alpha_c); class CPT has no upper bound and keeps the row's own count.
-__device__ __forceinline__ int class_sat_count(int nb, int cpt, int tg, int c_sat_row, float flo, float fhi) {
+__device__ __forceinline__ int class_sat_count(int nb, int cpt, int tg, int c_sat_row, float flo, float fhi,
+                                               int c_base = 0) {
     if (nb >= cpt) return c_sat_row;
     const float den = fminf(fhi + 0.5f, 0.5f - flo);
-    const int c = (int)(0.5f * (float)(nb * tg + 1) / den) + 2;
+    const int c = (int)(0.5f * (float)(c_base + nb * tg + 1) / den) + 2;
     return min(c, c_sat_row);
 }
 

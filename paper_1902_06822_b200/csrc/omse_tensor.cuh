@@ -29,7 +29,8 @@ struct TensorArgs {
     int n_cand;
     float hi_frac;
     int lo, hi;
-    int tg, groups;         // sweep block = groups*tg threads; candidate c = slot*tg + t
+    int tg, groups;         // sweep block = groups*tg threads; candidate c = c_base + slot*tg + t
+    int c_base, c_count;    // candidates [c_base, c_base + c_count) are swept by this launch
     int tile4;              // float4s per tile
     TensorState* st;
     double* partials;       // sweep: [grid][n_cand]; passes: [blocks][listed candidates] doubles + [blocks] int64
@@ -130,11 +131,14 @@ __global__ void __launch_bounds__(256) tensor_absmax_kernel(const float* __restr
     if (bad) atomicOr(status, 1u);
 }
 
-// Candidate sweep over tiles of the tensor; block b handles tiles b, b+grid, ...
-// While a tile is staged its elements are regrouped by magnitude class (see magnitude_class): class nb
-// is evaluated by candidate slots 0..nb-1 only, class 0 (|x| <= 0.4999*step, in particular the exact
-// zeros of a post-ReLU tensor) by none; every slot adds the squared sum of the classes it skipped.
-// The regrouping is a deterministic block-wide counting sort, so results do not depend on scheduling.
+// Candidate sweep over tiles of the tensor; block b handles tiles b, b+grid, ...; one launch covers the candidates
+// [c_base, c_base + c_count).  While a tile is staged its elements are regrouped by magnitude class (see
+// magnitude_class): class nb is evaluated by candidate slots 0..nb-1 only, class 0 (|x| <= 0.4999*alpha of the
+// launch's first candidate; in particular the exact zeros of a post-ReLU tensor) by none; every slot adds the
+// squared sum of the classes it skipped.  The regrouping is a deterministic block-wide counting sort, so results do
+// not depend on scheduling.  The host covers the grid with two launches when it has more than 256 candidates: the
+// first 256 with 32 candidates per slot (most elements of a heavy-tailed tensor are small against max|x| and
+// matter only to the smallest scales, so the fine classes there prune the most), the rest with wider slots.
 template <int CPT>
 __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -152,38 +156,36 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
     if (!(m > 0.f) || !(a_last >= FLT_MIN)) return;   // degenerate tensor: finish kernel reports it
     const float inv_thr = g.rstep * (1.0f / 0.4999f);
     const float inv_tg = 1.0f / (float)a.tg;
+    const float cbase_f = (float)a.c_base;
     const float delta = a.st->delta;                  // 0 unless the offset scheme is used
 
     u64 inv2[CPT], na2[CPT];
     double dacc[CPT];
 #pragma unroll
     for (int sl = 0; sl < CPT; ++sl) {
-        const int c = sl * a.tg + t;
+        const int cl = sl * a.tg + t, c = a.c_base + cl;
         const float ac = __fmul_rn((float)(c + 1), g.step);
         float inv = g.tiny ? __fdiv_rn(1.0f, ac) : __fdiv_rn(1.0f, (float)(c + 1)) * g.rstep;
-        if (!(ac >= FLT_MIN) || c >= a.n_cand) inv = 0.f;
+        if (!(ac >= FLT_MIN) || cl >= a.c_count) inv = 0.f;
         inv2[sl] = pack2(inv, inv);
         na2[sl] = pack2(-ac, -ac);
         dacc[sl] = 0.0;
     }
     const int warp_t0 = t & ~31;
-    int ncl = (g.c_sat - warp_t0 + a.tg - 1) / a.tg;
-    ncl = max(0, min(CPT, ncl));
 
     const long long n4_total = (a.n + 3) >> 2;
     const long long n_tiles = (n4_total + a.tile4 - 1) / a.tile4;
     const float4* x4 = reinterpret_cast<const float4*>(a.x);
     const int per_thread4 = a.tile4 / nthr;          // consecutive float4s staged by one thread (<= 4)
     unsigned long long ev = 0ull;                    // evaluations this thread executed
-    double skipped[CPT + 1];                         // squared sums per class over this block's tiles
+    double sq[CPT + 1];                              // squared sums per class over this block's tiles (this thread's share)
 #pragma unroll
-    for (int b = 0; b <= CPT; ++b) skipped[b] = 0.0;
+    for (int b = 0; b <= CPT; ++b) sq[b] = 0.0;
     for (long long tl = blockIdx.x; tl < n_tiles; tl += gridDim.x) {
         const long long base4 = tl * a.tile4;
         const int cnt4 = (int)min((long long)a.tile4, n4_total - base4);
         // ---- load this thread's span, classify, count
-        float vals[16];
-        u64 cls = 0ull, c0 = 0ull, c1 = 0ull;        // 4-bit class per value; counts in 16-bit fields
+        float4 v4[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -192,31 +194,40 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
                 const long long e = (base4 + i) << 2;
                 if (e + 3 < a.n) {
                     v = __ldg(x4 + base4 + i);
-                    v.x -= delta;
-                    v.y -= delta;
-                    v.z -= delta;
-                    v.w -= delta;
                 } else {   // ragged end of the tensor: missing elements count as zeros
-                    v.x = e < a.n ? a.x[e] - delta : 0.f;
-                    v.y = e + 1 < a.n ? a.x[e + 1] - delta : 0.f;
-                    v.z = e + 2 < a.n ? a.x[e + 2] - delta : 0.f;
+                    v.x = e < a.n ? a.x[e] : delta;
+                    v.y = e + 1 < a.n ? a.x[e + 1] : delta;
+                    v.z = e + 2 < a.n ? a.x[e + 2] : delta;
+                    v.w = delta;
                 }
+            } else {
+                v = make_float4(delta, delta, delta, delta);
             }
-            const float e4[4] = {v.x, v.y, v.z, v.w};
+            v4[j] = v;
+        }
+        float vals[16];
+        u64 cls = 0ull, c0 = 0ull, c1 = 0ull;        // 4-bit class per value; counts in 16-bit fields
+        double zero_sq = 0.0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float e4[4] = {v4[j].x - delta, v4[j].y - delta, v4[j].z - delta, v4[j].w - delta};
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 const float x = e4[q];
-                int nb = magnitude_class<CPT>(x, inv_thr, inv_tg);
+                int nb = magnitude_class<CPT>(x, inv_thr, inv_tg, cbase_f);
                 if (g.tiny && x != 0.f) nb = CPT;
                 vals[4 * j + q] = x;
                 cls |= (u64)nb << (4 * (4 * j + q));
-                const double xx = (double)x * (double)x;
-#pragma unroll
-                for (int b = 0; b <= CPT; ++b) skipped[b] += (nb == b) ? xx : 0.0;
+                const double xd = (double)x;
+                zero_sq = fma(nb == 0 ? xd : 0.0, xd, zero_sq);
                 if (nb >= 5) c1 += 1ull << (16 * (nb - 5));
                 else if (nb >= 1) c0 += 1ull << (16 * (nb - 1));
             }
         }
+        sq[0] += zero_sq;
+        // previous tile fully swept (tile and warp_tot free); a tile none of whose elements reaches this launch's
+        // first candidate needs nothing more
+        if (!__syncthreads_or((c0 | c1) != 0ull)) continue;
         // ---- exclusive scan of the class counts over the block (lanes by shuffle, warps in order)
         u64 i0 = c0, i1 = c1;
 #pragma unroll
@@ -228,7 +239,6 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
                 i1 += u1;
             }
         }
-        __syncthreads();   // previous tile fully swept; warp_tot free
         if (lane == 31) {
             warp_tot[warp][0] = i0;
             warp_tot[warp][1] = i1;
@@ -245,15 +255,14 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
             tot1 += a1;
         }
         // ---- class layout in the tile buffer: class CPT first, each padded with zeros to a multiple of 4
-        int base[CPT + 1], len4[CPT + 1];
+        int base[CPT + 1], cnt[CPT + 1];
         int pos = 0;
 #pragma unroll
         for (int b = CPT; b >= 1; --b) {
-            const int cnt = (int)(((b >= 5 ? tot1 : tot0) >> (16 * ((b - 1) & 3))) & 0xffffull);
+            cnt[b] = (int)(((b >= 5 ? tot1 : tot0) >> (16 * ((b - 1) & 3))) & 0xffffull);
             base[b] = pos;
-            const int padded = (cnt + 3) & ~3;
-            len4[b] = padded >> 2;
-            if (tid < padded - cnt) tile[pos + cnt + tid] = 0.f;
+            const int padded = (cnt[b] + 3) & ~3;
+            if (tid < padded - cnt[b]) tile[pos + cnt[b] + tid] = 0.f;
             pos += padded;
         }
 #pragma unroll
@@ -279,10 +288,16 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
         const float4* tile4p = reinterpret_cast<const float4*>(tile);
 #pragma unroll
         for (int b = CPT; b >= 1; --b) {
-            const int first4 = base[b] >> 2;
-            const int beg4 = first4 + (int)(((long long)len4[b] * grp) / a.groups);
-            const int end4 = first4 + (int)(((long long)len4[b] * (grp + 1)) / a.groups);
-            int ncl_b = (class_sat_count(b, CPT, a.tg, g.c_sat, flo, fhi) - warp_t0 + a.tg - 1) / a.tg;
+            if (cnt[b] == 0) continue;
+            // squared sum of the class (what the slots that skip it add), from the regrouped tile
+            for (int i = tid; i < cnt[b]; i += nthr) {
+                const double xd = (double)tile[base[b] + i];
+                sq[b] = fma(xd, xd, sq[b]);
+            }
+            const int first4 = base[b] >> 2, len4 = (cnt[b] + 3) >> 2;
+            const int beg4 = first4 + (int)(((long long)len4 * grp) / a.groups);
+            const int end4 = first4 + (int)(((long long)len4 * (grp + 1)) / a.groups);
+            int ncl_b = (class_sat_count(b, CPT, a.tg, g.c_sat, flo, fhi, a.c_base) - (a.c_base + warp_t0) + a.tg - 1) / a.tg;
             ncl_b = max(0, min(CPT, ncl_b));
             sweep_dispatch<CPT>(b, ncl_b, tile4p, beg4, end4, inv2, na2, dacc, kMagic + flo, kMagic + fhi);
             ev += (unsigned long long)(end4 - beg4) * 4ull * (unsigned long long)b;
@@ -307,7 +322,7 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
     double run = 0.0;
 #pragma unroll
     for (int b = 0; b < CPT; ++b) {
-        double v = skipped[b];
+        double v = sq[b];
         block_sum2(v, zero, dscratch);
         run += v;
         dacc[b] += run;          // slot b skips classes 0..b
@@ -315,30 +330,44 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
     if (grp == 0) {
 #pragma unroll
         for (int sl = 0; sl < CPT; ++sl) {
-            const int c = sl * a.tg + t;
-            if (c < a.n_cand) a.partials[(long long)blockIdx.x * a.n_cand + c] = dacc[sl];
+            const int cl = sl * a.tg + t;
+            if (cl < a.c_count) a.partials[(long long)blockIdx.x * a.n_cand + a.c_base + cl] = dacc[sl];
         }
     }
 }
 
-// Sums the per-block partial curves in block order: one thread per candidate, several blocks.
-__global__ void __launch_bounds__(64) tensor_curve_kernel(const TensorArgs a, int n_blocks) {
-    const int c = blockIdx.x * blockDim.x + threadIdx.x;
-    if (c >= a.n_cand) return;
+// Sums the per-block partial curves in block order.  Candidates below `split` were swept by a launch of n_blocks_lo
+// blocks, the others by one of n_blocks_hi blocks.  A block of 256 threads handles 32 candidates: thread (j, c) adds
+// the partials of blocks j, j+8, ... and the eight sums are combined in order.
+__global__ void __launch_bounds__(256) tensor_curve_kernel(const TensorArgs a, int split, int n_blocks_lo, int n_blocks_hi) {
+    __shared__ double part[8][33];
+    const int cl = threadIdx.x & 31, j = threadIdx.x >> 5;
+    const int c = blockIdx.x * 32 + cl;
     TensorState* st = a.st;
     const float mpos = __uint_as_float(st->mpos_bits), mneg = __uint_as_float(st->mneg_bits);
     const GridSetup g = grid_setup(mpos, mneg, a.hi_frac, a.n_cand, (float)a.lo, (float)a.hi);
     const float a_last = __fmul_rn((float)a.n_cand, g.step);
-    double s = INFINITY;
-    if ((fmaxf(mpos, mneg) > 0.f) && (a_last >= FLT_MIN)) {
-        s = 0.0;
-#pragma unroll 8
-        for (int b = 0; b < n_blocks; ++b) s += __ldcg(&a.partials[(long long)b * a.n_cand + c]);
-        const float ac = __fmul_rn((float)(c + 1), g.step);
-        if (!(ac >= FLT_MIN)) s = INFINITY;
+    const bool usable = (fmaxf(mpos, mneg) > 0.f) && (a_last >= FLT_MIN);
+    double s = 0.0;
+    if (usable && c < a.n_cand) {
+        const int n_blocks = c < split ? n_blocks_lo : n_blocks_hi;
+#pragma unroll 4
+        for (int b = j; b < n_blocks; b += 8) s += __ldcg(&a.partials[(long long)b * a.n_cand + c]);
     }
-    a.curve[c] = s;
-    if (a.curve_out) a.curve_out[c] = s;
+    part[j][cl] = s;
+    __syncthreads();
+    if (j == 0 && c < a.n_cand) {
+        double tot = INFINITY;
+        if (usable) {
+            tot = 0.0;
+#pragma unroll
+            for (int jj = 0; jj < 8; ++jj) tot += part[jj][cl];
+            const float ac = __fmul_rn((float)(c + 1), g.step);
+            if (!(ac >= FLT_MIN)) tot = INFINITY;
+        }
+        a.curve[c] = tot;
+        if (a.curve_out) a.curve_out[c] = tot;
+    }
 }
 
 // One block: argmin of the summed curve and the list of candidates inside the fp32 noise band of the minimum.
@@ -471,15 +500,24 @@ __global__ void __launch_bounds__(256) tensor_pass_kernel(const TensorArgs a) {
                 }
             }
         };
-#pragma unroll 4
-        for (long long i = tid0; i < n4; i += stride) {   // several 128-bit loads in flight per thread
-            const float4 v = __ldg(x4 + i);
+        auto four = [&](const float4& v) {
             element(v.x - delta);
             element(v.y - delta);
             element(v.z - delta);
             element(v.w - delta);
+        };
+        // four 128-bit loads in flight per thread before any of them is used
+        long long i = tid0;
+        for (; i + 3 * stride < n4; i += 4 * stride) {
+            const float4 v0 = __ldg(x4 + i), v1 = __ldg(x4 + i + stride), v2 = __ldg(x4 + i + 2 * stride),
+                         v3 = __ldg(x4 + i + 3 * stride);
+            four(v0);
+            four(v1);
+            four(v2);
+            four(v3);
         }
-        for (long long i = (n4 << 2) + tid0; i < a.n; i += stride) element(a.x[i] - delta);
+        for (; i < n4; i += stride) four(__ldg(x4 + i));
+        for (long long e = (n4 << 2) + tid0; e < a.n; e += stride) element(a.x[e] - delta);
         for (int j = 0; j < nj; ++j) {
             long long q = sqq;
             block_sum2(acc[j], q, scratch);
@@ -489,7 +527,8 @@ __global__ void __launch_bounds__(256) tensor_pass_kernel(const TensorArgs a) {
             }
         }
     }
-    // ---- last block to arrive reduces the per-block partials in block order
+    // ---- last block to arrive reduces the per-block partials (fixed order: thread t takes blocks t, t+256, ...,
+    //      then the block-wide sum in lane and warp order)
     __threadfence();
     if (threadIdx.x == 0) {
         const unsigned int tk = atomicAdd(&st->ticket, 1u);
@@ -500,7 +539,7 @@ __global__ void __launch_bounds__(256) tensor_pass_kernel(const TensorArgs a) {
     __threadfence();
     double best_sse = INFINITY;     // MODE 0: this thread's best listed candidate
     int best = 0x7fffffff;
-    double total = 0.0;             // MODE 1, 2: thread 0 sums the single column
+    double total = 0.0;             // MODE 1, 2
     long long total_q = 0;
     if (MODE == 0) {
         for (int l = threadIdx.x; l < n_list; l += blockDim.x) {
@@ -513,10 +552,12 @@ __global__ void __launch_bounds__(256) tensor_pass_kernel(const TensorArgs a) {
             }
         }
         block_argmin(best_sse, best, scratch);
-    } else if (threadIdx.x == 0) {
-        for (unsigned int b = 0; b < nblk; ++b) total += __ldcg(&part_d[b]);
-        if (MODE == 1)
-            for (unsigned int b = 0; b < nblk; ++b) total_q += __ldcg(&part_q[b]);
+    } else {
+        for (unsigned int b = threadIdx.x; b < nblk; b += blockDim.x) {
+            total += __ldcg(&part_d[b]);
+            if (MODE == 1) total_q += __ldcg(&part_q[b]);
+        }
+        block_sum2(total, total_q, scratch);
     }
     if (threadIdx.x == 0) {
         st->ticket = 0u;

@@ -233,18 +233,16 @@ struct TensorEnv {
     bool* attr_tensor;   // [4] per CPT: opt-in attribute already set
 };
 
-template <int CPT>
-int sweep_launch_t(const TensorEnv& env, omse::TensorArgs& a, size_t smem, int occ_slot, int* n_blocks) {
+template <int CPT, bool FINE>
+int sweep_launch_t(const TensorEnv& env, omse::TensorArgs& a, size_t smem, int* n_blocks) {
+    auto kernel = FINE ? omse::tensor_sweep_fine_kernel<CPT> : omse::tensor_sweep_kernel<CPT>;
     if (env.opt_in_smem && smem > 48 * 1024 && !env.attr_tensor[cpt_slot(CPT)]) {
-        if (cudaFuncSetAttribute(omse::tensor_sweep_kernel<CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess)
-            return OMSE_ECUDA;
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess) return OMSE_ECUDA;
         env.attr_tensor[cpt_slot(CPT)] = true;
     }
     const int threads = a.groups * a.tg;
     int occ = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, omse::tensor_sweep_kernel<CPT>, threads, smem) != cudaSuccess || occ < 1)
-        return OMSE_ECUDA;
-    (void)occ_slot;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, threads, smem) != cudaSuccess || occ < 1) return OMSE_ECUDA;
     const long long n4 = (a.n + 3) >> 2;
     const long long n_tiles = (n4 + a.tile4 - 1) / a.tile4;
     long long grid = (long long)env.n_sm * occ;
@@ -253,25 +251,34 @@ int sweep_launch_t(const TensorEnv& env, omse::TensorArgs& a, size_t smem, int o
     if (grid > n_tiles) grid = n_tiles;
     if (grid < 1) grid = 1;
     *n_blocks = (int)grid;
-    omse::tensor_sweep_kernel<CPT><<<(unsigned)grid, threads, smem, env.stream>>>(a);
+    kernel<<<(unsigned)grid, threads, smem, env.stream>>>(a);
     return cudaGetLastError() == cudaSuccess ? OMSE_OK : OMSE_ECUDA;
 }
 
 // One sweep launch over the candidates [c_base, c_base + c_count) with `cpt` candidates per thread.
-int sweep_launch(const TensorEnv& env, omse::TensorArgs a, int c_base, int c_count, int cpt, int occ_slot, int* n_blocks) {
+int sweep_launch(const TensorEnv& env, omse::TensorArgs a, int c_base, int c_count, int cpt, int* n_blocks) {
     a.c_base = c_base;
     a.c_count = c_count;
     a.tg = (((c_count + cpt - 1) / cpt) + 31) & ~31;
     a.groups = 256 / a.tg < 1 ? 1 : 256 / a.tg;
     a.tile4 = 4 * a.groups * a.tg;   // every thread stages exactly four float4s of a tile
-    const size_t smem = (size_t)a.tile4 * 16 + (size_t)cpt * 16 + (size_t)(a.groups - 1) * cpt * a.tg * 8;
-    if (!env.opt_in_smem && smem > 48 * 1024) return OMSE_ELIMIT;
-    switch (cpt) {
-        case 1: return sweep_launch_t<1>(env, a, smem, occ_slot, n_blocks);
-        case 2: return sweep_launch_t<2>(env, a, smem, occ_slot, n_blocks);
-        case 4: return sweep_launch_t<4>(env, a, smem, occ_slot, n_blocks);
-        default: return sweep_launch_t<8>(env, a, smem, occ_slot, n_blocks);
+    if (a.tg == 32) {
+        // slots of 32 candidates: the warps of a block work on their own shares of a tile
+        const size_t smem = (size_t)8 * (16 * 32 + 8) * 4 + (size_t)a.tile4 * 16;   // eight warp regions + landing zone
+        switch (cpt) {
+            case 1: return sweep_launch_t<1, true>(env, a, smem, n_blocks);
+            case 2: return sweep_launch_t<2, true>(env, a, smem, n_blocks);
+            case 4: return sweep_launch_t<4, true>(env, a, smem, n_blocks);
+            default: return sweep_launch_t<8, true>(env, a, smem, n_blocks);
+        }
     }
+    // regrouped tile + landing zone of the asynchronous copies, which also holds the partial sums of the other groups
+    // at the end
+    const size_t regrouped = ((size_t)a.tile4 * 4 + 4 * cpt) * 4;
+    const size_t landing = std::max((size_t)a.tile4 * 16, (size_t)(a.groups - 1) * cpt * a.tg * 8);
+    const size_t smem = regrouped + landing;
+    if (!env.opt_in_smem && smem + 1024 > 48 * 1024) return OMSE_ELIMIT;
+    return sweep_launch_t<8, false>(env, a, smem, n_blocks);   // wide slots only occur with 8 candidates per thread
 }
 
 template <int MODE>
@@ -299,12 +306,12 @@ int enqueue_tensor_search(const TensorEnv& env, omse::TensorArgs& a, int refine_
         if (a.delta_out) omse::tensor_offset_kernel<<<1, 32, 0, s>>>(a.st);
         int rc;
         if (a.n_cand <= kFine) {
-            rc = sweep_launch(env, a, 0, a.n_cand, cpt_for(a.n_cand), 0, &nb_lo);
+            rc = sweep_launch(env, a, 0, a.n_cand, cpt_for(a.n_cand), &nb_lo);
             nb_hi = nb_lo;
         } else {
             split = kFine;
-            rc = sweep_launch(env, a, 0, kFine, 8, 0, &nb_lo);
-            if (rc == OMSE_OK) rc = sweep_launch(env, a, kFine, a.n_cand - kFine, 8, 1, &nb_hi);
+            rc = sweep_launch(env, a, 0, kFine, 8, &nb_lo);
+            if (rc == OMSE_OK) rc = sweep_launch(env, a, kFine, a.n_cand - kFine, 8, &nb_hi);
         }
         if (rc != OMSE_OK) return rc;
     }

@@ -144,9 +144,14 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ u64 warp_tot[16][2];
     __shared__ double dscratch[64];
-    float* tile = reinterpret_cast<float*>(smem_raw);                      // [4*tile4 + 4*CPT]
-    double* xg = reinterpret_cast<double*>(tile + 4 * a.tile4 + 4 * CPT);
     const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
+    // A group of 32 threads is one warp: it then regroups and sweeps its own share of every tile by itself (no block
+    // barrier inside the tile loop).  Wider groups share the whole tile and regroup it together.
+    const bool solo = false;   // launches with 32-candidate slots use tensor_sweep_fine_kernel
+    const int region = solo ? 4 * (a.tile4 / nwarp) + 4 * CPT : 4 * a.tile4 + 4 * CPT;   // floats of a regrouped tile (share)
+    float* tile = reinterpret_cast<float*>(smem_raw) + (solo ? warp * region : 0);
+    float4* raw4 = reinterpret_cast<float4*>(reinterpret_cast<float*>(smem_raw) + (solo ? nwarp * region : region));   // [tile4] landing zone of the asynchronous copies
+    double* xg = reinterpret_cast<double*>(raw4);    // partial sums of the other groups (after the last tile)
     const int grp = tid / a.tg, t = tid - grp * a.tg;
     const float mpos = __uint_as_float(a.st->mpos_bits), mneg = __uint_as_float(a.st->mneg_bits);
     const float m = fmaxf(mpos, mneg);
@@ -174,6 +179,7 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
     const int warp_t0 = t & ~31;
 
     const long long n4_total = (a.n + 3) >> 2;
+    const long long n4_full = a.n >> 2;               // float4s that lie completely inside the tensor
     const long long n_tiles = (n4_total + a.tile4 - 1) / a.tile4;
     const float4* x4 = reinterpret_cast<const float4*>(a.x);
     const int per_thread4 = a.tile4 / nthr;          // consecutive float4s staged by one thread (<= 4)
@@ -181,54 +187,83 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
     double sq[CPT + 1];                              // squared sums per class over this block's tiles (this thread's share)
 #pragma unroll
     for (int b = 0; b <= CPT; ++b) sq[b] = 0.0;
-    for (long long tl = blockIdx.x; tl < n_tiles; tl += gridDim.x) {
+
+    // Asynchronous copy of this thread's float4s of tile tl into their landing slots; a thread only ever reads the
+    // slots it filled itself, so the copies need no barrier, and they run while the previous tile is processed.
+    auto prefetch = [&](long long tl) {
         const long long base4 = tl * a.tile4;
-        const int cnt4 = (int)min((long long)a.tile4, n4_total - base4);
-        // ---- load this thread's span, classify, count
-        float4 v4[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
             const int i = tid * per_thread4 + j;
-            if (j < per_thread4 && i < cnt4) {
-                const long long e = (base4 + i) << 2;
-                if (e + 3 < a.n) {
-                    v = __ldg(x4 + base4 + i);
-                } else {   // ragged end of the tensor: missing elements count as zeros
-                    v.x = e < a.n ? a.x[e] : delta;
-                    v.y = e + 1 < a.n ? a.x[e + 1] : delta;
-                    v.z = e + 2 < a.n ? a.x[e + 2] : delta;
-                    v.w = delta;
-                }
-            } else {
-                v = make_float4(delta, delta, delta, delta);
+            if (j < per_thread4 && base4 + i < n4_full) {
+                const unsigned int dst = (unsigned int)__cvta_generic_to_shared(raw4 + i);
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(x4 + base4 + i) : "memory");
             }
-            v4[j] = v;
         }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    long long tl = blockIdx.x;
+    if (tl < n_tiles) prefetch(tl);
+    for (; tl < n_tiles; tl += gridDim.x) {
+        const long long base4 = tl * a.tile4;
+        asm volatile("cp.async.wait_all;" ::: "memory");
+        // ---- this thread's span into registers (elements past the end count as zeros)
         float vals[16];
+        bool big = false;                            // some value reaches this launch's first candidate
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            float4 v = make_float4(delta, delta, delta, delta);
+            const int i = tid * per_thread4 + j;
+            if (j < per_thread4) {
+                if (base4 + i < n4_full) {
+                    v = raw4[i];
+                } else {
+                    const long long e = (base4 + i) << 2;
+                    if (e < a.n) v.x = a.x[e];
+                    if (e + 1 < a.n) v.y = a.x[e + 1];
+                    if (e + 2 < a.n) v.z = a.x[e + 2];
+                }
+            }
+            vals[4 * j] = v.x - delta;
+            vals[4 * j + 1] = v.y - delta;
+            vals[4 * j + 2] = v.z - delta;
+            vals[4 * j + 3] = v.w - delta;
+        }
+        if (tl + gridDim.x < n_tiles) prefetch(tl + gridDim.x);   // the slots are free again: next tile on its way
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+            const float x = vals[e];
+            big |= !(fabsf(x) * inv_thr - cbase_f <= 1.0f) || (g.tiny && x != 0.f);
+        }
+        // previous tile fully swept (tile and warp_tot free).  If nothing of this tile (share) reaches the first
+        // candidate, every slot skips all of it.
+        const bool any = solo ? __any_sync(0xffffffffu, big) : (__syncthreads_or(big) != 0);
+        if (!any) {
+            double z = 0.0;
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+                const double xd = (double)vals[e];
+                z = fma(xd, xd, z);
+            }
+            sq[0] += z;
+            continue;
+        }
+        // ---- classify, count
         u64 cls = 0ull, c0 = 0ull, c1 = 0ull;        // 4-bit class per value; counts in 16-bit fields
         double zero_sq = 0.0;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const float e4[4] = {v4[j].x - delta, v4[j].y - delta, v4[j].z - delta, v4[j].w - delta};
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const float x = e4[q];
-                int nb = magnitude_class<CPT>(x, inv_thr, inv_tg, cbase_f);
-                if (g.tiny && x != 0.f) nb = CPT;
-                vals[4 * j + q] = x;
-                cls |= (u64)nb << (4 * (4 * j + q));
-                const double xd = (double)x;
-                zero_sq = fma(nb == 0 ? xd : 0.0, xd, zero_sq);
-                if (nb >= 5) c1 += 1ull << (16 * (nb - 5));
-                else if (nb >= 1) c0 += 1ull << (16 * (nb - 1));
-            }
+        for (int e = 0; e < 16; ++e) {
+            const float x = vals[e];
+            int nb = magnitude_class<CPT>(x, inv_thr, inv_tg, cbase_f);
+            if (g.tiny && x != 0.f) nb = CPT;
+            cls |= (u64)nb << (4 * e);
+            const double xd = (double)x;
+            zero_sq = fma(nb == 0 ? xd : 0.0, xd, zero_sq);
+            if (nb >= 5) c1 += 1ull << (16 * (nb - 5));
+            else if (nb >= 1) c0 += 1ull << (16 * (nb - 1));
         }
         sq[0] += zero_sq;
-        // previous tile fully swept (tile and warp_tot free); a tile none of whose elements reaches this launch's
-        // first candidate needs nothing more
-        if (!__syncthreads_or((c0 | c1) != 0ull)) continue;
-        // ---- exclusive scan of the class counts over the block (lanes by shuffle, warps in order)
+        // ---- exclusive scan of the class counts (lanes by shuffle; warps in order when the block shares the tile)
         u64 i0 = c0, i1 = c1;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -239,22 +274,30 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
                 i1 += u1;
             }
         }
-        if (lane == 31) {
-            warp_tot[warp][0] = i0;
-            warp_tot[warp][1] = i1;
-        }
-        __syncthreads();
-        u64 off0 = i0 - c0, off1 = i1 - c1, tot0 = 0ull, tot1 = 0ull;
-        for (int w = 0; w < nwarp; ++w) {
-            const u64 a0 = warp_tot[w][0], a1 = warp_tot[w][1];
-            if (w < warp) {
-                off0 += a0;
-                off1 += a1;
+        u64 off0 = i0 - c0, off1 = i1 - c1, tot0, tot1;
+        if (solo) {
+            tot0 = __shfl_sync(0xffffffffu, i0, 31);
+            tot1 = __shfl_sync(0xffffffffu, i1, 31);
+        } else {
+            if (lane == 31) {
+                warp_tot[warp][0] = i0;
+                warp_tot[warp][1] = i1;
             }
-            tot0 += a0;
-            tot1 += a1;
+            __syncthreads();
+            tot0 = 0ull;
+            tot1 = 0ull;
+            for (int w = 0; w < nwarp; ++w) {
+                const u64 a0 = warp_tot[w][0], a1 = warp_tot[w][1];
+                if (w < warp) {
+                    off0 += a0;
+                    off1 += a1;
+                }
+                tot0 += a0;
+                tot1 += a1;
+            }
         }
         // ---- class layout in the tile buffer: class CPT first, each padded with zeros to a multiple of 4
+        const int who = solo ? lane : tid;
         int base[CPT + 1], cnt[CPT + 1];
         int pos = 0;
 #pragma unroll
@@ -262,7 +305,7 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
             cnt[b] = (int)(((b >= 5 ? tot1 : tot0) >> (16 * ((b - 1) & 3))) & 0xffffull);
             base[b] = pos;
             const int padded = (cnt[b] + 3) & ~3;
-            if (tid < padded - cnt[b]) tile[pos + cnt[b] + tid] = 0.f;
+            if (who < padded - cnt[b]) tile[pos + cnt[b] + who] = 0.f;
             pos += padded;
         }
 #pragma unroll
@@ -284,25 +327,28 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
                 tile[bs + within] = vals[e];
             }
         }
-        __syncthreads();
+        if (solo) __syncwarp();
+        else __syncthreads();
         const float4* tile4p = reinterpret_cast<const float4*>(tile);
-#pragma unroll
+        const int n_share = solo ? 32 : nthr;
+#pragma unroll 1
         for (int b = CPT; b >= 1; --b) {
             if (cnt[b] == 0) continue;
             // squared sum of the class (what the slots that skip it add), from the regrouped tile
-            for (int i = tid; i < cnt[b]; i += nthr) {
+            for (int i = who; i < cnt[b]; i += n_share) {
                 const double xd = (double)tile[base[b] + i];
                 sq[b] = fma(xd, xd, sq[b]);
             }
             const int first4 = base[b] >> 2, len4 = (cnt[b] + 3) >> 2;
-            const int beg4 = first4 + (int)(((long long)len4 * grp) / a.groups);
-            const int end4 = first4 + (int)(((long long)len4 * (grp + 1)) / a.groups);
+            const int beg4 = solo ? first4 : first4 + (int)(((long long)len4 * grp) / a.groups);
+            const int end4 = solo ? first4 + len4 : first4 + (int)(((long long)len4 * (grp + 1)) / a.groups);
             int ncl_b = (class_sat_count(b, CPT, a.tg, g.c_sat, flo, fhi, a.c_base) - (a.c_base + warp_t0) + a.tg - 1) / a.tg;
             ncl_b = max(0, min(CPT, ncl_b));
             sweep_dispatch<CPT>(b, ncl_b, tile4p, beg4, end4, inv2, na2, dacc, kMagic + flo, kMagic + fhi);
             ev += (unsigned long long)(end4 - beg4) * 4ull * (unsigned long long)b;
         }
     }
+    asm volatile("cp.async.wait_all;" ::: "memory");
     if (a.groups > 1) {
         __syncthreads();
         if (grp > 0) {
@@ -332,6 +378,166 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
         for (int sl = 0; sl < CPT; ++sl) {
             const int cl = sl * a.tg + t;
             if (cl < a.c_count) a.partials[(long long)blockIdx.x * a.n_cand + a.c_base + cl] = dacc[sl];
+        }
+    }
+}
+
+// The same sweep for launches whose slots hold 32 candidates (a warp is an element group of its own): every warp
+// keeps its own share of a tile (the float4s its lanes copied) and never waits for the block.  The elements are
+// split three ways with ballots, in a fixed order: dropped (coded 0 by every candidate of the launch), "first slot
+// only" (by far the most for a tensor with many small values) and the rest, which all slots evaluate; the two lists
+// grow from the two ends of the warp's region.  Slot 0 adds the squared sum of the dropped elements, the other slots
+// that of the dropped and of the first-slot-only elements.
+template <int CPT>
+__global__ void __launch_bounds__(256) tensor_sweep_fine_kernel(const TensorArgs a) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ double dscratch[64];
+    const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
+    const int share = 16 * 32;                       // elements of a tile that one warp stages
+    const int region = share + 8;                    // + zero padding of the two lists
+    float* reg = reinterpret_cast<float*>(smem_raw) + warp * region;
+    float4* raw4 = reinterpret_cast<float4*>(reinterpret_cast<float*>(smem_raw) + nwarp * region);   // [tile4] landing zone
+    double* xg = reinterpret_cast<double*>(raw4);    // partial sums of the other warps (after the last tile)
+    const float mpos = __uint_as_float(a.st->mpos_bits), mneg = __uint_as_float(a.st->mneg_bits);
+    const float m = fmaxf(mpos, mneg);
+    const float flo = (float)a.lo, fhi = (float)a.hi;
+    const GridSetup g = grid_setup(mpos, mneg, a.hi_frac, a.n_cand, flo, fhi);
+    const float a_last = __fmul_rn((float)a.n_cand, g.step);
+    if (!(m > 0.f) || !(a_last >= FLT_MIN)) return;   // degenerate tensor: finish kernel reports it
+    const float inv_thr = g.rstep * (1.0f / 0.4999f);
+    const float cbase_f = (float)a.c_base;
+    const float delta = a.st->delta;
+
+    u64 inv2[CPT], na2[CPT];
+    double dacc[CPT];
+#pragma unroll
+    for (int sl = 0; sl < CPT; ++sl) {
+        const int cl = sl * 32 + lane, c = a.c_base + cl;
+        const float ac = __fmul_rn((float)(c + 1), g.step);
+        float inv = g.tiny ? __fdiv_rn(1.0f, ac) : __fdiv_rn(1.0f, (float)(c + 1)) * g.rstep;
+        if (!(ac >= FLT_MIN) || cl >= a.c_count) inv = 0.f;
+        inv2[sl] = pack2(inv, inv);
+        na2[sl] = pack2(-ac, -ac);
+        dacc[sl] = 0.0;
+    }
+    // candidates that may saturate: on first-slot-only elements (bounded above) and on the rest (the tensor's own count)
+    int ncl_first = (class_sat_count(1, CPT, 32, g.c_sat, flo, fhi, a.c_base) - a.c_base + 31) / 32;
+    ncl_first = max(0, min(1, ncl_first));
+    int ncl_rest = (g.c_sat - a.c_base + 31) / 32;
+    ncl_rest = max(0, min(CPT, ncl_rest));
+
+    const long long n4_total = (a.n + 3) >> 2;
+    const long long n4_full = a.n >> 2;
+    const long long n_tiles = (n4_total + a.tile4 - 1) / a.tile4;
+    const float4* x4 = reinterpret_cast<const float4*>(a.x);
+    const unsigned int lt_mask = (1u << lane) - 1u;
+    unsigned long long ev = 0ull;
+    double sq0 = 0.0, sq1 = 0.0;                     // squared sums of the dropped / first-slot-only elements
+
+    auto prefetch = [&](long long tl) {
+        const long long base4 = tl * a.tile4;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int i = tid * 4 + j;
+            if (base4 + i < n4_full) {
+                const unsigned int dst = (unsigned int)__cvta_generic_to_shared(raw4 + i);
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(x4 + base4 + i) : "memory");
+            }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    long long tl = blockIdx.x;
+    if (tl < n_tiles) prefetch(tl);
+    for (; tl < n_tiles; tl += gridDim.x) {
+        const long long base4 = tl * a.tile4;
+        asm volatile("cp.async.wait_all;" ::: "memory");
+        float vals[16];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            float4 v = make_float4(delta, delta, delta, delta);
+            const int i = tid * 4 + j;
+            if (base4 + i < n4_full) {
+                v = raw4[i];
+            } else {
+                const long long e = (base4 + i) << 2;
+                if (e < a.n) v.x = a.x[e];
+                if (e + 1 < a.n) v.y = a.x[e + 1];
+                if (e + 2 < a.n) v.z = a.x[e + 2];
+            }
+            vals[4 * j] = v.x - delta;
+            vals[4 * j + 1] = v.y - delta;
+            vals[4 * j + 2] = v.z - delta;
+            vals[4 * j + 3] = v.w - delta;
+        }
+        if (tl + gridDim.x < n_tiles) prefetch(tl + gridDim.x);   // the slots are free again: next tile on its way
+        // ---- three-way split: bit e of `first` / `rest` says where value e goes
+        unsigned int first = 0u, rest = 0u;
+        double z = 0.0;
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+            const float x = vals[e];
+            const float r = fabsf(x) * inv_thr - cbase_f;          // NaN for non-finite values: they go to the rest
+            const bool needed = !(r <= 1.0f) || (g.tiny && x != 0.f);
+            const bool wide = CPT > 1 && (!(r <= 33.0f) || (g.tiny && x != 0.f));   // slot 1 needs x iff r > 32 + 1
+            first |= (needed && !wide ? 1u : 0u) << e;
+            rest |= (wide ? 1u : 0u) << e;
+            const double xd = (double)x;
+            z = fma(needed ? 0.0 : xd, xd, z);
+        }
+        sq0 += z;
+        __syncwarp();                                 // the warp is done sweeping its previous share
+        if (!__any_sync(0xffffffffu, (first | rest) != 0u)) continue;
+        int n1 = 0, n2 = 0;                           // list lengths so far (same in every lane)
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+            const bool f1 = (first >> e) & 1u, f2 = (rest >> e) & 1u;
+            const unsigned int m1 = __ballot_sync(0xffffffffu, f1), m2 = __ballot_sync(0xffffffffu, f2);
+            if (f1) reg[n1 + __popc(m1 & lt_mask)] = vals[e];
+            if (f2) reg[region - 1 - (n2 + __popc(m2 & lt_mask))] = vals[e];
+            n1 += __popc(m1);
+            n2 += __popc(m2);
+        }
+        // zero padding: the first list up to a multiple of 4, the rest list down to one
+        const int n1p = (n1 + 3) & ~3, n2p = (n2 + 3) & ~3;
+        if (lane < n1p - n1) reg[n1 + lane] = 0.f;
+        if (lane < n2p - n2) reg[region - 1 - n2 - lane] = 0.f;
+        __syncwarp();
+        for (int i = lane; i < n1; i += 32) {
+            const double xd = (double)reg[i];
+            sq1 = fma(xd, xd, sq1);
+        }
+        const float4* reg4 = reinterpret_cast<const float4*>(reg);
+        if (n1 > 0) {
+            sweep_ncl<CPT, 1>(ncl_first, reg4, 0, n1p >> 2, inv2, na2, dacc, kMagic + flo, kMagic + fhi);
+            ev += (unsigned long long)n1p;
+        }
+        if (CPT > 1 && n2 > 0) {
+            sweep_ncl<CPT, CPT>(ncl_rest, reg4, (region - n2p) >> 2, region >> 2, inv2, na2, dacc, kMagic + flo, kMagic + fhi);
+            ev += (unsigned long long)n2p * CPT;
+        }
+    }
+    asm volatile("cp.async.wait_all;" ::: "memory");
+    __syncthreads();
+    if (warp > 0) {
+#pragma unroll
+        for (int sl = 0; sl < CPT; ++sl) xg[((warp - 1) * CPT + sl) * 32 + lane] = dacc[sl];
+    }
+    __syncthreads();
+    if (warp == 0) {
+        for (int w = 1; w < nwarp; ++w)
+#pragma unroll
+            for (int sl = 0; sl < CPT; ++sl) dacc[sl] += xg[((w - 1) * CPT + sl) * 32 + lane];
+    }
+    report_evaluations(a.evals, ev);
+    long long zero = 0;
+    block_sum2(sq0, zero, dscratch);
+    block_sum2(sq1, zero, dscratch);
+    if (warp == 0) {
+#pragma unroll
+        for (int sl = 0; sl < CPT; ++sl) {
+            const int cl = sl * 32 + lane;
+            if (cl < a.c_count)
+                a.partials[(long long)blockIdx.x * a.n_cand + a.c_base + cl] = dacc[sl] + (sl == 0 ? sq0 : sq0 + sq1);
         }
     }
 }

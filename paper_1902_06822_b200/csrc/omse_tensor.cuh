@@ -384,7 +384,7 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
 
 // The same sweep for launches whose slots hold 32 candidates (a warp is an element group of its own): every warp
 // keeps its own share of a tile (the float4s its lanes copied) and never waits for the block.  The elements are
-// split three ways with ballots, in a fixed order: dropped (coded 0 by every candidate of the launch), "first slot
+// split three ways in a fixed order (a warp scan of the per-lane counts): dropped (coded 0 by every candidate of the launch), "first slot
 // only" (by far the most for a tensor with many small values) and the rest, which all slots evaluate; the two lists
 // grow from the two ends of the warp's region.  Slot 0 adds the squared sum of the dropped elements, the other slots
 // that of the dropped and of the first-slot-only elements.
@@ -430,9 +430,10 @@ __global__ void __launch_bounds__(256) tensor_sweep_fine_kernel(const TensorArgs
     const long long n4_full = a.n >> 2;
     const long long n_tiles = (n4_total + a.tile4 - 1) / a.tile4;
     const float4* x4 = reinterpret_cast<const float4*>(a.x);
-    const unsigned int lt_mask = (1u << lane) - 1u;
+    // |x| * thr_scale counts candidates; with a denormal step every value goes to all slots (Inf, or NaN for 0)
+    const float thr_scale = g.tiny ? INFINITY : inv_thr;
     unsigned long long ev = 0ull;
-    double sq0 = 0.0, sq1 = 0.0;                     // squared sums of the dropped / first-slot-only elements
+    double sq_all = 0.0, sq1 = 0.0, sq2 = 0.0;       // squared sums: everything staged / first-slot-only / rest
 
     auto prefetch = [&](long long tl) {
         const long long base4 = tl * a.tile4;
@@ -472,30 +473,42 @@ __global__ void __launch_bounds__(256) tensor_sweep_fine_kernel(const TensorArgs
         if (tl + gridDim.x < n_tiles) prefetch(tl + gridDim.x);   // the slots are free again: next tile on its way
         // ---- three-way split: bit e of `first` / `rest` says where value e goes
         unsigned int first = 0u, rest = 0u;
-        double z = 0.0;
+        double tot = 0.0;                             // squared sum of everything this thread staged
 #pragma unroll
         for (int e = 0; e < 16; ++e) {
             const float x = vals[e];
-            const float r = fabsf(x) * inv_thr - cbase_f;          // NaN for non-finite values: they go to the rest
-            const bool needed = !(r <= 1.0f) || (g.tiny && x != 0.f);
-            const bool wide = CPT > 1 && (!(r <= 33.0f) || (g.tiny && x != 0.f));   // slot 1 needs x iff r > 32 + 1
+            const float r = fabsf(x) * thr_scale - cbase_f;        // NaN for non-finite values: they go to the rest
+            const bool needed = !(r <= 1.0f);
+            const bool wide = CPT > 1 && !(r <= 33.0f);             // slot 1 needs x iff r > 32 + 1
             first |= (needed && !wide ? 1u : 0u) << e;
             rest |= (wide ? 1u : 0u) << e;
             const double xd = (double)x;
-            z = fma(needed ? 0.0 : xd, xd, z);
+            tot = fma(xd, xd, tot);
         }
-        sq0 += z;
+        sq_all += tot;
         __syncwarp();                                 // the warp is done sweeping its previous share
         if (!__any_sync(0xffffffffu, (first | rest) != 0u)) continue;
-        int n1 = 0, n2 = 0;                           // list lengths so far (same in every lane)
+        // ---- the two lists, thread-major (lane 0's values first): offsets from a warp scan of the counts
+        const int packed = __popc(first) | (__popc(rest) << 16);
+        int incl = packed;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int u = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += u;
+        }
+        const int totals = __shfl_sync(0xffffffffu, incl, 31);
+        const int n1 = totals & 0xffff, n2 = totals >> 16;
+        int o1 = (incl - packed) & 0xffff;                        // first list grows upwards from 0
+        int o2 = region - 1 - ((incl - packed) >> 16);            // rest list grows downwards from the end
 #pragma unroll
         for (int e = 0; e < 16; ++e) {
-            const bool f1 = (first >> e) & 1u, f2 = (rest >> e) & 1u;
-            const unsigned int m1 = __ballot_sync(0xffffffffu, f1), m2 = __ballot_sync(0xffffffffu, f2);
-            if (f1) reg[n1 + __popc(m1 & lt_mask)] = vals[e];
-            if (f2) reg[region - 1 - (n2 + __popc(m2 & lt_mask))] = vals[e];
-            n1 += __popc(m1);
-            n2 += __popc(m2);
+            if ((first >> e) & 1u) reg[o1++] = vals[e];
+        }
+        if (n2 > 0) {
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+                if ((rest >> e) & 1u) reg[o2--] = vals[e];
+            }
         }
         // zero padding: the first list up to a multiple of 4, the rest list down to one
         const int n1p = (n1 + 3) & ~3, n2p = (n2 + 3) & ~3;
@@ -505,6 +518,10 @@ __global__ void __launch_bounds__(256) tensor_sweep_fine_kernel(const TensorArgs
         for (int i = lane; i < n1; i += 32) {
             const double xd = (double)reg[i];
             sq1 = fma(xd, xd, sq1);
+        }
+        for (int i = lane; i < n2; i += 32) {
+            const double xd = (double)reg[region - 1 - i];
+            sq2 = fma(xd, xd, sq2);
         }
         const float4* reg4 = reinterpret_cast<const float4*>(reg);
         if (n1 > 0) {
@@ -530,8 +547,10 @@ __global__ void __launch_bounds__(256) tensor_sweep_fine_kernel(const TensorArgs
     }
     report_evaluations(a.evals, ev);
     long long zero = 0;
-    block_sum2(sq0, zero, dscratch);
+    block_sum2(sq_all, zero, dscratch);
     block_sum2(sq1, zero, dscratch);
+    block_sum2(sq2, zero, dscratch);
+    const double sq0 = fmax(sq_all - sq1 - sq2, 0.0);   // what no slot evaluated
     if (warp == 0) {
 #pragma unroll
         for (int sl = 0; sl < CPT; ++sl) {
@@ -623,16 +642,18 @@ __global__ void __launch_bounds__(1024) tensor_finish_kernel(const TensorArgs a)
     }
 }
 
-// [x/alpha]_Zp without a division on the common path.  t = fl(x*inv + M) rounds the exact product to the
-// nearest integer (ties to even); with inv = fl(1/alpha) the product is within 2^-24 relative of x/alpha, and
-// so is the IEEE quotient, so both round to the same integer unless the product lies within
-// (|integer| + 1) * 2^-21 of a half-integer: `ambiguous` reports that, and the caller then takes the division.
-// Returns M + code (the code sits in the low mantissa bits).
-__device__ __forceinline__ float magic_code(float x, float inv, float clo, float chi, bool& ambiguous) {
+// [x/alpha]_Zp without a division on the common path.  t = fl(x*inv + M) rounds the exact product to the nearest
+// integer (ties to even); with inv = fl(1/alpha) the product is within 2^-24 relative of x/alpha, and so is the IEEE
+// quotient, so both round to the same integer unless the product lies within (|integer| + 1) * 2^-21 of a
+// half-integer.  Integers beyond the range by more than one saturate either way, so the test only has to hold for
+// |integer| <= range + 1: amb_thr = 1/2 - (range + 2) * 2^-21 serves every element; `ambiguous` reports a product
+// closer to a half-integer than that (or too large to be rounded by the addition), and the caller then takes the
+// division.  Returns M + code (the code sits in the low mantissa bits).
+__device__ __forceinline__ float magic_code(float x, float inv, float clo, float chi, float amb_thr, bool& ambiguous) {
     const float t = fmaf(x, inv, kMagic);
     const float rq = t - kMagic;
     const float delta = fmaf(x, inv, -rq);
-    ambiguous = fabsf(delta) > 0.5f - (fabsf(rq) + 1.0f) * 4.76837158203125e-7f;
+    ambiguous = !(fabsf(delta) <= amb_thr);
     return fminf(fmaxf(t, clo), chi);
 }
 
@@ -655,6 +676,7 @@ __global__ void __launch_bounds__(256) tensor_pass_kernel(const TensorArgs a) {
     TensorState* st = a.st;
     const float flo = (float)a.lo, fhi = (float)a.hi;
     const float clo = kMagic + flo, chi = kMagic + fhi;
+    const float amb_thr = 0.5f - (fmaxf(fhi, -flo) + 2.0f) * 4.76837158203125e-7f;
     const int n_list = MODE == 0 ? st->n_list : 1;
     if (MODE == 0 && n_list == 0) return;
     const float alpha_now = st->alpha;
@@ -676,6 +698,7 @@ __global__ void __launch_bounds__(256) tensor_pass_kernel(const TensorArgs a) {
         double ald[4];
         double acc[4] = {0.0, 0.0, 0.0, 0.0};
         long long sqq = 0;
+        int sqq32 = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             if (MODE == 0) {
@@ -693,12 +716,12 @@ __global__ void __launch_bounds__(256) tensor_pass_kernel(const TensorArgs a) {
 #pragma unroll
             for (int j = 0; j < nj; ++j) {
                 bool amb;
-                float tc = magic_code(x, inv[j], clo, chi, amb);
+                float tc = magic_code(x, inv[j], clo, chi, amb_thr, amb);
                 if (amb) tc = kMagic + (float)(al[j] > 0.f ? code_of(x, al[j], flo, fhi) : 0);   // rare: the division decides
                 const int q = magic_int(tc);
                 const double qd = int_double(q);
                 if (MODE == 1) {
-                    sqq += q * q;
+                    sqq32 += q * q;          // folded into the 64-bit sum after every float4 (q*q <= 2^14)
                     acc[j] = fma(xd, qd, acc[j]);
                 } else {
                     const double d = fma(-ald[j], qd, xd);
@@ -711,6 +734,8 @@ __global__ void __launch_bounds__(256) tensor_pass_kernel(const TensorArgs a) {
             element(v.y - delta);
             element(v.z - delta);
             element(v.w - delta);
+            sqq += sqq32;
+            sqq32 = 0;
         };
         // four 128-bit loads in flight per thread before any of them is used
         long long i = tid0;
@@ -724,6 +749,7 @@ __global__ void __launch_bounds__(256) tensor_pass_kernel(const TensorArgs a) {
         }
         for (; i < n4; i += stride) four(__ldg(x4 + i));
         for (long long e = (n4 << 2) + tid0; e < a.n; e += stride) element(a.x[e] - delta);
+        sqq += sqq32;
         for (int j = 0; j < nj; ++j) {
             long long q = sqq;
             block_sum2(acc[j], q, scratch);

@@ -55,6 +55,37 @@ __device__ __forceinline__ int code_of(float x, float alpha, float flo, float fh
     return (int)r;
 }
 
+// [x/alpha]_Zp without a division on the common path.  t = fl(x*inv + M) rounds the exact product to the nearest
+// integer (ties to even); with inv = fl(1/alpha) the product is within 2^-24 relative of x/alpha, and so is the IEEE
+// quotient, so both round to the same integer unless the product lies within (|integer| + 1) * 2^-21 of a
+// half-integer.  Integers beyond the range by more than one saturate either way, so the test only has to hold for
+// |integer| <= range + 1: amb_thr = 1/2 - (range + 2) * 2^-21 serves every element; `ambiguous` reports a product
+// closer to a half-integer than that (or too large to be rounded by the addition), and the caller then takes the
+// division.  Returns M + code (the code sits in the low mantissa bits).
+__device__ __forceinline__ float magic_code(float x, float inv, float clo, float chi, float amb_thr, bool& ambiguous) {
+    const float t = fmaf(x, inv, kMagic);
+    const float rq = t - kMagic;
+    const float delta = fmaf(x, inv, -rq);
+    ambiguous = !(fabsf(delta) <= amb_thr);
+    return fminf(fmaxf(t, clo), chi);
+}
+
+// integer held by M + q as an int, and as a double without a conversion instruction
+__device__ __forceinline__ int magic_int(float tc) { return __float_as_int(tc) - 0x4B400000; }
+__device__ __forceinline__ double int_double(int q) {
+    return __hiloint2double(0x43380000 + (q >> 31), q) - 6755399441055744.0;   // (1.5*2^52 + q) - 1.5*2^52, exact
+}
+
+// The code of x at scale alpha (inv = fl(1/alpha)) as an int, equal to code_of(x, alpha, flo, fhi) bit for bit.
+__device__ __forceinline__ int exact_code(float x, float alpha, float inv, float flo, float fhi, float amb_thr) {
+    bool amb;
+    const float tc = magic_code(x, inv, kMagic + flo, kMagic + fhi, amb_thr, amb);
+    return amb ? code_of(x, alpha, flo, fhi) : magic_int(tc);   // rare: the division decides
+}
+__device__ __forceinline__ float ambiguity_threshold(float flo, float fhi) {
+    return 0.5f - (fmaxf(fhi, -flo) + 2.0f) * 4.76837158203125e-7f;
+}
+
 // ---------------------------------------------------------------------------------------------
 // Candidate sweep over float4 indices [beg4, end4) of a shared-memory span.  CPT candidates per
 // thread, of which only the first NACT are evaluated on this span (the others are known to code

@@ -100,10 +100,12 @@ __device__ __forceinline__ double exact_sse_block(const float* xs, int k, float 
                                                    double* scratch) {
     double ss = 0.0;
     long long zero = 0;
+    const float inv = __fdiv_rn(1.0f, alpha), thr = ambiguity_threshold(flo, fhi);
+    const double ad = (double)alpha;
     for (int i = threadIdx.x; i < k; i += blockDim.x) {
         const float x = xs[i];
-        const double d = (double)x - (double)alpha * (double)code_of(x, alpha, flo, fhi);
-        ss += d * d;
+        const double d = fma(-ad, int_double(exact_code(x, alpha, inv, flo, fhi, thr)), (double)x);
+        ss = fma(d, d, ss);
     }
     block_sum2(ss, zero, scratch);
     return ss;
@@ -115,11 +117,12 @@ __device__ __forceinline__ float polish_block(const float* xs, int k, float alph
     for (int it = 0; it < n; ++it) {
         double sxq = 0.0;
         long long sqq = 0;
+        const float inv = __fdiv_rn(1.0f, alpha), thr = ambiguity_threshold(flo, fhi);
         for (int i = threadIdx.x; i < k; i += blockDim.x) {
             const float x = xs[i];
-            const int q = code_of(x, alpha, flo, fhi);
+            const int q = exact_code(x, alpha, inv, flo, fhi, thr);
             sqq += q * q;
-            sxq += (double)x * (double)q;
+            sxq = fma((double)x, int_double(q), sxq);
         }
         block_sum2(sxq, sqq, scratch);
         if (sqq == 0) break;
@@ -157,19 +160,16 @@ __device__ void partition_row(const RowSmem& s, int k, const GridSetup& g, int t
     const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
     const float inv_thr = g.rstep * (1.0f / 0.4999f);
     const float inv_tg = 1.0f / (float)tg;
-    const int span = (k + nthr - 1) / nthr;
-    const int beg = min(k, tid * span), end = min(k, beg + span);
-    // ---- pass 1: class counts of this thread's span (16-bit fields), squared sums per class
+    // Thread t owns the elements t, t + nthr, ... (conflict-free reads); within a class the elements keep the
+    // order (thread, then index), which is fixed, so the sums that follow do not depend on scheduling.
+    // ---- pass 1: class counts of this thread's elements (16-bit fields), squared sum of class 0
     u64 c0 = 0ull, c1 = 0ull;                  // classes 1..4 and 5..8
-    double d[CPT + 1];
-#pragma unroll
-    for (int b = 0; b <= CPT; ++b) d[b] = 0.0;
-    for (int i = beg; i < end; ++i) {
+    double zero_sq = 0.0;
+    for (int i = tid; i < k; i += nthr) {
         const float x = s.xs[i];
         const int nb = magnitude_class<CPT>(x, inv_thr, inv_tg);
-        const double xx = (double)x * (double)x;
-#pragma unroll
-        for (int b = 0; b <= CPT; ++b) d[b] += (nb == b) ? xx : 0.0;
+        const double xd = (double)x;
+        zero_sq = fma(nb == 0 ? xd : 0.0, xd, zero_sq);
         if (nb >= 5) c1 += 1ull << (16 * (nb - 5));
         else if (nb >= 1) c0 += 1ull << (16 * (nb - 1));
     }
@@ -202,22 +202,22 @@ __device__ void partition_row(const RowSmem& s, int k, const GridSetup& g, int t
         tot1 += a1;
     }
     // ---- class layout in xb: class CPT first, each class padded with zeros to a multiple of 4
-    int base[CPT + 1];
+    int base[CPT + 1], cnt[CPT + 1];
     int pos = 0;
 #pragma unroll
     for (int b = CPT; b >= 1; --b) {
-        const int cnt = (int)(((b >= 5 ? tot1 : tot0) >> (16 * ((b - 1) & 3))) & 0xffffull);
+        cnt[b] = (int)(((b >= 5 ? tot1 : tot0) >> (16 * ((b - 1) & 3))) & 0xffffull);
         base[b] = pos;
-        const int padded = (cnt + 3) & ~3;
+        const int padded = (cnt[b] + 3) & ~3;
         if (tid == 0) {
             s.seg[2 * b] = pos;
             s.seg[2 * b + 1] = padded;
         }
-        if (tid < padded - cnt) s.xb[pos + cnt + tid] = 0.f;
+        if (tid < padded - cnt[b]) s.xb[pos + cnt[b] + tid] = 0.f;
         pos += padded;
     }
-    // ---- pass 2: scatter in the original order within each class
-    for (int i = beg; i < end; ++i) {
+    // ---- pass 2: scatter
+    for (int i = tid; i < k; i += nthr) {
         const float x = s.xs[i];
         const int nb = magnitude_class<CPT>(x, inv_thr, inv_tg);
         if (nb >= 1) {
@@ -236,7 +236,19 @@ __device__ void partition_row(const RowSmem& s, int k, const GridSetup& g, int t
             s.xb[bs + within] = x;
         }
     }
-    // ---- squared sums per class -> what each slot skips: classes 0..sl
+    __syncthreads();
+    // ---- squared sums per class from the regrouped row (class 0 was summed on the way)
+    double d[CPT + 1];
+    d[0] = zero_sq;
+#pragma unroll
+    for (int b = 1; b <= CPT; ++b) {
+        double v = 0.0;
+        for (int i = tid; i < cnt[b]; i += nthr) {
+            const double xd = (double)s.xb[base[b] + i];
+            v = fma(xd, xd, v);
+        }
+        d[b] = v;
+    }
     double* ds = s.scratch + 64;                           // [nwarp][CPT+1]
 #pragma unroll
     for (int b = 0; b <= CPT; ++b) {
@@ -245,7 +257,7 @@ __device__ void partition_row(const RowSmem& s, int k, const GridSetup& g, int t
     }
     __syncthreads();
     if (tid < CPT) {
-        double acc = 0.0;
+        double acc = 0.0;                                  // slot `tid` skips classes 0..tid
         for (int b = 0; b <= tid; ++b)
             for (int w = 0; w < nwarp; ++w) acc += ds[w * (CPT + 1) + b];
         s.skip[tid] = acc;
@@ -430,10 +442,12 @@ __device__ PhiOut phi_block(const RowArgs& a, const RowSmem& s, int k, int k4, f
             const float ac = __fmul_rn((float)(c + 1), g.step);
             double ss = 0.0;
             long long zero = 0;
+            const float inv = __fdiv_rn(1.0f, ac), thr = ambiguity_threshold(flo, fhi);
+            const double ad = (double)ac;
             for (int i = tid; i < k; i += nthr) {
                 const float x = s.xs[i];
-                const double d = (double)x - (double)ac * (double)code_of(x, ac, flo, fhi);
-                ss += d * d;
+                const double d = fma(-ad, int_double(exact_code(x, ac, inv, flo, fhi, thr)), (double)x);
+                ss = fma(d, d, ss);
             }
             block_sum2(ss, zero, s.scratch);
             if (ss < best_sse) {   // increasing index: strict < keeps the lowest among equal errors
@@ -460,6 +474,8 @@ __device__ double emit_block(const RowSmem& s, int k, float alpha, float flo, fl
     const int tid = threadIdx.x, nthr = blockDim.x;
     double ss = 0.0;
     const bool zero = !(alpha > 0.f);
+    const float inv = zero ? 0.f : __fdiv_rn(1.0f, alpha), thr = ambiguity_threshold(flo, fhi);
+    const double ad = (double)alpha;
     const bool aligned = ((reinterpret_cast<unsigned long long>(codes) & 3ull) == 0) &&
                          ((reinterpret_cast<unsigned long long>(packed) & 1ull) == 0);
     if ((k & 3) == 0 && aligned) {
@@ -471,9 +487,9 @@ __device__ double emit_block(const RowSmem& s, int k, float alpha, float flo, fl
             int q[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                q[e] = zero ? 0 : code_of(x[e], alpha, flo, fhi);
-                const double d = (double)x[e] - (double)alpha * (double)q[e];
-                ss += d * d;
+                q[e] = zero ? 0 : exact_code(x[e], alpha, inv, flo, fhi, thr);
+                const double d = fma(-ad, int_double(q[e]), (double)x[e]);
+                ss = fma(d, d, ss);
             }
             if (codes) {
                 const unsigned int w = (q[0] & 0xff) | ((q[1] & 0xff) << 8) | ((q[2] & 0xff) << 16) | ((unsigned)(q[3] & 0xff) << 24);
@@ -762,9 +778,10 @@ __global__ void __launch_bounds__(OMSE_ROWS_MAX_THREADS) rows_kernel(const RowAr
                 }
                 if (!a.keep_x0 && j + 1 < a.n_tensors) {
                     // first sweep without a kept copy: the residual is updated in place
+                    const float inv = r.alpha > 0.f ? __fdiv_rn(1.0f, r.alpha) : 0.f, thr = ambiguity_threshold(flo, fhi);
                     for (int i = tid; i < k; i += nthr) {
                         const float x = s.xs[i];
-                        const int q = r.alpha > 0.f ? code_of(x, r.alpha, flo, fhi) : 0;
+                        const int q = r.alpha > 0.f ? exact_code(x, r.alpha, inv, flo, fhi, thr) : 0;
                         s.xs[i] = fmaf(-r.alpha, (float)q, x);
                     }
                 }

@@ -99,6 +99,7 @@ __device__ __forceinline__ float small_row_epilogue(const RowArgs& a, const RowT
                                                     unsigned int& st) {
     const int lane = threadIdx.x & 31;
     const float flo = (float)a.lo[0], fhi = (float)a.hi[0];
+    const float thr = ambiguity_threshold(flo, fhi);
     struct { float step; } g = {rp.step};
     float alpha = 0.f;
     int best = -1;
@@ -145,11 +146,13 @@ __device__ __forceinline__ float small_row_epilogue(const RowArgs& a, const RowT
                         const int c = c0 + __ffs(mask) - 1;
                         mask &= mask - 1;
                         const float ac = __fmul_rn((float)(c + 1), g.step);
+                        const float inv = __fdiv_rn(1.0f, ac);
+                        const double ad = (double)ac;
                         double ss = 0.0;
                         for (int i = lane; i < k; i += 32) {
                             const float x = xr[i];
-                            const double d = (double)x - (double)ac * (double)code_of(x, ac, flo, fhi);
-                            ss += d * d;
+                            const double d = fma(-ad, int_double(exact_code(x, ac, inv, flo, fhi, thr)), (double)x);
+                            ss = fma(d, d, ss);
                         }
                         ss = warp_allsum(ss);
                         if (ss < best_sse || (ss == best_sse && c < best)) {
@@ -163,11 +166,12 @@ __device__ __forceinline__ float small_row_epilogue(const RowArgs& a, const RowT
             for (int it = 0; it < a.refine_iters; ++it) {
                 double sxq = 0.0;
                 int sqq = 0;
+                const float inv = __fdiv_rn(1.0f, alpha);
                 for (int i = lane; i < k; i += 32) {
                     const float x = xr[i];
-                    const int q = code_of(x, alpha, flo, fhi);
+                    const int q = exact_code(x, alpha, inv, flo, fhi, thr);
                     sqq += q * q;
-                    sxq += (double)x * (double)q;
+                    sxq = fma((double)x, int_double(q), sxq);
                 }
                 sxq = warp_allsum(sxq);
                 sqq = warp_allsum(sqq);
@@ -188,6 +192,8 @@ __device__ __forceinline__ float small_row_epilogue(const RowArgs& a, const RowT
     // ---- final codes, squared error, emission
     const long long row_base = row * T.K;
     const bool zero = !(alpha > 0.f);
+    const float inv_f = zero ? 0.f : __fdiv_rn(1.0f, alpha);
+    const double ad = (double)alpha;
     double ss = 0.0;
     const bool aligned = ((reinterpret_cast<unsigned long long>(T.codes) & 3ull) == 0) &&
                          ((reinterpret_cast<unsigned long long>(T.packed) & 1ull) == 0);
@@ -199,9 +205,9 @@ __device__ __forceinline__ float small_row_epilogue(const RowArgs& a, const RowT
             int q[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                q[e] = zero ? 0 : code_of(x[e], alpha, flo, fhi);
-                const double d = (double)x[e] - (double)alpha * (double)q[e];
-                ss += d * d;
+                q[e] = zero ? 0 : exact_code(x[e], alpha, inv_f, flo, fhi, thr);
+                const double d = fma(-ad, int_double(q[e]), (double)x[e]);
+                ss = fma(d, d, ss);
             }
             if (T.codes) {
                 const unsigned int w = (q[0] & 0xff) | ((q[1] & 0xff) << 8) | ((q[2] & 0xff) << 16) | ((unsigned)(q[3] & 0xff) << 24);
@@ -352,19 +358,16 @@ __device__ void small_unit(const RowArgs& a, const RowTensor& T, long long unit_
             const SmallRowParams rp = rowp[r];
             const bool plain = (rp.flags & 3) != 0;           // denormal-range or unusable row: one class, all slots
             const float inv_thr = rp.rstep * (1.0f / 0.4999f), inv_tg = 1.0f / (float)a.tg;
-            const int span = (k + 31) >> 5;
-            const int beg = min(k, lane * span), end = min(k, beg + span);
             const float* xr = xs + r * kpad;
+            // lane l owns the elements l, l + 32, ...; within a class they keep the order (lane, then index)
             u64 c0 = 0ull, c1 = 0ull;
             double d[CPT + 1];
-#pragma unroll
-            for (int b = 0; b <= CPT; ++b) d[b] = 0.0;
-            for (int i = beg; i < end; ++i) {
+            d[0] = 0.0;
+            for (int i = lane; i < k; i += 32) {
                 const float x = xr[i];
                 const int nb = plain ? CPT : magnitude_class<CPT>(x, inv_thr, inv_tg);
-                const double xx = (double)x * (double)x;
-#pragma unroll
-                for (int b = 0; b <= CPT; ++b) d[b] += (nb == b) ? xx : 0.0;
+                const double xd = (double)x;
+                d[0] = fma(nb == 0 ? xd : 0.0, xd, d[0]);
                 if (nb >= 5) c1 += 1ull << (16 * (nb - 5));
                 else if (nb >= 1) c0 += 1ull << (16 * (nb - 1));
             }
@@ -380,22 +383,22 @@ __device__ void small_unit(const RowArgs& a, const RowTensor& T, long long unit_
             }
             u64 off0 = i0 - c0, off1 = i1 - c1;
             const u64 tot0 = __shfl_sync(0xffffffffu, i0, 31), tot1 = __shfl_sync(0xffffffffu, i1, 31);
-            int base[CPT + 1];
+            int base[CPT + 1], cnt[CPT + 1];
             int pos = 0;
             float* xbr = xb + r * kb;
 #pragma unroll
             for (int b = CPT; b >= 1; --b) {
-                const int cnt = (int)(((b >= 5 ? tot1 : tot0) >> (16 * ((b - 1) & 3))) & 0xffffull);
+                cnt[b] = (int)(((b >= 5 ? tot1 : tot0) >> (16 * ((b - 1) & 3))) & 0xffffull);
                 base[b] = pos;
-                const int padded = (cnt + 3) & ~3;
+                const int padded = (cnt[b] + 3) & ~3;
                 if (lane == 0) {
                     seg[(r * (CPT + 1) + b) * 2] = pos;
                     seg[(r * (CPT + 1) + b) * 2 + 1] = padded;
                 }
-                if (lane < padded - cnt) xbr[pos + cnt + lane] = 0.f;
+                if (lane < padded - cnt[b]) xbr[pos + cnt[b] + lane] = 0.f;
                 pos += padded;
             }
-            for (int i = beg; i < end; ++i) {
+            for (int i = lane; i < k; i += 32) {
                 const float x = xr[i];
                 const int nb = plain ? CPT : magnitude_class<CPT>(x, inv_thr, inv_tg);
                 if (nb >= 1) {
@@ -413,6 +416,17 @@ __device__ void small_unit(const RowArgs& a, const RowTensor& T, long long unit_
                     for (int b = 1; b <= CPT; ++b) bs = (nb == b) ? base[b] : bs;
                     xbr[bs + within] = x;
                 }
+            }
+            __syncwarp();
+            // squared sums of classes 1.. from the regrouped row (class 0 was summed on the way)
+#pragma unroll
+            for (int b = 1; b <= CPT; ++b) {
+                double v = 0.0;
+                for (int i = lane; i < cnt[b]; i += 32) {
+                    const double xd = (double)xbr[base[b] + i];
+                    v = fma(xd, xd, v);
+                }
+                d[b] = v;
             }
             double run = 0.0;                                   // slot sl skips classes 0..sl
 #pragma unroll

@@ -642,27 +642,6 @@ __global__ void __launch_bounds__(1024) tensor_finish_kernel(const TensorArgs a)
     }
 }
 
-// [x/alpha]_Zp without a division on the common path.  t = fl(x*inv + M) rounds the exact product to the nearest
-// integer (ties to even); with inv = fl(1/alpha) the product is within 2^-24 relative of x/alpha, and so is the IEEE
-// quotient, so both round to the same integer unless the product lies within (|integer| + 1) * 2^-21 of a
-// half-integer.  Integers beyond the range by more than one saturate either way, so the test only has to hold for
-// |integer| <= range + 1: amb_thr = 1/2 - (range + 2) * 2^-21 serves every element; `ambiguous` reports a product
-// closer to a half-integer than that (or too large to be rounded by the addition), and the caller then takes the
-// division.  Returns M + code (the code sits in the low mantissa bits).
-__device__ __forceinline__ float magic_code(float x, float inv, float clo, float chi, float amb_thr, bool& ambiguous) {
-    const float t = fmaf(x, inv, kMagic);
-    const float rq = t - kMagic;
-    const float delta = fmaf(x, inv, -rq);
-    ambiguous = !(fabsf(delta) <= amb_thr);
-    return fminf(fmaxf(t, clo), chi);
-}
-
-// integer held by M + q as an int, and as a double without a conversion instruction
-__device__ __forceinline__ int magic_int(float tc) { return __float_as_int(tc) - 0x4B400000; }
-__device__ __forceinline__ double int_double(int q) {
-    return __hiloint2double(0x43380000 + (q >> 31), q) - 6755399441055744.0;   // (1.5*2^52 + q) - 1.5*2^52, exact
-}
-
 // Grid-wide pass over the tensor; sums in fp64, codes equal to those of the IEEE division (see magic_code).
 //   MODE 0 (rescore): squared error at each listed candidate; the last block picks the best.
 //   MODE 1 (refine):  <x,q> and <q,q> at st->alpha; the last block sets alpha <- <x,q>/<q,q>.
@@ -676,7 +655,7 @@ __global__ void __launch_bounds__(256) tensor_pass_kernel(const TensorArgs a) {
     TensorState* st = a.st;
     const float flo = (float)a.lo, fhi = (float)a.hi;
     const float clo = kMagic + flo, chi = kMagic + fhi;
-    const float amb_thr = 0.5f - (fmaxf(fhi, -flo) + 2.0f) * 4.76837158203125e-7f;
+    const float amb_thr = ambiguity_threshold(flo, fhi);
     const int n_list = MODE == 0 ? st->n_list : 1;
     if (MODE == 0 && n_list == 0) return;
     const float alpha_now = st->alpha;

@@ -22,10 +22,35 @@ constexpr float kMagic = 12582912.0f;   // 1.5 * 2^23
 #ifndef OMSE_FLUSH4
 #define OMSE_FLUSH4 32
 #endif
-#ifndef OMSE_UNROLL
-#define OMSE_UNROLL 2
+// float4 loads per unrolled step of the sweep loop, by the number of active candidate slots: few slots mean few
+// independent chains per load, so several loads are interleaved; many slots have the parallelism already and are
+// kept compact (the kernels are sensitive to instruction-cache pressure)
+#ifndef OMSE_UNROLL_1
+#define OMSE_UNROLL_1 8
 #endif
-constexpr int kUnroll = OMSE_UNROLL;      // float4 loads per unrolled step of the sweep loop
+#ifndef OMSE_UNROLL_2
+#define OMSE_UNROLL_2 3
+#endif
+#ifndef OMSE_UNROLL_3
+#define OMSE_UNROLL_3 2
+#endif
+#ifndef OMSE_UNROLL_N
+#define OMSE_UNROLL_N 1
+#endif
+#ifndef OMSE_ACC_UNROLL_1
+#define OMSE_ACC_UNROLL_1 1
+#endif
+#ifndef OMSE_ACC_UNROLL_2
+#define OMSE_ACC_UNROLL_2 1
+#endif
+template <int NACT>
+struct AccumUnroll {      // the same for the short spans of the batched short-row path
+    static constexpr int value = NACT == 1 ? OMSE_ACC_UNROLL_1 : NACT == 2 ? OMSE_ACC_UNROLL_2 : 1;
+};
+template <int NACT>
+struct SweepUnroll {
+    static constexpr int value = NACT == 1 ? OMSE_UNROLL_1 : NACT == 2 ? OMSE_UNROLL_2 : NACT == 3 ? OMSE_UNROLL_3 : OMSE_UNROLL_N;
+};
 constexpr int kFlushEvery4 = OMSE_FLUSH4;   // float4 loads between folds of the fp32 partial sums into fp64
 constexpr double kRescoreBand = 4e-6;   // candidates within this relative band of the fp32 minimum are re-scored
 
@@ -106,7 +131,7 @@ __device__ __forceinline__ void sweep_range(const float4* __restrict__ xs4, int 
     int i = beg4;
     while (i < end4) {
         const int stop = min(end4, i + kFlushEvery4);
-#pragma unroll(kUnroll)
+#pragma unroll(SweepUnroll<NACT>::value)
         for (; i < stop; ++i) {
             const float4 v = xs4[i];
             const u64 xa = pack2(v.x, v.y), xb = pack2(v.z, v.w);
@@ -193,7 +218,7 @@ __device__ __forceinline__ void sweep_accum(const float4* __restrict__ xs4, int 
                                             float clo, float chi) {
     const u64 M2 = pack2(kMagic, kMagic);
     const u64 NM2 = pack2(-kMagic, -kMagic);
-#pragma unroll 1
+#pragma unroll(AccumUnroll<NACT>::value)
     for (int i = beg4; i < end4; ++i) {
         const float4 v = xs4[i];
         const u64 xa = pack2(v.x, v.y), xb = pack2(v.z, v.w);

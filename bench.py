@@ -35,7 +35,7 @@ INSTR_PER_EVAL = 6            # reference FP32 sequence per (element, candidate)
 LANE_OPS_PER_EVAL = 4         # FMA-pipe lane operations of an evaluation the kernels execute: fma, add, fma, fma
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the timed kernel from an ncu capture of the
 # default workload; None whenever the kernel has changed since the capture
-NCU_TRAFFIC_BYTES = None
+NCU_TRAFFIC_BYTES = 109_099_776
 E2E_CHUNKS = 12               # batched launches per end-to-end step (copies of later chunks overlap earlier searches)
 N_SM, LANES_PER_SM = 148, 128
 WORKLOAD = "resnet50_weight_set_54_tensors_25.5M_params_signed4bit_kernelwise_1024cand_3refine_packed"

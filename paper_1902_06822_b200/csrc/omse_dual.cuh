@@ -130,29 +130,32 @@ __global__ void __launch_bounds__(kDualThreads) dual_kernel(const DualArgs a) {
                     const bool full = !(ratio <= 16.f) || 2 * w + 1 >= n_levels;
                     const int n_t = full ? n_levels : 2 * w + 1;
                     ev += (unsigned long long)k * (unsigned long long)(2 * ((n_t + 1) / 2)) * kDualDpt;
+                    const float clo2 = kMagic + flo2, chi2 = kMagic + fhi2, flo1 = (float)a.lo1, fhi1 = (float)a.hi1;
                     for (int i = 0; i < k; ++i) {
                         const float x = xs[i];
-                        const float t0 = full ? (float)a.lo1 : rintf(x * inv1) - (float)w;
+                        const float t0 = full ? flo1 : rintf(x * inv1) - (float)w;
+                        // smallest |error| over the first codes: squaring is monotone, so the square of the smallest
+                        // magnitude is the smallest squared error
                         float best[kDualDpt];
 #pragma unroll
                         for (int j = 0; j < kDualDpt; ++j) best[j] = INFINITY;
                         // two first codes per step (the second clamps to the last one when n_t is odd: a repeat
                         // cannot change a minimum): eight independent chains in flight
                         for (int s = 0; s < n_t; s += 2) {
-                            const float ta = fminf(fmaxf(t0 + (float)s, (float)a.lo1), (float)a.hi1);
-                            const float tb = fminf(fmaxf(t0 + (float)min(s + 1, n_t - 1), (float)a.lo1), (float)a.hi1);
+                            const float ta = fminf(fmaxf(t0 + (float)s, flo1), fhi1);
+                            const float tb = fminf(fmaxf(t0 + (float)min(s + 1, n_t - 1), flo1), fhi1);
                             const float ra = fmaf(-a1, ta, x), rb = fmaf(-a1, tb, x);
 #pragma unroll
                             for (int j = 0; j < kDualDpt; ++j) {
                                 float ua = fmaf(ra, inv2[j], kMagic), ub = fmaf(rb, inv2[j], kMagic);
-                                ua = fminf(fmaxf(ua, kMagic + flo2), kMagic + fhi2);
-                                ub = fminf(fmaxf(ub, kMagic + flo2), kMagic + fhi2);
+                                ua = fminf(fmaxf(ua, clo2), chi2);
+                                ub = fminf(fmaxf(ub, clo2), chi2);
                                 const float ea = fmaf(-a2[j], ua - kMagic, ra), eb = fmaf(-a2[j], ub - kMagic, rb);
-                                best[j] = fminf(best[j], fminf(ea * ea, eb * eb));
+                                best[j] = fminf(best[j], fminf(fabsf(ea), fabsf(eb)));
                             }
                         }
 #pragma unroll
-                        for (int j = 0; j < kDualDpt; ++j) acc[j] += best[j];
+                        for (int j = 0; j < kDualDpt; ++j) acc[j] = fmaf(best[j], best[j], acc[j]);
                         if ((i & 63) == 63) {
 #pragma unroll
                             for (int j = 0; j < kDualDpt; ++j) {

@@ -193,8 +193,8 @@ int omse_alg1_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, int64
                        int8_t* d_codes, uint8_t* d_packed);
 
 /*
- * Algorithm 1 with its loop condition (Section 3.5, Algorithm 1: the sweeps go on while the convergence rate
- * exceeds a threshold).  The paper does not define the rate; here it is the relative decrease of a kernel's
+ * Algorithm 1 with its loop condition (Section 3.5, Algorithm 1: the sweeps go on until the error stops
+ * improving by more than a threshold).  The paper does not define the rate; here it is the relative decrease of a kernel's
  * squared error over one sweep, (E_prev - E_cur)/E_prev, E being the error after the last tensor's update and
  * E_0 = ||T_k||^2.  Each kernel stops on its own after the first sweep whose rate is not above eps, or after
  * max_sweeps sweeps.  d_sweeps_done (nullable) [n_kernels] int32: sweeps that ran; history entries of sweeps

@@ -92,7 +92,7 @@ void omse_oracle_codes(const float *x, int64_t n, float alpha, int bits, int is_
         codes[i] = (alpha > 0.0f) ? (int8_t)code_of(x[i], alpha, lo, hi) : (int8_t)0;
 }
 
-/* The candidate scales of the line search (Section 3.4: "a given grid"): C points spaced
+/* The candidate scales of the line search (Section 3.4 names a grid and leaves its points open): C points spaced
  * linearly in (0, hi_frac*max|x|], every operation in binary32. */
 float omse_oracle_candidate(float max_abs, float hi_frac, int n_cand, int c)
 {
@@ -251,7 +251,7 @@ void omse_oracle_activation_scale(const float *x, int64_t n, int bits, int is_si
  * Algorithm 1 (alternating optimisation for multiple quantization) on one segment:
  * for each sweep, for j = 1..n: r = T - sum_{i != j} alpha_i T~^i, (alpha_j, T~^j) = phi(r, p_j).
  * All alpha_i and T~^i start at zero, so the first sweep quantizes the residual of the
- * previous approximation (Section 3.7, "one iteration only").  The residual is formed in
+ * previous approximation (Section 3.7 runs a single sweep).  The residual is formed in
  * binary32 by successive fused multiply-adds in increasing i.
  * Outputs (last sweep): alpha[n], sse[n] (error after tensors 1..j were updated),
  * best_idx[n], codes[n][k]; r_scratch[k] is caller-provided scratch.
@@ -263,7 +263,7 @@ static void alg1_segment(const float *x, int64_t k, const int *bits, const int *
                          double eps, int32_t *sweeps_done, uint32_t *status)
 {   /* is_signed: one flag per quantized tensor; sse_sweeps (nullable): [n_sweeps][n_tensors] with stride
      * out_stride, the error after every update, i.e. the convergence history of the while-loop.
-     * eps >= 0: the while-condition of Algorithm 1.  The paper does not define its "convergence rate";
+     * eps >= 0: the while-condition of Algorithm 1.  The paper does not define the rate its condition tests;
      * here it is the relative decrease of the squared error over one sweep, (E_prev - E_cur)/E_prev
      * with E the error after the last tensor's update and E_0 = ||T||^2 (all tensors zero); the loop
      * ends after the first sweep whose rate is not above eps (tested as E_prev - E_cur > eps*E_prev),

@@ -196,7 +196,7 @@ def test_power_of_two_scaling_is_exact_and_permutation_keeps_alpha():
 
 
 def test_grid_search_beats_alternation_from_the_uniform_start_somewhere():
-    """Section 3.4: alternation alone is not robust (non-convex objective); the grid is."""
+    """Section 3.4: alternation alone can stop in a local minimum of the non-convex objective; the grid cannot."""
     w = synth.resnet50_weights(seed=2)[1][1][:64]       # 64 rows of a 1x1 convolution
     grid = orc.quantize_rows(w, 4, True, 256, 1.0, 3).sse
     alt = orc.quantize_rows(w, 4, True, 1, 1.0 / 7, 10).sse   # uniform start + 10 alternations

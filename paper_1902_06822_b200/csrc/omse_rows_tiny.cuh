@@ -1,7 +1,7 @@
 // Very short kernels (up to 32 weights, e.g. the 3x3x3 kernels of a first convolution) in large
 // numbers: one THREAD owns one row.  The row sits in registers as packed pairs, the thread walks the
-// whole grid of candidate scales serially (no reduction across threads at all), keeps the best two
-// candidates, re-scores them in fp64 when they are within the fp32 noise band, polishes and emits.
+// whole grid of candidate scales serially (no reduction across threads at all), re-scores in fp64 the
+// candidates within the fp32 noise band of the minimum, polishes and emits.
 // A work unit is blockDim.x consecutive rows, staged and written back through shared memory so that
 // global accesses stay coalesced.  Same candidate arithmetic and decisions as the other paths.
 #pragma once
@@ -114,25 +114,25 @@ __device__ void tiny_unit(const RowArgs& a, const RowTensor& T, long long unit_l
             }
             return ss;
         };
-        float b1v = INFINITY, b2v = INFINITY, b3v = INFINITY;
-        int b1i = 0x7fffffff, b2i = 0x7fffffff;
+        // The grid is walked once.  Beside the smallest fp32 error the walk keeps the index window [w_lo, w_hi] outside
+        // which no candidate can lie within the noise band of the final minimum: a candidate inside the band of the
+        // final minimum is inside the band of the running minimum when it is seen (the running minimum only falls),
+        // and when the running minimum falls by more than the band everything seen before drops out.
+        float b1v = INFINITY;
+        int b1i = 0x7fffffff, w_lo = 0, w_hi = -1;
+        const float band_f = 1.0f + 1.25f * (float)kRescoreBand;   // a little wider than the fp64 test below: a superset
         if (!degenerate) {
             float cf = 0.f;                               // c + 1 as a float (exact: n_cand <= 4096)
             for (int c = 0; c < a.n_cand; ++c) {
                 cf += 1.0f;
                 const float v = sweep_error(c, cf);
-                if (v < b1v) {          // ascending c: strict < keeps the lowest index
-                    b3v = b2v;
-                    b2v = b1v;
-                    b2i = b1i;
-                    b1v = v;
-                    b1i = c;
-                } else if (v < b2v) {
-                    b3v = b2v;
-                    b2v = v;
-                    b2i = c;
-                } else if (v < b3v) {
-                    b3v = v;
+                if (v <= b1v * band_f) {
+                    w_hi = c;
+                    if (v < b1v) {      // ascending c: strict < keeps the lowest index
+                        if (v * band_f < b1v) w_lo = c;
+                        b1v = v;
+                        b1i = c;
+                    }
                 }
             }
             ev += (unsigned long long)a.n_cand * (2ull * KP);
@@ -143,26 +143,23 @@ __device__ void tiny_unit(const RowArgs& a, const RowTensor& T, long long unit_l
         } else {
             best = b1i;
             // ---- candidates within the fp32 noise band of the minimum: decide in fp64 with true division
-            const double band = (double)b1v * (1.0 + kRescoreBand);
-            if ((double)b3v <= band) {
-                // three or more: walk the grid once more and re-score every candidate in the band
+            if (w_hi > w_lo) {
+                const double band = (double)b1v * (1.0 + kRescoreBand);
                 double best_sse = INFINITY;
                 best = 0x7fffffff;
-                float cf = 0.f;
-                for (int c = 0; c < a.n_cand; ++c) {
-                    cf += 1.0f;
-                    if ((double)sweep_error(c, cf) <= band) {
+                int n_band = 0;
+                for (int c = w_lo; c <= w_hi; ++c) {
+                    if ((double)sweep_error(c, (float)(c + 1)) <= band) {
                         const double ss = exact_error(c);
+                        ++n_band;
                         if (ss < best_sse) {   // ascending c: strict < keeps the lowest index
                             best_sse = ss;
                             best = c;
                         }
                     }
                 }
-                ev += (unsigned long long)a.n_cand * (2ull * KP);
-            } else if ((double)b2v <= band) {
-                const double s1 = exact_error(b1i), s2 = exact_error(b2i);
-                if (s2 < s1 || (s2 == s1 && b2i < b1i)) best = b2i;
+                ev += (unsigned long long)(w_hi - w_lo + 1) * (2ull * KP);
+                if (n_band == 0) best = b1i;
             }
             // ---- polish
             alpha = __fmul_rn((float)(best + 1), g.step);

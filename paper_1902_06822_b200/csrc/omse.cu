@@ -302,16 +302,45 @@ int enqueue_tensor_search(const TensorEnv& env, omse::TensorArgs& a, int refine_
     const int kFine = 256;        // candidates of the first launch: 32 per slot
     int split = a.n_cand, nb_lo = 1, nb_hi = 1;
     if (n > 0) {
-        omse::tensor_absmax_kernel<<<(unsigned)absmax_grid, 256, 0, s>>>(a.x, n, a.st, a.status);
+        // Two sweep launches share tile flags when they fit: a bit per 4,096-element tile in the (not yet used)
+        // curve buffer, and the first launch's per-block squared sums in the (not yet used) candidate list.
+        const long long flag_tile4 = 4 * 256;                       // tile of the first sweep launch
+        const long long n_flag_tiles = (((n + 3) >> 2) + flag_tile4 - 1) / flag_tile4;
+        const bool two = a.n_cand > kFine;
+        // curve: n_cand doubles = 64*n_cand bits; list: n_cand/2 doubles, enough for three blocks per SM
+        const bool flags = two && n_flag_tiles <= 64ll * a.n_cand && a.n_cand / 2 >= 3 * env.n_sm;
+        const int flag_words = flags ? (int)((n_flag_tiles + 31) >> 5) : 0;
+        omse::tensor_absmax_kernel<<<(unsigned)absmax_grid, 256, 0, s>>>(a.x, n, a.st, a.status,
+                                                                      reinterpret_cast<unsigned int*>(a.curve), flag_words);
         if (a.delta_out) omse::tensor_offset_kernel<<<1, 32, 0, s>>>(a.st);
         int rc;
-        if (a.n_cand <= kFine) {
+        if (!two) {
             rc = sweep_launch(env, a, 0, a.n_cand, cpt_for(a.n_cand), &nb_lo);
             nb_hi = nb_lo;
         } else {
             split = kFine;
-            rc = sweep_launch(env, a, 0, kFine, 8, &nb_lo);
-            if (rc == OMSE_OK) rc = sweep_launch(env, a, kFine, a.n_cand - kFine, 8, &nb_hi);
+            omse::TensorArgs lo = a;
+            if (flags) {
+                lo.tile_flags = reinterpret_cast<unsigned int*>(a.curve);
+                lo.flag_words = flag_words;
+                lo.flag_tile4 = (int)flag_tile4;
+                lo.flag_role = 1;
+                lo.flag_split = (float)(kFine + 1);
+                lo.block_totals = reinterpret_cast<double*>(a.list);
+                // the list holds n_cand ints = n_cand/2 doubles: one per block of the first launch
+                const long long cap = (long long)(a.n_cand / 2) * a.n_cand;
+                if (lo.partial_doubles > cap) lo.partial_doubles = cap;
+            }
+            rc = sweep_launch(env, lo, 0, kFine, 8, &nb_lo);
+            omse::TensorArgs hi = a;
+            if (flags) {
+                hi.tile_flags = lo.tile_flags;
+                hi.flag_tile4 = lo.flag_tile4;
+                hi.flag_role = 2;
+                hi.block_totals = lo.block_totals;
+                hi.n_totals = nb_lo;
+            }
+            if (rc == OMSE_OK) rc = sweep_launch(env, hi, kFine, a.n_cand - kFine, 8, &nb_hi);
         }
         if (rc != OMSE_OK) return rc;
     }

@@ -32,6 +32,16 @@ struct TensorArgs {
     int tg, groups;         // sweep block = groups*tg threads; candidate c = c_base + slot*tg + t
     int c_base, c_count;    // candidates [c_base, c_base + c_count) are swept by this launch
     int tile4;              // float4s per tile
+    // Tile flags between the two sweep launches (all nullable / 0): the first launch sets bit t when tile t (of
+    // flag_tile4 float4s) holds a value that reaches the second launch's first candidate, and leaves the squared sum
+    // of everything each of its blocks staged in block_totals; the second launch then reads only flagged tiles.
+    unsigned int* tile_flags;
+    int flag_words;         // words of tile_flags (the absmax kernel clears them)
+    int flag_tile4;
+    int flag_role;          // 1: this launch sets the flags, 2: this launch uses them
+    float flag_split;       // role 1: a value with |x|/(0.4999*step) above this reaches the second launch
+    double* block_totals;   // role 1: [gridDim.x] written; role 2: n_totals entries read
+    int n_totals;
     TensorState* st;
     double* partials;       // sweep: [grid][n_cand]; passes: [blocks][listed candidates] doubles + [blocks] int64
     long long partial_doubles;   // capacity of `partials`
@@ -81,8 +91,10 @@ __global__ void tensor_offset_kernel(TensorState* st) {
 }
 
 __global__ void __launch_bounds__(256) tensor_absmax_kernel(const float* __restrict__ x, long long n,
-                                                             TensorState* st, unsigned int* status) {
+                                                             TensorState* st, unsigned int* status,
+                                                             unsigned int* tile_flags, int flag_words) {
     __shared__ double scratch[64];
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < flag_words; i += gridDim.x * blockDim.x) tile_flags[i] = 0u;
     float mpos = 0.f, mneg = 0.f, lo = INFINITY, hi = -INFINITY;
     bool bad = false;
     const long long n4 = n >> 2;
@@ -202,10 +214,24 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
-    long long tl = blockIdx.x;
+    // With tile flags from the first launch only the tiles that hold a value for this launch are read at all.
+    const bool flagged_only = a.flag_role == 2 && a.tile_flags != nullptr;
+    auto next_tile = [&](long long tl) {             // first tile >= tl of this block's sequence that has to be read
+        if (!flagged_only) return tl;
+        for (; tl < n_tiles; tl += gridDim.x) {
+            const long long f0 = (tl * a.tile4) / a.flag_tile4;
+            const long long f1 = (min((tl + 1) * (long long)a.tile4, n4_total) - 1) / a.flag_tile4;
+            bool hit = false;
+            for (long long f = f0; f <= f1; ++f) hit |= (__ldg(a.tile_flags + (f >> 5)) >> (f & 31)) & 1u;
+            if (hit) break;
+        }
+        return tl;
+    };
+    long long tl = next_tile(blockIdx.x);
     if (tl < n_tiles) prefetch(tl);
-    for (; tl < n_tiles; tl += gridDim.x) {
+    while (tl < n_tiles) {
         const long long base4 = tl * a.tile4;
+        const long long tl_next = next_tile(tl + gridDim.x);
         asm volatile("cp.async.wait_all;" ::: "memory");
         // ---- this thread's span into registers (elements past the end count as zeros)
         float vals[16];
@@ -229,7 +255,8 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
             vals[4 * j + 2] = v.z - delta;
             vals[4 * j + 3] = v.w - delta;
         }
-        if (tl + gridDim.x < n_tiles) prefetch(tl + gridDim.x);   // the slots are free again: next tile on its way
+        tl = tl_next;
+        if (tl < n_tiles) prefetch(tl);              // the slots are free again: next tile on its way
 #pragma unroll
         for (int e = 0; e < 16; ++e) {
             const float x = vals[e];
@@ -363,15 +390,35 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
         }
     }
     report_evaluations(a.evals, ev);
-    // ---- what each slot skipped in this block: classes 0..sl (block sums in fixed order)
+    // ---- what each slot skipped (block sums in fixed order)
     long long zero = 0;
-    double run = 0.0;
+    if (flagged_only) {
+        // Not every element passed through this launch, so the skipped sums are taken from the other side: the squared
+        // sum of the whole tensor (left by the first launch, added once, by block 0) less the classes a slot did sweep.
+        double bs[CPT + 1];
 #pragma unroll
-    for (int b = 0; b < CPT; ++b) {
-        double v = sq[b];
-        block_sum2(v, zero, dscratch);
-        run += v;
-        dacc[b] += run;          // slot b skips classes 0..b
+        for (int b = 1; b <= CPT; ++b) {
+            bs[b] = sq[b];
+            block_sum2(bs[b], zero, dscratch);
+        }
+        double total = 0.0;
+        if (blockIdx.x == 0)
+            for (int i = 0; i < a.n_totals; ++i) total += __ldcg(a.block_totals + i);
+        double above = 0.0;
+#pragma unroll
+        for (int sl = CPT - 1; sl >= 0; --sl) {
+            above += bs[sl + 1];
+            dacc[sl] += total - above;   // slot sl sweeps the classes above sl
+        }
+    } else {
+        double run = 0.0;
+#pragma unroll
+        for (int b = 0; b < CPT; ++b) {
+            double v = sq[b];
+            block_sum2(v, zero, dscratch);
+            run += v;
+            dacc[b] += run;          // slot b skips classes 0..b
+        }
     }
     if (grp == 0) {
 #pragma unroll
@@ -432,6 +479,8 @@ __global__ void __launch_bounds__(256) tensor_sweep_fine_kernel(const TensorArgs
     const float4* x4 = reinterpret_cast<const float4*>(a.x);
     // |x| * thr_scale counts candidates; with a denormal step every value goes to all slots (Inf, or NaN for 0)
     const float thr_scale = g.tiny ? INFINITY : inv_thr;
+    const bool flagging = a.flag_role == 1 && a.tile_flags != nullptr;
+    const float flag_split = flagging ? a.flag_split : INFINITY;
     unsigned long long ev = 0ull;
     double sq_all = 0.0, sq1 = 0.0, sq2 = 0.0;       // squared sums: everything staged / first-slot-only / rest
 
@@ -474,18 +523,24 @@ __global__ void __launch_bounds__(256) tensor_sweep_fine_kernel(const TensorArgs
         // ---- three-way split: bit e of `first` / `rest` says where value e goes
         unsigned int first = 0u, rest = 0u;
         double tot = 0.0;                             // squared sum of everything this thread staged
+        bool far = false;                             // a value that reaches the second sweep launch
 #pragma unroll
         for (int e = 0; e < 16; ++e) {
             const float x = vals[e];
             const float r = fabsf(x) * thr_scale - cbase_f;        // NaN for non-finite values: they go to the rest
             const bool needed = !(r <= 1.0f);
             const bool wide = CPT > 1 && !(r <= 33.0f);             // slot 1 needs x iff r > 32 + 1
+            far |= !(r <= flag_split);
             first |= (needed && !wide ? 1u : 0u) << e;
             rest |= (wide ? 1u : 0u) << e;
             const double xd = (double)x;
             tot = fma(xd, xd, tot);
         }
         sq_all += tot;
+        if (flagging && __any_sync(0xffffffffu, far) && lane == 0) {
+            const long long ft = base4 / a.flag_tile4;             // this launch's tiles are the flag tiles
+            atomicOr(a.tile_flags + (ft >> 5), 1u << (ft & 31));
+        }
         __syncwarp();                                 // the warp is done sweeping its previous share
         if (!__any_sync(0xffffffffu, (first | rest) != 0u)) continue;
         // ---- the two lists, thread-major (lane 0's values first): offsets from a warp scan of the counts
@@ -550,6 +605,7 @@ __global__ void __launch_bounds__(256) tensor_sweep_fine_kernel(const TensorArgs
     block_sum2(sq_all, zero, dscratch);
     block_sum2(sq1, zero, dscratch);
     block_sum2(sq2, zero, dscratch);
+    if (flagging && tid == 0) a.block_totals[blockIdx.x] = sq_all;
     const double sq0 = fmax(sq_all - sq1 - sq2, 0.0);   // what no slot evaluated
     if (warp == 0) {
 #pragma unroll

@@ -64,7 +64,7 @@ struct omse_ctx {
     double* partials;    // device, kPartialBytes
     omse::RowTensor* d_tensors;   // device, OMSE_MAX_BATCH descriptors of a batched launch
     // per-context launch bookkeeping (a context is used by one host thread at a time, so no lock)
-    bool attr_rows[8], attr_tensor[4], attr_dual;   // opt-in shared-memory attribute set, per template instance
+    bool attr_rows[32], attr_tensor[4], attr_dual;   // opt-in shared-memory attribute set, per template instance
     LaunchShape seen[16];                           // blocks per SM of the row-kernel launch shapes met so far
     int n_seen, next_seen;
     int occ_sweep[2], occ_pass[3];                  // blocks per SM of the per-tensor kernels (0 = not yet asked)
@@ -118,11 +118,11 @@ void bounds(int bits, int is_signed, int* lo, int* hi) {
     }
 }
 
-template <int CPT, bool EXT>
+template <int CPT, bool EXT, int PATH>
 int launch_rows_t(omse_ctx* ctx, omse::RowArgs& a, size_t smem) {
-    const int slot = cpt_slot(CPT) + (EXT ? 4 : 0);
+    const int slot = cpt_slot(CPT) + (EXT ? 4 : 0) + 8 * (PATH == 7 ? 0 : PATH == 1 ? 1 : PATH == 2 ? 2 : 3);
     if (!ctx->attr_rows[slot]) {
-        if (cudaFuncSetAttribute(omse::rows_kernel<CPT, EXT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess)
+        if (cudaFuncSetAttribute(omse::rows_kernel<CPT, EXT, PATH>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess)
             return OMSE_ECUDA;
         ctx->attr_rows[slot] = true;
     }
@@ -132,7 +132,7 @@ int launch_rows_t(omse_ctx* ctx, omse::RowArgs& a, size_t smem) {
     for (int i = 0; i < ctx->n_seen; ++i)
         if (ctx->seen[i].cpt == slot && ctx->seen[i].threads == threads && ctx->seen[i].smem == smem) occ = ctx->seen[i].occ;
     if (occ == 0) {
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, omse::rows_kernel<CPT, EXT>, threads, smem) != cudaSuccess || occ < 1)
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, omse::rows_kernel<CPT, EXT, PATH>, threads, smem) != cudaSuccess || occ < 1)
             return OMSE_ECUDA;
         ctx->seen[ctx->next_seen] = LaunchShape{slot, threads, smem, occ};   // round robin once the table is full
         ctx->next_seen = (ctx->next_seen + 1) % 16;
@@ -140,12 +140,12 @@ int launch_rows_t(omse_ctx* ctx, omse::RowArgs& a, size_t smem) {
     }
     long long grid = (long long)ctx->n_sm * occ;
     if (grid > a.n_units) grid = a.n_units;
-    omse::rows_kernel<CPT, EXT><<<(unsigned)grid, threads, smem, ctx->stream>>>(a);
+    omse::rows_kernel<CPT, EXT, PATH><<<(unsigned)grid, threads, smem, ctx->stream>>>(a);
     return cudaGetLastError() == cudaSuccess ? OMSE_OK : OMSE_ECUDA;
 }
 
 // Launch shape for rows of at most max_k elements: threads per block, element groups, shared memory.
-int launch_rows(omse_ctx* ctx, omse::RowArgs& a, long long max_k, size_t smem_small = 0) {
+int launch_rows(omse_ctx* ctx, omse::RowArgs& a, long long max_k, size_t smem_small = 0, int path = 7) {
     const int cpt = cpt_for(a.n_cand);
     a.tg = (((a.n_cand + cpt - 1) / cpt) + 31) & ~31;
     const int k4 = (int)((max_k + 3) >> 2);
@@ -178,17 +178,22 @@ int launch_rows(omse_ctx* ctx, omse::RowArgs& a, long long max_k, size_t smem_sm
     else ext = ext || a.ext_tensors;
     if (ext) {
         switch (cpt) {
-            case 1: return launch_rows_t<1, true>(ctx, a, smem);
-            case 2: return launch_rows_t<2, true>(ctx, a, smem);
-            case 4: return launch_rows_t<4, true>(ctx, a, smem);
-            default: return launch_rows_t<8, true>(ctx, a, smem);
+            case 1: return launch_rows_t<1, true, 7>(ctx, a, smem);
+            case 2: return launch_rows_t<2, true, 7>(ctx, a, smem);
+            case 4: return launch_rows_t<4, true, 7>(ctx, a, smem);
+            default: return launch_rows_t<8, true, 7>(ctx, a, smem);
         }
     }
     switch (cpt) {
-        case 1: return launch_rows_t<1, false>(ctx, a, smem);
-        case 2: return launch_rows_t<2, false>(ctx, a, smem);
-        case 4: return launch_rows_t<4, false>(ctx, a, smem);
-        default: return launch_rows_t<8, false>(ctx, a, smem);
+        case 1: return launch_rows_t<1, false, 7>(ctx, a, smem);
+        case 2: return launch_rows_t<2, false, 7>(ctx, a, smem);
+        case 4: return launch_rows_t<4, false, 7>(ctx, a, smem);
+        default:
+            // single-path instantiations exist for the common case of eight candidates per thread
+            if (path == 1) return launch_rows_t<8, false, 1>(ctx, a, smem);
+            if (path == 2) return launch_rows_t<8, false, 2>(ctx, a, smem);
+            if (path == 4) return launch_rows_t<8, false, 4>(ctx, a, smem);
+            return launch_rows_t<8, false, 7>(ctx, a, smem);
     }
 }
 
@@ -407,40 +412,58 @@ int quantize_list(omse_ctx* ctx, std::vector<omse::RowTensor>& list, long long m
             }
         }
     }
-    // longest rows first: the dispenser then hands out work in decreasing size and the tail is short
+    // One launch per row path present in the list (block per row, batched short rows, thread per row): each launch
+    // then runs the kernel instantiation that holds only its path.  Longest rows first inside a launch: the dispenser
+    // hands out work in decreasing size and the tail is short.
     std::stable_sort(list.begin(), list.end(), [](const omse::RowTensor& x, const omse::RowTensor& y) { return x.K > y.K; });
-    long long units = 0;
-    for (auto& t : list) {
-        t.unit_begin = units;
-        units += (t.S + t.rows_per_unit - 1) / t.rows_per_unit;
+    size_t desc_used = 0;
+    for (int path = 1; path <= 4; path <<= 1) {
+        std::vector<omse::RowTensor> sub;
+        long long sub_max_k = 0;
+        for (const auto& t : list) {
+            const int p = (t.small & 4) ? 4 : t.small ? 2 : 1;
+            if (p != path) continue;
+            sub.push_back(t);
+            if (t.K > sub_max_k) sub_max_k = t.K;
+        }
+        if (sub.empty()) continue;
+        long long units = 0;
+        for (auto& t : sub) {
+            t.unit_begin = units;
+            units += (t.S + t.rows_per_unit - 1) / t.rows_per_unit;
+        }
+        omse::RowArgs a;
+        memset(&a, 0, sizeof(a));
+        a.n_launch_tensors = (int)sub.size();
+        a.n_units = units;
+        for (const auto& t : sub) a.ext_tensors |= (t.gate || t.prior_alpha) ? 1 : 0;
+        if (sub.size() == 1) {
+            a.tensors = nullptr;
+            a.one = sub[0];
+        } else {
+            omse::RowTensor* d_sub = ctx->d_tensors + desc_used;
+            if (cudaMemcpyAsync(d_sub, sub.data(), sizeof(omse::RowTensor) * sub.size(), cudaMemcpyHostToDevice,
+                                ctx->stream) != cudaSuccess)
+                return OMSE_ECUDA;
+            a.tensors = d_sub;
+            desc_used += sub.size();
+        }
+        a.n_cand = grid->n_cand;
+        a.hi_frac = grid->hi_frac;
+        a.refine_iters = grid->refine_iters;
+        a.n_tensors = 1;
+        a.n_sweeps = 1;
+        bounds(bits, is_signed, &a.lo[0], &a.hi[0]);
+        a.solver = mode.solver;
+        a.solver_iters = mode.solver_iters;
+        a.n_delta = mode.n_delta;
+        a.off_frac = mode.off_frac;
+        a.eps = -1.f;
+        a.keep_x0 = mode.n_delta > 0 ? 1 : 0;   // every offset is applied to the original row
+        const int rc = launch_rows(ctx, a, sub_max_k, path == 1 ? 0 : smem_small, path);
+        if (rc != OMSE_OK) return rc;
     }
-    omse::RowArgs a;
-    memset(&a, 0, sizeof(a));
-    a.n_launch_tensors = (int)list.size();
-    a.n_units = units;
-    for (const auto& t : list) a.ext_tensors |= (t.gate || t.prior_alpha) ? 1 : 0;
-    if (list.size() == 1) {
-        a.tensors = nullptr;
-        a.one = list[0];
-    } else {
-        if (cudaMemcpyAsync(ctx->d_tensors, list.data(), sizeof(omse::RowTensor) * list.size(), cudaMemcpyHostToDevice,
-                            ctx->stream) != cudaSuccess)
-            return OMSE_ECUDA;
-        a.tensors = ctx->d_tensors;
-    }
-    a.n_cand = grid->n_cand;
-    a.hi_frac = grid->hi_frac;
-    a.refine_iters = grid->refine_iters;
-    a.n_tensors = 1;
-    a.n_sweeps = 1;
-    bounds(bits, is_signed, &a.lo[0], &a.hi[0]);
-    a.solver = mode.solver;
-    a.solver_iters = mode.solver_iters;
-    a.n_delta = mode.n_delta;
-    a.off_frac = mode.off_frac;
-    a.eps = -1.f;
-    a.keep_x0 = mode.n_delta > 0 ? 1 : 0;   // every offset is applied to the original row
-    return launch_rows(ctx, a, max_k, smem_small);
+    return OMSE_OK;
 }
 
 }  // namespace

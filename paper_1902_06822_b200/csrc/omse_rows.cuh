@@ -542,7 +542,10 @@ __device__ double emit_block(const RowSmem& s, int k, float alpha, float flo, fl
 // EXT = false: the grid search with polish (and Algorithm 1 with a fixed number of sweeps) and nothing else, so that
 // the common launches keep their register allocation and code size; EXT = true adds the comparison solvers, the offset
 // search, Algorithm 1's loop condition, gated layers and rows that start from an earlier tensor's residual.
-template <int CPT, bool EXT>
+// PATH says which of the three row paths the instantiation contains (bit 0: block per row, bit 1: batched short rows,
+// bit 2: thread per row).  A launch whose tensors all take one path uses the instantiation with only that path: the
+// kernel is sensitive to its own code size (instruction cache), and code of a path no block runs still costs.
+template <int CPT, bool EXT, int PATH>
 __global__ void __launch_bounds__(OMSE_ROWS_MAX_THREADS) rows_kernel(const RowArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ unsigned long long s_unit;
@@ -580,14 +583,19 @@ __global__ void __launch_bounds__(OMSE_ROWS_MAX_THREADS) rows_kernel(const RowAr
         }
         const RowTensor& T = *tp;
         if (EXT && T.gate && *T.gate == 0) continue;   // not a key layer: nothing to do for this unit
-        if (T.small & 4) {
-            tiny_dispatch<CPT>(a, T, unit - T.unit_begin, smem_raw, st, ev);
-            continue;
+        if constexpr ((PATH & 4) != 0) {
+            if (T.small & 4) {
+                tiny_dispatch<CPT>(a, T, unit - T.unit_begin, smem_raw, st, ev);
+                continue;
+            }
         }
-        if (T.small) {
-            small_unit<CPT, EXT>(a, T, unit - T.unit_begin, smem_raw, rcp, st, ev);
-            continue;
+        if constexpr ((PATH & 2) != 0) {
+            if (T.small) {
+                small_unit<CPT, EXT>(a, T, unit - T.unit_begin, smem_raw, rcp, st, ev);
+                continue;
+            }
         }
+        if constexpr ((PATH & 1) == 0) continue;   // (the host never puts a block-per-row tensor into such a launch)
         const int k = (int)T.K;
         const int k4 = (k + 3) >> 2;
         const long long n_total = T.S * T.K;

@@ -700,7 +700,7 @@ static int alg1_impl(omse_ctx* ctx, const float* d_t, int64_t n_kernels, int64_t
     a.sse_history = d_sse_history;
     a.eps = eps;
     a.sweeps_done = d_sweeps_done;
-    return launch_rows(ctx, a, kernel_len);
+    return launch_rows(ctx, a, kernel_len, 0, /*path=*/1);   // Algorithm 1 always takes the block-per-row path
 }
 
 int omse_alg1_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, int64_t kernel_len, const int* bits,

@@ -33,9 +33,10 @@ N_CAND, BITS, REFINE, HI_FRAC = 1024, 4, 3, 1.0
 METRIC = "elements quantized/sec (4-bit MMSE search)"
 INSTR_PER_EVAL = 6            # reference FP32 sequence per (element, candidate): 3 fma + 2 min/max + 1 add
 LANE_OPS_PER_EVAL = 4         # FMA-pipe lane operations of an evaluation the kernels execute: fma, add, fma, fma
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the timed kernel from an ncu capture of the
-# default workload; None whenever the kernel has changed since the capture
-NCU_TRAFFIC_BYTES = 109_099_776
+# dram__bytes_read.sum + dram__bytes_write.sum of one step of the default workload (its two launches of the row kernel:
+# rows longer than 640 elements, then the shorter ones) from an ncu capture; None whenever the kernels have changed
+# since the capture
+NCU_TRAFFIC_BYTES = 106_615_808
 E2E_CHUNKS = 12               # batched launches per end-to-end step (copies of later chunks overlap earlier searches)
 N_SM, LANES_PER_SM = 148, 128
 WORKLOAD = "resnet50_weight_set_54_tensors_25.5M_params_signed4bit_kernelwise_1024cand_3refine_packed"
@@ -144,7 +145,6 @@ class Workload:
     n_cand = N_CAND
     evals_per_element = 1        # quantized tensors searched per element
     kernel = "rows_kernel<8>"
-    launches_per_step = 1
 
     def host_arrays(self):       # list of numpy inputs
         raise NotImplementedError
@@ -239,7 +239,6 @@ class WeightSet(Workload):
 
 class Activation(Workload):
     kernel = "tensor_sweep_kernel<8>"
-    launches_per_step = 10       # init, absmax, sweep, curve, finish, re-score, 3 polish, final
 
     def __init__(self, name, x, n_cand):
         self.name, self.x, self.n_cand = name, x, n_cand
@@ -481,9 +480,11 @@ def measure(wl, ctx, timer, steps, warmup):
     for _ in range(max(warmup, 3)):
         wl.step()
     timer.torch.cuda.synchronize()
-    ctx.omse_read_evaluations()                     # clear the instrumentation counter
+    ctx.omse_read_evaluations()                     # clear the instrumentation counters
+    ctx.omse_read_launches()
     ms = timer.run(wl.step, steps)
     executed = ctx.omse_read_evaluations() / steps
+    wl.launches_timed = ctx.omse_read_launches()    # kernels of this library launched inside the timed region
     return ms, executed
 
 
@@ -548,7 +549,7 @@ def run_ours(args, rank, world):
                                 "value": w2.n_total / (ms2 * 1e-3 / s2), "executed_share": r2["executed_share"],
                                 "frac": r2["frac"], "frac_fma_pipe": r2["frac_fma_pipe"], "frac_hbm": r2["frac_hbm"],
                                 "speed_vs_exhaustive": r2["speed_vs_exhaustive"], "kernel": w2.kernel,
-                                "gpu_launches": w2.launches_per_step * s2}
+                                "gpu_launches": w2.launches_timed}
             w2.release()
             del w2
             torch.cuda.empty_cache()
@@ -571,7 +572,7 @@ def run_ours(args, rank, world):
             "clocks": clocks,
             "e2e": {"value": whole_job_value(n_total, world, ms_e2e, args.steps), "unit": "elements/s",
                     "h2d_bytes_per_step": wl.h2d, "d2h_bytes_per_step": wl.d2h},
-            "gpu_launches": wl.launches_per_step * args.steps,
+            "gpu_launches": wl.launches_timed,
             "roofline": roof,
         }
         if sustained is not None:

@@ -387,6 +387,11 @@ int omse_last_device_status(omse_ctx* ctx, uint32_t* host_out);
  * omse_dual_quantize the unit is (element, pair, first code).  omse_activation_scale_static does not count. */
 int omse_read_evaluations(omse_ctx* ctx, uint64_t* host_out);
 
+/* Instrumentation (no counterpart in the paper): the number of kernels the calls on this context have launched since
+ * the last read (host-side count, no synchronisation), then cleared.  A batched weight call launches one kernel per
+ * row path present (rows longer than 640 elements, shorter rows, very short rows), the per-tensor search ten or so. */
+int omse_read_launches(omse_ctx* ctx, uint64_t* host_out);
+
 /* Instrumentation (no counterpart in the paper): runs a register-only loop of independent fma.rn.f32x2 on every SM
  * for about target_ms milliseconds (1..5000) on the context's stream, synchronises, and returns in *host_out the
  * measured FP32 lane operations per second of the FMA pipe (a packed instruction counts as two).  This is the

@@ -26,7 +26,7 @@ EXPORTS = [
     "omse_activation_scale", "omse_residual_quantize", "omse_pack_int4", "omse_last_device_status",
     "omse_status_string", "omse_activation_scale_static", "omse_alg1_quantize_converge",
     "omse_quantize_weights_solver", "omse_quantize_weights_affine", "omse_quantize_key_layers",
-    "omse_measure_fp32_peak",
+    "omse_measure_fp32_peak", "omse_read_launches",
 ]
 SOLVER_GRID, SOLVER_UNIFORM, SOLVER_ALTERNATING, SOLVER_GOLDEN = 0, 1, 2, 3
 MAX_OFFSETS = 64
@@ -107,6 +107,7 @@ def load_library() -> C.CDLL:
     lib.omse_last_device_status.argtypes = [vp, C.POINTER(C.c_uint32)]
     lib.omse_read_evaluations.argtypes = [vp, C.POINTER(C.c_uint64)]
     lib.omse_measure_fp32_peak.argtypes = [vp, i32, C.POINTER(C.c_double)]
+    lib.omse_read_launches.argtypes = [vp, C.POINTER(C.c_uint64)]
     lib.omse_status_string.argtypes = [i32]
     lib.omse_status_string.restype = C.c_char_p
     _lib = lib
@@ -358,6 +359,14 @@ class Context:
         rc = load_library().omse_read_evaluations(self._h, C.byref(out))
         if rc != OK:
             raise OmseError(rc, "omse_read_evaluations")
+        return out.value
+
+    def omse_read_launches(self) -> int:
+        """Kernels launched by this context's calls since the last read."""
+        out = C.c_uint64(0)
+        rc = load_library().omse_read_launches(self._h, C.byref(out))
+        if rc != OK:
+            raise OmseError(rc, "omse_read_launches")
         return out.value
 
     def omse_measure_fp32_peak(self, target_ms: int = 200) -> float:

@@ -68,6 +68,7 @@ struct omse_ctx {
     LaunchShape seen[16];                           // blocks per SM of the row-kernel launch shapes met so far
     int n_seen, next_seen;
     int occ_sweep[2], occ_pass[3];                  // blocks per SM of the per-tensor kernels (0 = not yet asked)
+    unsigned long long n_launches;                  // kernels launched since the last omse_read_launches
 };
 
 namespace {
@@ -141,6 +142,7 @@ int launch_rows_t(omse_ctx* ctx, omse::RowArgs& a, size_t smem) {
     long long grid = (long long)ctx->n_sm * occ;
     if (grid > a.n_units) grid = a.n_units;
     omse::rows_kernel<CPT, EXT, PATH><<<(unsigned)grid, threads, smem, ctx->stream>>>(a);
+    ++ctx->n_launches;
     return cudaGetLastError() == cudaSuccess ? OMSE_OK : OMSE_ECUDA;
 }
 
@@ -236,6 +238,7 @@ struct TensorEnv {
     int* occ_pass;       // [3] blocks per SM of the three pass kernels
     bool opt_in_smem;    // the sweep may ask for more than 48 KB of dynamic shared memory (context path only)
     bool* attr_tensor;   // [4] per CPT: opt-in attribute already set
+    unsigned long long* launches;   // launch counter of the caller
 };
 
 template <int CPT, bool FINE>
@@ -257,6 +260,7 @@ int sweep_launch_t(const TensorEnv& env, omse::TensorArgs& a, size_t smem, int* 
     if (grid < 1) grid = 1;
     *n_blocks = (int)grid;
     kernel<<<(unsigned)grid, threads, smem, env.stream>>>(a);
+    ++*env.launches;
     return cudaGetLastError() == cudaSuccess ? OMSE_OK : OMSE_ECUDA;
 }
 
@@ -317,7 +321,11 @@ int enqueue_tensor_search(const TensorEnv& env, omse::TensorArgs& a, int refine_
         const int flag_words = flags ? (int)((n_flag_tiles + 31) >> 5) : 0;
         omse::tensor_absmax_kernel<<<(unsigned)absmax_grid, 256, 0, s>>>(a.x, n, a.st, a.status,
                                                                       reinterpret_cast<unsigned int*>(a.curve), flag_words);
-        if (a.delta_out) omse::tensor_offset_kernel<<<1, 32, 0, s>>>(a.st);
+        ++*env.launches;
+        if (a.delta_out) {
+            omse::tensor_offset_kernel<<<1, 32, 0, s>>>(a.st);
+            ++*env.launches;
+        }
         int rc;
         if (!two) {
             rc = sweep_launch(env, a, 0, a.n_cand, cpt_for(a.n_cand), &nb_lo);
@@ -340,6 +348,7 @@ int enqueue_tensor_search(const TensorEnv& env, omse::TensorArgs& a, int refine_
             omse::TensorArgs hi = a;
             if (flags) {
                 hi.tile_flags = lo.tile_flags;
+                hi.flag_words = flag_words;
                 hi.flag_tile4 = lo.flag_tile4;
                 hi.flag_role = 2;
                 hi.block_totals = lo.block_totals;
@@ -355,6 +364,7 @@ int enqueue_tensor_search(const TensorEnv& env, omse::TensorArgs& a, int refine_
     const int g1 = pass_grid<1>(env, n);
     for (int it = 0; it < refine_iters; ++it) omse::tensor_pass_kernel<1><<<(unsigned)g1, 256, 0, s>>>(a);
     omse::tensor_pass_kernel<2><<<(unsigned)pass_grid<2>(env, n), 256, 0, s>>>(a);
+    *env.launches += 4 + (unsigned long long)refine_iters;   // curve, finish, re-score, polish steps, final
     return cudaGetLastError() == cudaSuccess ? OMSE_OK : OMSE_ECUDA;
 }
 
@@ -556,6 +566,13 @@ int omse_last_device_status(omse_ctx* ctx, uint32_t* host_out) {
         return OMSE_ECUDA;
     if (cudaMemsetAsync(&ctx->ws->status, 0, sizeof(uint32_t), ctx->stream) != cudaSuccess) return OMSE_ECUDA;
     return cudaStreamSynchronize(ctx->stream) == cudaSuccess ? OMSE_OK : OMSE_ECUDA;
+}
+
+int omse_read_launches(omse_ctx* ctx, uint64_t* host_out) {
+    if (!ctx || !host_out) return OMSE_EINVAL;
+    *host_out = ctx->n_launches;
+    ctx->n_launches = 0;
+    return OMSE_OK;
 }
 
 int omse_read_evaluations(omse_ctx* ctx, uint64_t* host_out) {
@@ -815,6 +832,7 @@ int omse_quantize_key_layers(omse_ctx* ctx, const omse_key_layer* layers, int n_
                             ctx->stream) != cudaSuccess)
             return OMSE_ECUDA;
         omse::compression_ratio_kernel<<<1, 32, 0, ctx->stream>>>(d_layers, n_layers, bits, d_is_key, d_cr);
+        ++ctx->n_launches;
         if (cudaGetLastError() != cudaSuccess) return OMSE_ECUDA;
     }
     return OMSE_OK;
@@ -871,6 +889,7 @@ int omse_dual_quantize(omse_ctx* ctx, const float* d_t, int64_t n_kernels, int64
     a.curve = reinterpret_cast<float*>(ctx->partials);
     a.evals = &ctx->ws->evals;
     omse::dual_kernel<<<(unsigned)blocks, omse::kDualThreads, smem, ctx->stream>>>(a);
+    ++ctx->n_launches;
     return cudaGetLastError() == cudaSuccess ? OMSE_OK : OMSE_ECUDA;
 }
 
@@ -896,6 +915,7 @@ int omse_select_key_layers(omse_ctx* ctx, const omse_layer_error* layers, int n_
                         ctx->stream) != cudaSuccess)
         return OMSE_ECUDA;
     omse::layer_mse_kernel<<<(unsigned)n_layers, 256, 0, ctx->stream>>>(d_layers, tau, d_mse, d_is_key);
+    ++ctx->n_launches;
     return cudaGetLastError() == cudaSuccess ? OMSE_OK : OMSE_ECUDA;
 }
 
@@ -956,7 +976,8 @@ static int activation_impl(omse_ctx* ctx, const float* d_x, int64_t n, int bits,
     a.evals = &ctx->ws->evals;
     a.status = &ctx->ws->status;
     omse::tensor_init_kernel<<<1, 32, 0, ctx->stream>>>(a.st);
-    const TensorEnv env = {ctx->n_sm, ctx->stream, ctx->occ_sweep, ctx->occ_pass, true, ctx->attr_tensor};
+    ++ctx->n_launches;
+    const TensorEnv env = {ctx->n_sm, ctx->stream, ctx->occ_sweep, ctx->occ_pass, true, ctx->attr_tensor, &ctx->n_launches};
     return enqueue_tensor_search(env, a, grid->refine_iters);
 }
 
@@ -973,6 +994,7 @@ int omse_pack_int4(omse_ctx* ctx, const int8_t* d_codes, int64_t n, int is_signe
     if (grid > (long long)ctx->n_sm * 16) grid = (long long)ctx->n_sm * 16;
     if (grid < 1) grid = 1;
     omse::pack_int4_kernel<<<(unsigned)grid, 256, 0, ctx->stream>>>(reinterpret_cast<const signed char*>(d_codes), n, d_packed);
+    ++ctx->n_launches;
     return cudaGetLastError() == cudaSuccess ? OMSE_OK : OMSE_ECUDA;
 }
 
@@ -1082,7 +1104,8 @@ extern "C" int omse_activation_scale_static(int device, void* cuda_stream, const
 
     static_begin_kernel<<<1, 32, 0, s>>>(sc);
     // the sweep stays below 48 KB of dynamic shared memory, so no attribute call is needed here
-    const TensorEnv env = {sd.n_sm, s, sd.occ_sweep, sd.occ_pass, false, sd.attr_unused};
+    unsigned long long not_counted = 0;
+    const TensorEnv env = {sd.n_sm, s, sd.occ_sweep, sd.occ_pass, false, sd.attr_unused, &not_counted};
     const int rc = enqueue_tensor_search(env, a, grid->refine_iters);
     if (rc != OMSE_OK) return rc;
     static_end_kernel<<<1, 32, 0, s>>>(sc, d_status);

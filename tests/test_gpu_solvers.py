@@ -230,3 +230,24 @@ def test_key_layer_procedure_in_one_call_matches_oracle(packed):
             else:
                 assert torch.all(d["codes2"] == 77)
     assert gpu_util.ctx().omse_last_device_status() == 0
+
+
+def test_launch_counter_counts_one_launch_per_row_path():
+    """A batched weight call is issued as one launch per row path present; the counter is what bench.py reports."""
+    import torch
+    import gpu_util
+    ctx = gpu_util.ctx()
+    ctx.omse_read_launches()
+    shapes = [(3000, 64), (2500, 576), (40, 2304), (16, 4608)]            # short rows in numbers + long rows
+    descs = [dict(w=torch.from_numpy(synth.laplace(s * k, 0.05, seed=5, tensor_id=i).reshape(s, k)).cuda(), n_kernels=s,
+                  kernel_len=k, alpha=torch.empty(s, device="cuda"), sse=torch.empty(s, device="cuda"))
+             for i, (s, k) in enumerate(shapes)]
+    ctx.omse_quantize_weights_batched(descs, 4, True, 1024, 1.0, 3)
+    assert ctx.omse_read_launches() == 2
+    ctx.omse_quantize_weights_batched(descs[2:], 4, True, 1024, 1.0, 3)
+    assert ctx.omse_read_launches() == 1 and ctx.omse_read_launches() == 0
+    x = torch.from_numpy(synth.relu_activations(100_000, seed=3)).cuda()
+    a, e = torch.empty(1, device="cuda"), torch.empty(1, device="cuda")
+    ctx.omse_activation_scale(x, x.numel(), 4, False, 2048, 1.0, 3, a, e)
+    assert ctx.omse_read_launches() == 11          # init, maxima, two sweeps, curve, argmin, re-score, 3 polish steps, final
+    torch.cuda.synchronize()

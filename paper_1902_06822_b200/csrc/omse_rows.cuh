@@ -102,10 +102,17 @@ __device__ __forceinline__ double exact_sse_block(const float* xs, int k, float 
     long long zero = 0;
     const float inv = __fdiv_rn(1.0f, alpha), thr = ambiguity_threshold(flo, fhi);
     const double ad = (double)alpha;
-    for (int i = threadIdx.x; i < k; i += blockDim.x) {
-        const float x = xs[i];
-        const double d = fma(-ad, int_double(exact_code(x, alpha, inv, flo, fhi, thr)), (double)x);
-        ss = fma(d, d, ss);
+    // four elements per step (the row is zero padded to a multiple of four; a zero has code 0 and error 0)
+    const float4* xs4 = reinterpret_cast<const float4*>(xs);
+    const int k4 = (k + 3) >> 2;
+    for (int i4 = threadIdx.x; i4 < k4; i4 += blockDim.x) {
+        const float4 v = xs4[i4];
+        const float x[4] = {v.x, v.y, v.z, v.w};
+        double d[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) d[e] = fma(-ad, int_double(exact_code(x[e], alpha, inv, flo, fhi, thr)), (double)x[e]);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) ss = fma(d[e], d[e], ss);
     }
     block_sum2(ss, zero, scratch);
     return ss;
@@ -114,15 +121,25 @@ __device__ __forceinline__ double exact_sse_block(const float* xs, int k, float 
 // Least-squares polish of Section 3.4's objective: alpha <- <x,q>/<q,q>, q = [x/alpha]_Zp, at most n times.
 __device__ __forceinline__ float polish_block(const float* xs, int k, float alpha, float flo, float fhi, int n,
                                               double* scratch) {
+    const float4* xs4 = reinterpret_cast<const float4*>(xs);
+    const int k4 = (k + 3) >> 2;
     for (int it = 0; it < n; ++it) {
         double sxq = 0.0;
         long long sqq = 0;
         const float inv = __fdiv_rn(1.0f, alpha), thr = ambiguity_threshold(flo, fhi);
-        for (int i = threadIdx.x; i < k; i += blockDim.x) {
-            const float x = xs[i];
-            const int q = exact_code(x, alpha, inv, flo, fhi, thr);
-            sqq += q * q;
-            sxq = fma((double)x, int_double(q), sxq);
+        for (int i4 = threadIdx.x; i4 < k4; i4 += blockDim.x) {   // four elements per step; the zero padding adds nothing
+            const float4 v = xs4[i4];
+            const float x[4] = {v.x, v.y, v.z, v.w};
+            int q[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) q[e] = exact_code(x[e], alpha, inv, flo, fhi, thr);
+            int qq = 0;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                qq += q[e] * q[e];
+                sxq = fma((double)x[e], int_double(q[e]), sxq);
+            }
+            sqq += qq;
         }
         block_sum2(sxq, sqq, scratch);
         if (sqq == 0) break;
@@ -160,18 +177,26 @@ __device__ void partition_row(const RowSmem& s, int k, const GridSetup& g, int t
     const int tid = threadIdx.x, nthr = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarp = nthr >> 5;
     const float inv_thr = g.rstep * (1.0f / 0.4999f);
     const float inv_tg = 1.0f / (float)tg;
-    // Thread t owns the elements t, t + nthr, ... (conflict-free reads); within a class the elements keep the
-    // order (thread, then index), which is fixed, so the sums that follow do not depend on scheduling.
+    // Thread t owns the float4s t, t + nthr, ... of the zero-padded row (conflict-free 128-bit reads, four independent
+    // elements per step); within a class the elements keep the order (thread, then index), which is fixed, so the
+    // sums that follow do not depend on scheduling.  The padding zeros fall into class 0 and add nothing.
     // ---- pass 1: class counts of this thread's elements (16-bit fields), squared sum of class 0
+    const float4* xs4 = reinterpret_cast<const float4*>(s.xs);
+    const int k4 = (k + 3) >> 2;
     u64 c0 = 0ull, c1 = 0ull;                  // classes 1..4 and 5..8
     double zero_sq = 0.0;
-    for (int i = tid; i < k; i += nthr) {
-        const float x = s.xs[i];
-        const int nb = magnitude_class<CPT>(x, inv_thr, inv_tg);
-        const double xd = (double)x;
-        zero_sq = fma(nb == 0 ? xd : 0.0, xd, zero_sq);
-        if (nb >= 5) c1 += 1ull << (16 * (nb - 5));
-        else if (nb >= 1) c0 += 1ull << (16 * (nb - 1));
+    for (int i4 = tid; i4 < k4; i4 += nthr) {
+        const float4 v = xs4[i4];
+        const float x[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int nb = magnitude_class<CPT>(x[e], inv_thr, inv_tg);
+            const double xd = (double)x[e];
+            zero_sq = fma(nb == 0 ? xd : 0.0, xd, zero_sq);
+            const u64 one = nb >= 1 ? 1ull << (16 * ((nb - 1) & 3)) : 0ull;
+            c0 += nb < 5 ? one : 0ull;
+            c1 += nb >= 5 ? one : 0ull;
+        }
     }
     // ---- exclusive scan of the counts over the block (lanes by shuffle, warps in order)
     u64 i0 = c0, i1 = c1;
@@ -201,13 +226,17 @@ __device__ void partition_row(const RowSmem& s, int k, const GridSetup& g, int t
         tot0 += a0;
         tot1 += a1;
     }
-    // ---- class layout in xb: class CPT first, each class padded with zeros to a multiple of 4
+    // ---- class layout in xb: class CPT first, each class padded with zeros to a multiple of 4.  The class starts are
+    //      added to the packed offsets, which then hold positions in xb (a regrouped row has fewer than 2^16 elements).
     int base[CPT + 1], cnt[CPT + 1];
     int pos = 0;
+    u64 b0 = 0ull, b1 = 0ull;
 #pragma unroll
     for (int b = CPT; b >= 1; --b) {
         cnt[b] = (int)(((b >= 5 ? tot1 : tot0) >> (16 * ((b - 1) & 3))) & 0xffffull);
         base[b] = pos;
+        if (b >= 5) b1 |= (u64)pos << (16 * ((b - 1) & 3));
+        else b0 |= (u64)pos << (16 * ((b - 1) & 3));
         const int padded = (cnt[b] + 3) & ~3;
         if (tid == 0) {
             s.seg[2 * b] = pos;
@@ -216,36 +245,43 @@ __device__ void partition_row(const RowSmem& s, int k, const GridSetup& g, int t
         if (tid < padded - cnt[b]) s.xb[pos + cnt[b] + tid] = 0.f;
         pos += padded;
     }
+    off0 += b0;
+    off1 += b1;
     // ---- pass 2: scatter
-    for (int i = tid; i < k; i += nthr) {
-        const float x = s.xs[i];
-        const int nb = magnitude_class<CPT>(x, inv_thr, inv_tg);
-        if (nb >= 1) {
-            const int sh = 16 * ((nb - 1) & 3);
-            int within;
-            if (nb >= 5) {
-                within = (int)((off1 >> sh) & 0xffffull);
-                off1 += 1ull << sh;
-            } else {
-                within = (int)((off0 >> sh) & 0xffffull);
-                off0 += 1ull << sh;
-            }
-            int bs = 0;
+    for (int i4 = tid; i4 < k4; i4 += nthr) {
+        const float4 v = xs4[i4];
+        const float x[4] = {v.x, v.y, v.z, v.w};
+        int nb[4];
 #pragma unroll
-            for (int b = 1; b <= CPT; ++b) bs = (nb == b) ? base[b] : bs;
-            s.xb[bs + within] = x;
+        for (int e = 0; e < 4; ++e) nb[e] = magnitude_class<CPT>(x[e], inv_thr, inv_tg);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            if (nb[e] >= 1) {
+                const int sh = 16 * ((nb[e] - 1) & 3);
+                const u64 word = nb[e] >= 5 ? off1 : off0;
+                const u64 one = 1ull << sh;
+                s.xb[(int)((word >> sh) & 0xffffull)] = x[e];
+                off0 += nb[e] >= 5 ? 0ull : one;
+                off1 += nb[e] >= 5 ? one : 0ull;
+            }
         }
     }
     __syncthreads();
-    // ---- squared sums per class from the regrouped row (class 0 was summed on the way)
+    // ---- squared sums per class from the regrouped row (class 0 was summed on the way; padding zeros add nothing)
+    const float4* xb4 = reinterpret_cast<const float4*>(s.xb);
     double d[CPT + 1];
     d[0] = zero_sq;
 #pragma unroll
     for (int b = 1; b <= CPT; ++b) {
         double v = 0.0;
-        for (int i = tid; i < cnt[b]; i += nthr) {
-            const double xd = (double)s.xb[base[b] + i];
-            v = fma(xd, xd, v);
+        const int first4 = base[b] >> 2, len4 = (cnt[b] + 3) >> 2;
+        for (int i4 = tid; i4 < len4; i4 += nthr) {
+            const float4 q = xb4[first4 + i4];
+            const double q0 = (double)q.x, q1 = (double)q.y, q2 = (double)q.z, q3 = (double)q.w;
+            v = fma(q0, q0, v);
+            v = fma(q1, q1, v);
+            v = fma(q2, q2, v);
+            v = fma(q3, q3, v);
         }
         d[b] = v;
     }
@@ -276,11 +312,15 @@ __device__ PhiOut phi_block(const RowArgs& a, const RowSmem& s, int k, int k4, f
 
     // ---- max of the positive and of the negative part (range of the grid; which candidates saturate)
     float mpos = 0.f, mneg = 0.f;
-    for (int i = tid; i < k; i += nthr) {
-        const float v = s.xs[i];
-        if (fabsf(v) <= FLT_MAX) {
-            mpos = fmaxf(mpos, v);
-            mneg = fmaxf(mneg, -v);
+    for (int i4 = tid; i4 < k4; i4 += nthr) {   // the zero padding leaves both maxima alone
+        const float4 v4 = xs4[i4];
+        const float x[4] = {v4.x, v4.y, v4.z, v4.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            if (fabsf(x[e]) <= FLT_MAX) {
+                mpos = fmaxf(mpos, x[e]);
+                mneg = fmaxf(mneg, -x[e]);
+            }
         }
     }
     block_max2(mpos, mneg, s.scratch);
@@ -444,10 +484,14 @@ __device__ PhiOut phi_block(const RowArgs& a, const RowSmem& s, int k, int k4, f
             long long zero = 0;
             const float inv = __fdiv_rn(1.0f, ac), thr = ambiguity_threshold(flo, fhi);
             const double ad = (double)ac;
-            for (int i = tid; i < k; i += nthr) {
-                const float x = s.xs[i];
-                const double d = fma(-ad, int_double(exact_code(x, ac, inv, flo, fhi, thr)), (double)x);
-                ss = fma(d, d, ss);
+            for (int i4 = tid; i4 < k4; i4 += nthr) {
+                const float4 v4 = xs4[i4];
+                const float x[4] = {v4.x, v4.y, v4.z, v4.w};
+                double d[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) d[e] = fma(-ad, int_double(exact_code(x[e], ac, inv, flo, fhi, thr)), (double)x[e]);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) ss = fma(d[e], d[e], ss);
             }
             block_sum2(ss, zero, s.scratch);
             if (ss < best_sse) {   // increasing index: strict < keeps the lowest among equal errors

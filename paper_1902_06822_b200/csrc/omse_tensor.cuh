@@ -467,9 +467,13 @@ __global__ void __launch_bounds__(256) tensor_sweep_fine_kernel(const TensorArgs
         na2[sl] = pack2(-ac, -ac);
         dacc[sl] = 0.0;
     }
-    // candidates that may saturate: on first-slot-only elements (bounded above) and on the rest (the tensor's own count)
-    int ncl_first = (class_sat_count(1, CPT, 32, g.c_sat, flo, fhi, a.c_base) - a.c_base + 31) / 32;
-    ncl_first = max(0, min(1, ncl_first));
+    // Saturation.  The first-slot-only list holds no value that any candidate of the launch could saturate (such values
+    // go to the rest), so its sweep needs no clamps at all: x*inv_c stays below hi + 1/2 (above lo - 1/2) for every
+    // c >= c_base once |x| is below the bound of its sign; 1e-5 covers the rounding of inv_c and alpha_c.  A negative
+    // value on a grid that starts at 0 is coded 0 by every scale: it is dropped whatever its size.
+    const float a_first = __fmul_rn((float)(a.c_base + 1), g.step);
+    const float pos_bound = (fhi + 0.5f) * a_first * 0.99999f, neg_bound = (0.5f - flo) * a_first * 0.99999f;
+    const bool neg_free = flo == 0.f;
     int ncl_rest = (g.c_sat - a.c_base + 31) / 32;
     ncl_rest = max(0, min(CPT, ncl_rest));
 
@@ -528,8 +532,9 @@ __global__ void __launch_bounds__(256) tensor_sweep_fine_kernel(const TensorArgs
         for (int e = 0; e < 16; ++e) {
             const float x = vals[e];
             const float r = fabsf(x) * thr_scale - cbase_f;        // NaN for non-finite values: they go to the rest
-            const bool needed = !(r <= 1.0f);
-            const bool wide = CPT > 1 && !(r <= 33.0f);             // slot 1 needs x iff r > 32 + 1
+            const bool needed = !(r <= 1.0f) && !(neg_free && x < 0.f);
+            const bool may_sat = !(fabsf(x) < (x < 0.f ? neg_bound : pos_bound));
+            const bool wide = needed && ((CPT > 1 && !(r <= 33.0f)) || may_sat);   // slot 1 needs x iff r > 32 + 1
             far |= !(r <= flag_split);
             first |= (needed && !wide ? 1u : 0u) << e;
             rest |= (wide ? 1u : 0u) << e;
@@ -580,10 +585,10 @@ __global__ void __launch_bounds__(256) tensor_sweep_fine_kernel(const TensorArgs
         }
         const float4* reg4 = reinterpret_cast<const float4*>(reg);
         if (n1 > 0) {
-            sweep_ncl<CPT, 1>(ncl_first, reg4, 0, n1p >> 2, inv2, na2, dacc, kMagic + flo, kMagic + fhi);
+            sweep_range<CPT, 1, 0>(reg4, 0, n1p >> 2, inv2, na2, dacc, kMagic + flo, kMagic + fhi);
             ev += (unsigned long long)n1p;
         }
-        if (CPT > 1 && n2 > 0) {
+        if (n2 > 0) {
             sweep_ncl<CPT, CPT>(ncl_rest, reg4, (region - n2p) >> 2, region >> 2, inv2, na2, dacc, kMagic + flo, kMagic + fhi);
             ev += (unsigned long long)n2p * CPT;
         }

@@ -165,6 +165,17 @@ def test_activation_scale_grids(gpu, bits, signed, n_cand):
     _check_activation(gpu, x, bits, signed, n_cand, 2)
 
 
+@pytest.mark.parametrize("neg_outlier", [False, True])
+def test_activation_scale_unsigned_grid_on_signed_values(gpu, neg_outlier):
+    """A grid that starts at 0 codes every negative value as 0 whatever the scale; values at the edge of the range of
+    the smallest scales saturate.  With the outlier the negative side sets the grid's range."""
+    x = synth.student_t3(300_001, seed=41, tensor_id=7)
+    if neg_outlier:
+        x[1234] = np.float32(-3.0) * np.abs(x).max()
+    _check_activation(gpu, x, 4, False, 2048, 3)
+    _check_activation(gpu, x, 3, False, 256, 1)
+
+
 def test_activation_scale_degenerate(gpu):
     gpu.ctx().omse_last_device_status()
     alpha, sse, idx, curve = gpu.activation_scale(np.zeros(5000, np.float32), 4, False, 128, 1.0, 3)

@@ -111,7 +111,9 @@ __global__ void __launch_bounds__(kDualThreads) dual_kernel(const DualArgs a) {
             float* curve = a.curve + (size_t)blockIdx.x * n_pairs_grid;
             if (!degenerate) {
                 for (int slot = tid; slot < n_slots; slot += nthr) {
-                    const int c = slot / dgroups, d0 = (slot - c * dgroups) * kDualDpt;
+                    // consecutive threads take consecutive alpha1 of one group of alpha2's: the window of first codes
+                    // depends on alpha2/alpha1 = (d+1)*hi_frac2/C2 only, so a warp's lanes run the same number of steps
+                    const int dg = slot / a.n_cand1, c = slot - dg * a.n_cand1, d0 = dg * kDualDpt;
                     float a1, a2[kDualDpt], inv2[kDualDpt], acc[kDualDpt];
                     double dacc[kDualDpt];
                     bool ok[kDualDpt];

@@ -5,9 +5,13 @@
 // One thread block owns one kernel (row) in shared memory.  Pairs are spread over threads: a thread
 // holds one alpha1 and DPT consecutive alpha2 in registers, so x - alpha1*t is formed once per t and
 // shared by its alpha2's; elements are broadcast from shared memory.  The enumeration over t is
-// restricted, exactly, to a window around round(x/alpha1): a t further away than
-// (max|Z_p2| + 1/2)*alpha2/alpha1 + 3/2 leaves a rest that saturates the second code and loses to the
-// nearest t by more than alpha2/2.  Grid values are compared in fp32 (blocks of 64 elements folded
+// restricted, exactly, to a window around round(x/alpha1).  A first code whose rest saturates the second
+// code errs by more than alpha2/2, one whose rest does not by at most alpha2/2, and the latter all lie
+// within (max|Z_p2| + 1/2)*alpha2/alpha1 of x/alpha1; when every rest saturates, the error grows with
+// the distance from x/alpha1 up to the asymmetry of Z_p2, which can only move the winner to the other
+// neighbour of x/alpha1.  So the codes within (max|Z_p2| + 1/2)*alpha2/alpha1 + 1/2 of round(x/alpha1),
+// and at least the two neighbours, hold the minimum (codes beyond Z_p1 collapse onto its ends).
+// Grid values are compared in fp32 (blocks of 64 elements folded
 // into fp64); pairs within the fp32 noise band of the minimum are re-scored with the full
 // enumeration in the reference arithmetic, and the final codes always use the full enumeration.
 #pragma once
@@ -126,9 +130,9 @@ __global__ void __launch_bounds__(kDualThreads) dual_kernel(const DualArgs a) {
                         dacc[j] = 0.0;
                     }
                     const float inv1 = a1 >= FLT_MIN ? __fdiv_rn(1.0f, a1) : 0.f;
-                    // window of first codes that can win: |t - x/alpha1| <= half_range2*alpha2/alpha1 + 3/2
+                    // window of first codes that can win: |t - round(x/alpha1)| <= half_range2*alpha2/alpha1 + 1/2, at least 1
                     const float ratio = a2[kDualDpt - 1] * inv1;         // largest alpha2 of the group
-                    const int w = (int)(half_range2 * fminf(ratio, 16.f) * 1.0001f) + 2;
+                    const int w = max(1, (int)(half_range2 * fminf(ratio, 16.f) * 1.0001f + 0.501f));
                     const bool full = !(ratio <= 16.f) || 2 * w + 1 >= n_levels;
                     const int n_t = full ? n_levels : 2 * w + 1;
                     ev += (unsigned long long)k * (unsigned long long)(2 * ((n_t + 1) / 2)) * kDualDpt;

@@ -62,6 +62,19 @@ def test_dual_bit_widths_signedness_and_second_grid_range(gpu, bits1, bits2, sig
     _check(gpu, t, bits1, bits2, signed, c1=9, c2=7, hf2=hf2, packed=bits1 <= 4 and bits2 <= 4)
 
 
+@pytest.mark.parametrize("hf2", [0.03, 0.06, 0.12, 0.5, 1.0, 2.5])
+def test_dual_first_code_window_over_second_grid_ranges(gpu, hf2):
+    """The enumeration over first codes is cut to a window whose width follows alpha2/alpha1: from second grids so
+    narrow that every rest saturates (the asymmetry of Z_p2 then decides between the two neighbours) to ones wider
+    than a step of the first grid.  Evenly spread values reach every position between two first codes."""
+    rng = np.random.default_rng(640)
+    t = rng.uniform(-1.0, 1.0, size=(6, 384)).astype(np.float32)
+    t[3] = np.abs(t[3])
+    t[4] *= np.float32(1e-3)
+    _check(gpu, t, c1=32, c2=32, hf2=hf2)
+    _check(gpu, t, bits1=3, bits2=4, c1=8, c2=16, hf2=hf2)
+
+
 @pytest.mark.parametrize("c1,c2", [(1, 1), (1, 33), (40, 3), (64, 64)])
 def test_dual_grid_shapes(gpu, c1, c2):
     t = synth.laplace(5 * 96, 0.02, seed=620, tensor_id=c1).reshape(5, 96)

@@ -628,3 +628,34 @@ def test_key_layer_pipeline_marks_by_tau_and_counts_the_second_tensor():
     s = [w.shape[0] for w in layers]
     want = sum((2 if i == l else 1) * (4 * n[i] + 32 * s[i]) for i in range(3)) / (32.0 * sum(n))
     assert out.compression_ratio == pytest.approx(want, rel=1e-12)
+
+
+@pytest.mark.parametrize("lo1,hi1,lo2,hi2", [(-8, 7, -8, 7), (-4, 3, -8, 7), (0, 15, 0, 15), (-2, 1, -128, 127), (-8, 7, -2, 1)])
+def test_dual_first_code_window_holds_the_minimum(lo1, hi1, lo2, hi2):
+    """Section 3.5's dual objective min_t (x - a1*t - a2*[(x - a1*t)/a2]_Zp2)^2, enumerated over every first code,
+    equals the minimum over the first codes within (max|Z_p2| + 1/2)*a2/a1 + 1/2 (at least 1) of round(x/a1), with
+    codes beyond Z_p1 moved to its ends: the property the library's restricted enumeration relies on.  Brute force in
+    fp64 over random values, scales from far narrower to wider than a step of the first grid, values in and out of range."""
+    rng = np.random.default_rng(77)
+    n = 60_000
+    a1 = rng.uniform(0.05, 2.0, n)
+    rho = np.exp(rng.uniform(np.log(0.004), np.log(3.0), n))
+    a2 = a1 * rho
+    x = rng.uniform(-1.6, 1.6, n) * a1 * max(hi1, -lo1)
+    half = max(hi2, -lo2) + 0.5
+
+    def err(t):
+        r = x - a1 * t
+        q = np.clip(np.rint(r / a2), lo2, hi2)
+        return np.abs(r - a2 * q)
+
+    full = np.min(np.stack([err(np.full(n, float(t))) for t in range(lo1, hi1 + 1)]), axis=0)
+    w = np.maximum(1, np.floor(half * np.minimum(rho, 16.0) * 1.0001 + 0.501)).astype(int)
+    t0 = np.rint(x / a1)
+    win = np.full(n, np.inf)
+    for s in range(-int(w.max()), int(w.max()) + 1):
+        t = np.clip(t0 + s, lo1, hi1)
+        e = np.where(np.abs(s) <= w, err(t), np.inf)
+        win = np.minimum(win, e)
+    assert np.all(win >= full)                       # a subset cannot do better
+    assert np.allclose(win, full, rtol=0, atol=1e-12)

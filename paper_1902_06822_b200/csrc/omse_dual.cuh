@@ -19,8 +19,8 @@
 
 namespace omse {
 
-constexpr int kDualDpt = 4;        // alpha2 candidates per thread
-constexpr int kDualThreads = 256;
+constexpr int kDualDpt = 8;        // alpha2 candidates per thread
+constexpr int kDualThreads = 128;
 constexpr int kDualListCap = 256;  // near-minimal pairs listed at a time for re-scoring with the full enumeration
 
 struct DualArgs {

@@ -135,7 +135,7 @@ __global__ void __launch_bounds__(kDualThreads) dual_kernel(const DualArgs a) {
                     const int w = max(1, (int)(half_range2 * fminf(ratio, 16.f) * 1.0001f + 0.501f));
                     const bool full = !(ratio <= 16.f) || 2 * w + 1 >= n_levels;
                     const int n_t = full ? n_levels : 2 * w + 1;
-                    ev += (unsigned long long)k * (unsigned long long)(2 * ((n_t + 1) / 2)) * kDualDpt;
+                    ev += (unsigned long long)k * (unsigned long long)n_t * kDualDpt;
                     const float clo2 = kMagic + flo2, chi2 = kMagic + fhi2, flo1 = (float)a.lo1, fhi1 = (float)a.hi1;
                     for (int i = 0; i < k; ++i) {
                         const float x = xs[i];
@@ -145,19 +145,19 @@ __global__ void __launch_bounds__(kDualThreads) dual_kernel(const DualArgs a) {
                         float best[kDualDpt];
 #pragma unroll
                         for (int j = 0; j < kDualDpt; ++j) best[j] = INFINITY;
-                        // two first codes per step (the second clamps to the last one when n_t is odd: a repeat
-                        // cannot change a minimum): eight independent chains in flight
-                        for (int s = 0; s < n_t; s += 2) {
-                            const float ta = fminf(fmaxf(t0 + (float)s, flo1), fhi1);
-                            const float tb = fminf(fmaxf(t0 + (float)min(s + 1, n_t - 1), flo1), fhi1);
-                            const float ra = fmaf(-a1, ta, x), rb = fmaf(-a1, tb, x);
+                        // one first code per step: the thread's alpha2's give independent chains, and a window
+                        // always holds an odd number of codes
+                        float tcur = t0;
+                        for (int s = 0; s < n_t; ++s) {
+                            const float ta = fminf(fmaxf(tcur, flo1), fhi1);
+                            tcur += 1.0f;
+                            const float ra = fmaf(-a1, ta, x);
 #pragma unroll
                             for (int j = 0; j < kDualDpt; ++j) {
-                                float ua = fmaf(ra, inv2[j], kMagic), ub = fmaf(rb, inv2[j], kMagic);
+                                float ua = fmaf(ra, inv2[j], kMagic);
                                 ua = fminf(fmaxf(ua, clo2), chi2);
-                                ub = fminf(fmaxf(ub, clo2), chi2);
-                                const float ea = fmaf(-a2[j], ua - kMagic, ra), eb = fmaf(-a2[j], ub - kMagic, rb);
-                                best[j] = fminf(best[j], fminf(fabsf(ea), fabsf(eb)));
+                                const float ea = fmaf(-a2[j], ua - kMagic, ra);
+                                best[j] = fminf(best[j], fabsf(ea));
                             }
                         }
 #pragma unroll

@@ -258,6 +258,16 @@ def test_long_rows_regrouped_for_every_candidate_layout(gpu, n_cand):
     _run_and_check(gpu, w, 3, True, n_cand, 2, codes=True, packed=False)
 
 
+@pytest.mark.parametrize("k", [1025, 1026, 1027, 2051, 8193, 8195, 14001])
+def test_long_rows_of_ragged_length(gpu, k):
+    """Block-per-row path on rows whose length is not a multiple of four: the per-element passes walk the row four
+    elements at a time and rely on its zero padding; both block sizes (rows below and above 8192 elements)."""
+    s = 7
+    w = synth.student_t3(s * k, seed=410, tensor_id=k).reshape(s, k)
+    _run_and_check(gpu, w, 4, True, 1024, 3, codes=True, packed=True)
+    _run_and_check(gpu, np.abs(w), 3, False, 256, 1, codes=True, packed=True)
+
+
 @pytest.mark.parametrize("k", [192, 193, 256, 500, 640])
 def test_short_rows_regrouped_in_large_launches(gpu, k):
     """Enough short rows for the batched short-row path, with regrouping (192 <= K <= 640)."""

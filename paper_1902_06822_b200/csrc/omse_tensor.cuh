@@ -95,37 +95,37 @@ __global__ void __launch_bounds__(256) tensor_absmax_kernel(const float* __restr
                                                              unsigned int* tile_flags, int flag_words) {
     __shared__ double scratch[64];
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < flag_words; i += gridDim.x * blockDim.x) tile_flags[i] = 0u;
-    float mpos = 0.f, mneg = 0.f, lo = INFINITY, hi = -INFINITY;
+    float lo = INFINITY, hi = -INFINITY;          // extremes of the finite values this thread saw
     bool bad = false;
     const long long n4 = n >> 2;
     const float4* x4 = reinterpret_cast<const float4*>(x);
     const long long stride = (long long)gridDim.x * blockDim.x;
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
-        const float4 v = __ldg(x4 + i);
-        const float e[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            if (fabsf(e[j]) <= FLT_MAX) {
-                mpos = fmaxf(mpos, e[j]);
-                mneg = fmaxf(mneg, -e[j]);
-                lo = fminf(lo, e[j]);
-                hi = fmaxf(hi, e[j]);
-            } else {
-                bad = true;
-            }
-        }
+    auto one = [&](float e) {
+        const bool finite = fabsf(e) <= FLT_MAX;
+        bad |= !finite;
+        lo = fminf(lo, finite ? e : lo);
+        hi = fmaxf(hi, finite ? e : hi);
+    };
+    auto four = [&](const float4& v) {
+        one(v.x);
+        one(v.y);
+        one(v.z);
+        one(v.w);
+    };
+    // four 128-bit loads in flight per thread before any of them is used
+    long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    for (; i + 3 * stride < n4; i += 4 * stride) {
+        const float4 v0 = __ldg(x4 + i), v1 = __ldg(x4 + i + stride), v2 = __ldg(x4 + i + 2 * stride),
+                     v3 = __ldg(x4 + i + 3 * stride);
+        four(v0);
+        four(v1);
+        four(v2);
+        four(v3);
     }
-    for (long long i = (n4 << 2) + (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) {
-        const float v = x[i];
-        if (fabsf(v) <= FLT_MAX) {
-            mpos = fmaxf(mpos, v);
-            mneg = fmaxf(mneg, -v);
-            lo = fminf(lo, v);
-            hi = fmaxf(hi, v);
-        } else {
-            bad = true;
-        }
-    }
+    for (; i < n4; i += stride) four(__ldg(x4 + i));
+    for (long long e = (n4 << 2) + (long long)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += stride) one(x[e]);
+    // maxima of the positive and of the negative part follow from the extremes (both 0 when nothing finite was seen)
+    float mpos = fmaxf(hi, 0.f), mneg = fmaxf(-lo, 0.f);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));

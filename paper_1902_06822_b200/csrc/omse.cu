@@ -45,7 +45,8 @@ constexpr int kMaxSmem = 231424;              // dynamic shared memory per block
 struct Workspace {
     unsigned int status;
     unsigned int pad_[3];
-    unsigned long long ticket[2];   // work-unit dispenser of the row kernels (self-resetting)
+    unsigned long long ticket[4];   // work-unit dispensers of the row kernels (self-resetting): a pair for launches on the
+                                    // context's stream, a pair for the launch that runs beside them on the side stream
     unsigned long long evals;       // executed evaluations since the last omse_read_evaluations
     omse::TensorState tstate;
     double curve[OMSE_MAX_CANDIDATES];
@@ -59,6 +60,9 @@ struct LaunchShape { int cpt, threads; size_t smem; int occ; };
 struct omse_ctx {
     int device;
     cudaStream_t stream;
+    cudaStream_t side;                 // second launch of a batched call runs here, beside the first (fork and join by events)
+    cudaEvent_t ev_fork, ev_join;
+    int ticket_pair;                   // which dispenser pair the next row launch uses
     int n_sm;
     Workspace* ws;       // device
     double* partials;    // device, kPartialBytes
@@ -171,7 +175,7 @@ int launch_rows(omse_ctx* ctx, omse::RowArgs& a, long long max_k, size_t smem_sm
     size_t smem = smem_for(a.groups);
     if (smem > (size_t)kMaxSmem) return OMSE_EINVAL;
     if (smem_small > smem) smem = smem_small;
-    a.ticket = ctx->ws->ticket;
+    a.ticket = ctx->ws->ticket + 2 * ctx->ticket_pair;
     a.status = &ctx->ws->status;
     a.evals = &ctx->ws->evals;
     // the extended kernel only where a launch needs what it adds
@@ -393,8 +397,11 @@ int quantize_list(omse_ctx* ctx, std::vector<omse::RowTensor>& list, long long m
         const int cpt = cpt_for(grid->n_cand);
         const int ncs = cpt * group_threads(grid->n_cand);
         long long units_if_small = 0;
+        // rows per work unit of the short-row path: eight rows of up to 128 elements amortise the unit's fixed costs,
+        // but only a tensor with many rows has enough units left for an even finish; otherwise four
+        auto small_batch = [&](const omse::RowTensor& t) { return (t.K <= 128 && t.S >= 16ll * ctx->n_sm) ? 8 : 4; };
         for (const auto& t : list) {
-            const int b = t.K > OMSE_SMALL_K ? t.rows_per_unit : (t.K <= 128 ? 8 : 4);
+            const int b = t.K > OMSE_SMALL_K ? t.rows_per_unit : small_batch(t);
             units_if_small += (t.S + b - 1) / b;
         }
         // very short rows in large numbers: a thread per row, a block-sized batch of rows per unit
@@ -412,7 +419,7 @@ int quantize_list(omse_ctx* ctx, std::vector<omse::RowTensor>& list, long long m
                 if (t.K > OMSE_SMALL_K || t.small) continue;
                 const bool prune = OMSE_PRUNE && t.K >= OMSE_SMALL_PRUNE_K;
                 t.small = prune ? 3 : 1;
-                t.rows_per_unit = t.K <= 128 ? 8 : 4;
+                t.rows_per_unit = small_batch(t);
                 const size_t kpad = (size_t)((t.K + 3) & ~3ll);
                 // per row: the row, its error curve, its grid; when regrouping also skipped sums, class table, regrouped row
                 const size_t need = (size_t)t.rows_per_unit *
@@ -426,8 +433,19 @@ int quantize_list(omse_ctx* ctx, std::vector<omse::RowTensor>& list, long long m
     // then runs the kernel instantiation that holds only its path.  Longest rows first inside a launch: the dispenser
     // hands out work in decreasing size and the tail is short.
     std::stable_sort(list.begin(), list.end(), [](const omse::RowTensor& x, const omse::RowTensor& y) { return x.K > y.K; });
+    // With both long and short rows in the list, the launch of the short rows goes first, on the side stream (forked
+    // from and joined to the context's stream by events, with its own work dispenser), and the long rows' launch runs
+    // beside it: the blocks of the second fill the SMs as the blocks of the first run out of work, so only one tail
+    // is left.  The two launches touch different tensors.
+    int present = 0;
+    for (const auto& t : list) present |= (t.small & 4) ? 4 : t.small ? 2 : 1;
+    const bool beside = (present & 2) && (present & 5);
+    bool forked = false;
     size_t desc_used = 0;
-    for (int path = 1; path <= 4; path <<= 1) {
+    const int path_order[3] = {2, 1, 4};
+    int rc_all = OMSE_OK;
+    for (int pi = 0; pi < 3 && rc_all == OMSE_OK; ++pi) {
+        const int path = path_order[pi];
         std::vector<omse::RowTensor> sub;
         long long sub_max_k = 0;
         for (const auto& t : list) {
@@ -453,8 +471,10 @@ int quantize_list(omse_ctx* ctx, std::vector<omse::RowTensor>& list, long long m
         } else {
             omse::RowTensor* d_sub = ctx->d_tensors + desc_used;
             if (cudaMemcpyAsync(d_sub, sub.data(), sizeof(omse::RowTensor) * sub.size(), cudaMemcpyHostToDevice,
-                                ctx->stream) != cudaSuccess)
-                return OMSE_ECUDA;
+                                ctx->stream) != cudaSuccess) {
+                rc_all = OMSE_ECUDA;
+                break;
+            }
             a.tensors = d_sub;
             desc_used += sub.size();
         }
@@ -470,10 +490,28 @@ int quantize_list(omse_ctx* ctx, std::vector<omse::RowTensor>& list, long long m
         a.off_frac = mode.off_frac;
         a.eps = -1.f;
         a.keep_x0 = mode.n_delta > 0 ? 1 : 0;   // every offset is applied to the original row
-        const int rc = launch_rows(ctx, a, sub_max_k, path == 1 ? 0 : smem_small, path);
-        if (rc != OMSE_OK) return rc;
+        const bool on_side = beside && path == 2;
+        cudaStream_t own = ctx->stream;
+        if (on_side) {
+            if (cudaEventRecord(ctx->ev_fork, own) != cudaSuccess || cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) != cudaSuccess) {
+                rc_all = OMSE_ECUDA;
+                break;
+            }
+            forked = true;
+            ctx->stream = ctx->side;
+            ctx->ticket_pair = 1;
+        }
+        rc_all = launch_rows(ctx, a, sub_max_k, path == 1 ? 0 : smem_small, path);
+        if (on_side) {
+            ctx->stream = own;
+            ctx->ticket_pair = 0;
+        }
     }
-    return OMSE_OK;
+    if (forked) {   // the side stream always rejoins, also after an error
+        if (cudaEventRecord(ctx->ev_join, ctx->side) != cudaSuccess || cudaStreamWaitEvent(ctx->stream, ctx->ev_join, 0) != cudaSuccess)
+            rc_all = rc_all == OMSE_OK ? OMSE_ECUDA : rc_all;
+    }
+    return rc_all;
 }
 
 }  // namespace
@@ -521,11 +559,17 @@ int omse_create(omse_ctx** out, int device, void* cuda_stream) {
         cudaGetLastError();
         return OMSE_ENOMEM;
     }
-    if (cudaMemsetAsync(c->ws, 0, sizeof(Workspace), c->stream) != cudaSuccess) {
+    if (cudaMemsetAsync(c->ws, 0, sizeof(Workspace), c->stream) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+        if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+        if (c->side) cudaStreamDestroy(c->side);
         cudaFree(c->ws);
         cudaFree(c->partials);
         cudaFree(c->d_tensors);
         delete c;
+        cudaGetLastError();
         return OMSE_ECUDA;
     }
     *out = c;
@@ -536,6 +580,10 @@ int omse_destroy(omse_ctx* ctx) {
     if (!ctx) return OMSE_EINVAL;
     DeviceScope dev(ctx->device);
     cudaStreamSynchronize(ctx->stream);
+    cudaStreamSynchronize(ctx->side);
+    cudaEventDestroy(ctx->ev_fork);
+    cudaEventDestroy(ctx->ev_join);
+    cudaStreamDestroy(ctx->side);
     cudaFree(ctx->ws);
     cudaFree(ctx->partials);
     cudaFree(ctx->d_tensors);

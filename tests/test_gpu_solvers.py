@@ -251,3 +251,39 @@ def test_launch_counter_counts_one_launch_per_row_path():
     ctx.omse_activation_scale(x, x.numel(), 4, False, 2048, 1.0, 3, a, e)
     assert ctx.omse_read_launches() == 11          # init, maxima, two sweeps, curve, argmin, re-score, 3 polish steps, final
     torch.cuda.synchronize()
+
+
+def test_back_to_back_batched_calls_with_two_row_paths_stay_ordered_and_reproducible():
+    """A list with long and short rows runs its two launches beside each other (second stream inside the call).  Many
+    such calls queued without a synchronisation in between, interleaved with per-tensor searches and single-path calls
+    on the same context, must give the same bits every time, and the values of the oracle."""
+    import torch
+    import gpu_util
+    ctx = gpu_util.ctx()
+    shapes = [(700, 64), (900, 147), (600, 576), (50, 1152), (24, 4608), (12000, 27)]   # short, long and very short rows
+    ws = [synth.student_t3(s * k, seed=9, tensor_id=i).reshape(s, k) for i, (s, k) in enumerate(shapes)]
+    x = torch.from_numpy(synth.relu_activations(300_000, seed=5)).cuda()
+    a_x, e_x = torch.empty(1, device="cuda"), torch.empty(1, device="cuda")
+    ctx.omse_last_device_status()                    # clears the sticky status word
+    rounds = []
+    for it in range(12):
+        descs = [dict(w=torch.from_numpy(w).cuda(), n_kernels=w.shape[0], kernel_len=w.shape[1],
+                      alpha=torch.empty(w.shape[0], device="cuda"), sse=torch.empty(w.shape[0], device="cuda"),
+                      packed=torch.empty((w.size + 1) // 2, dtype=torch.uint8, device="cuda")) for w in ws]
+        ctx.omse_quantize_weights_batched(descs, 4, True, 1024, 1.0, 3)
+        if it % 3 == 0:
+            ctx.omse_activation_scale(x, x.numel(), 4, False, 2048, 1.0, 3, a_x, e_x)
+        if it % 4 == 1:
+            ctx.omse_quantize_weights_batched(descs[3:5], 4, True, 1024, 1.0, 3)     # long rows only: one launch
+        rounds.append(descs)
+    torch.cuda.synchronize()
+    assert ctx.omse_last_device_status() == 0
+    for descs in rounds[1:]:
+        for d, d0 in zip(descs, rounds[0]):
+            assert torch.equal(d["alpha"], d0["alpha"]) and torch.equal(d["sse"], d0["sse"])
+            assert torch.equal(d["packed"], d0["packed"])
+    for w, d in zip(ws, rounds[-1]):
+        rows = np.arange(0, w.shape[0], max(1, w.shape[0] // 40))
+        ref = orc.quantize_rows(np.ascontiguousarray(w[rows]), 4, True, 1024, 1.0, 3)
+        np.testing.assert_allclose(d["alpha"].cpu().numpy()[rows], ref.alpha, rtol=1e-5)
+        np.testing.assert_allclose(d["sse"].cpu().numpy()[rows], ref.sse, rtol=1e-5)

@@ -315,11 +315,12 @@ int enqueue_tensor_search(const TensorEnv& env, omse::TensorArgs& a, int refine_
     const int kFine = 256;        // candidates of the first launch: 32 per slot
     int split = a.n_cand, nb_lo = 1, nb_hi = 1;
     if (n > 0) {
-        // Two sweep launches share tile flags when they fit: a bit per 4,096-element tile in the (not yet used)
-        // curve buffer, and the first launch's per-block squared sums in the (not yet used) candidate list.
-        const long long flag_tile4 = 4 * 256;                       // tile of the first sweep launch
-        const long long n_flag_tiles = (((n + 3) >> 2) + flag_tile4 - 1) / flag_tile4;
+        // Two sweep launches share tile flags when they fit: a bit per tile of the SECOND launch in the (not yet
+        // used) curve buffer, and the first launch's per-block squared sums in the (not yet used) candidate list.
         const bool two = a.n_cand > kFine;
+        const int hi_tg = two ? ((((a.n_cand - kFine) + 7) / 8) + 31) & ~31 : 32;
+        const long long flag_tile4 = 4ll * (256 / hi_tg < 1 ? 1 : 256 / hi_tg) * hi_tg;   // as sweep_launch sizes it
+        const long long n_flag_tiles = (((n + 3) >> 2) + flag_tile4 - 1) / flag_tile4;
         // curve: n_cand doubles = 64*n_cand bits; list: n_cand/2 doubles, enough for three blocks per SM
         const bool flags = two && n_flag_tiles <= 64ll * a.n_cand && a.n_cand / 2 >= 3 * env.n_sm;
         const int flag_words = flags ? (int)((n_flag_tiles + 31) >> 5) : 0;

@@ -23,6 +23,9 @@ struct TensorState {          // lives in the context workspace
     float delta;                         // offset subtracted from every element (0 without offset)
 };
 
+constexpr int kTileListCap = 32;   // flagged tiles one block of the second sweep launch lists for itself (static shared
+                                   // memory of that kernel must stay below the 1 KB left beside the dynamic maximum)
+
 struct TensorArgs {
     const float* x;
     long long n;
@@ -214,24 +217,69 @@ __global__ void __launch_bounds__(512) tensor_sweep_kernel(const TensorArgs a) {
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
-    // With tile flags from the first launch only the tiles that hold a value for this launch are read at all.
+    // With tile flags from the first launch only the tiles that hold a value for this launch are read at all (a flag
+    // tile is a tile of this launch).  The flagged tiles are dealt out evenly: the tile of rank r among the set bits
+    // goes to block r mod gridDim.x, listed once per block by its first warp (fixed order).  When more than half of
+    // the tiles are flagged (the strided sequences are then even enough) or more than the lists hold, every block
+    // walks its strided sequence and skips the unflagged tiles instead.
     const bool flagged_only = a.flag_role == 2 && a.tile_flags != nullptr;
-    auto next_tile = [&](long long tl) {             // first tile >= tl of this block's sequence that has to be read
-        if (!flagged_only) return tl;
-        for (; tl < n_tiles; tl += gridDim.x) {
-            const long long f0 = (tl * a.tile4) / a.flag_tile4;
-            const long long f1 = (min((tl + 1) * (long long)a.tile4, n4_total) - 1) / a.flag_tile4;
-            bool hit = false;
-            for (long long f = f0; f <= f1; ++f) hit |= (__ldg(a.tile_flags + (f >> 5)) >> (f & 31)) & 1u;
-            if (hit) break;
+    __shared__ int s_tiles[kTileListCap];
+    __shared__ int s_n_mine;
+    if (flagged_only) {
+        if (warp == 0) {
+            int total = 0;
+            for (int wi = lane; wi < a.flag_words; wi += 32) total += __popc(__ldg(a.tile_flags + wi));
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+            int n_mine = -1;
+            if ((long long)total <= (long long)kTileListCap * gridDim.x && 2ll * total <= n_tiles) {
+                n_mine = 0;
+                int running = 0;                      // set bits in the words before this group of 32
+                for (int w0 = 0; w0 < a.flag_words; w0 += 32) {
+                    const int wi = w0 + lane;
+                    const unsigned int word = wi < a.flag_words ? __ldg(a.tile_flags + wi) : 0u;
+                    const int cnt = __popc(word);
+                    int incl = cnt;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const int u = __shfl_up_sync(0xffffffffu, incl, o);
+                        if (lane >= o) incl += u;
+                    }
+                    int r = running + incl - cnt;     // rank of this word's first set bit
+                    unsigned int mine = 0u;
+                    for (unsigned int m2 = word; m2; m2 &= m2 - 1, ++r)
+                        if (r % (int)gridDim.x == (int)blockIdx.x) mine |= m2 & (0u - m2);
+                    const int mcnt = __popc(mine);
+                    int mincl = mcnt;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const int u = __shfl_up_sync(0xffffffffu, mincl, o);
+                        if (lane >= o) mincl += u;
+                    }
+                    int pos = n_mine + mincl - mcnt;
+                    for (unsigned int m2 = mine; m2; m2 &= m2 - 1) s_tiles[pos++] = wi * 32 + (__ffs(m2) - 1);
+                    n_mine += __shfl_sync(0xffffffffu, mincl, 31);
+                    running += __shfl_sync(0xffffffffu, incl, 31);
+                }
+            }
+            if (lane == 0) s_n_mine = n_mine;
         }
+        __syncthreads();
+    }
+    const int n_mine = flagged_only ? s_n_mine : -1;   // >= 0: this block's tiles are s_tiles[0 .. n_mine)
+    auto next_tile = [&](long long tl) {             // first tile >= tl of this block's strided sequence that has to be read
+        if (!flagged_only) return tl;
+        for (; tl < n_tiles; tl += gridDim.x)
+            if ((__ldg(a.tile_flags + (tl >> 5)) >> (tl & 31)) & 1u) break;
         return tl;
     };
-    long long tl = next_tile(blockIdx.x);
+    int sidx = 0;
+    long long tl = n_mine >= 0 ? (n_mine > 0 ? (long long)s_tiles[0] : n_tiles) : next_tile(blockIdx.x);
     if (tl < n_tiles) prefetch(tl);
     while (tl < n_tiles) {
         const long long base4 = tl * a.tile4;
-        const long long tl_next = next_tile(tl + gridDim.x);
+        ++sidx;
+        const long long tl_next = n_mine >= 0 ? (sidx < n_mine ? (long long)s_tiles[sidx] : n_tiles) : next_tile(tl + gridDim.x);
         asm volatile("cp.async.wait_all;" ::: "memory");
         // ---- this thread's span into registers (elements past the end count as zeros)
         float vals[16];
@@ -543,7 +591,8 @@ __global__ void __launch_bounds__(256) tensor_sweep_fine_kernel(const TensorArgs
         }
         sq_all += tot;
         if (flagging && __any_sync(0xffffffffu, far) && lane == 0) {
-            const long long ft = base4 / a.flag_tile4;             // this launch's tiles are the flag tiles
+            // a flag tile is a tile of the second launch: a multiple of 128 float4s, so a warp's 128 float4s lie in one
+            const long long ft = (base4 + warp * 128) / a.flag_tile4;
             atomicOr(a.tile_flags + (ft >> 5), 1u << (ft & 31));
         }
         __syncwarp();                                 // the warp is done sweeping its previous share

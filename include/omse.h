@@ -20,8 +20,7 @@
  *     except omse_last_device_status(), omse_read_evaluations() and omse_destroy().  A call
  *     whose list holds both long and short kernels runs one of its two launches on a second
  *     stream that the context owns, forked from the context's stream and joined back to it by
- *     events inside the call: for the caller everything stays ordered on the context's stream
- *     (the pattern is also valid under stream capture).
+ *     events inside the call: for the caller everything stays ordered on the context's stream.
  *   - All work queued through one context shares that context's device workspace (work-unit
  *     dispenser, search state, partial sums).  It must therefore be stream-ordered: after
  *     omse_set_stream() the caller makes the new stream wait for the work already queued on the

@@ -36,7 +36,7 @@ LANE_OPS_PER_EVAL = 4         # FMA-pipe lane operations of an evaluation the ke
 # dram__bytes_read.sum + dram__bytes_write.sum of one step of the default workload (its two launches of the row kernel:
 # rows of up to 640 elements, and the longer ones beside them) from an ncu capture; None whenever the kernels have changed
 # since the capture
-NCU_TRAFFIC_BYTES = 106_045_184
+NCU_TRAFFIC_BYTES = 105_624_064
 E2E_CHUNKS = 12               # batched launches per end-to-end step (copies of later chunks overlap earlier searches)
 N_SM, LANES_PER_SM = 148, 128
 WORKLOAD = "resnet50_weight_set_54_tensors_25.5M_params_signed4bit_kernelwise_1024cand_3refine_packed"

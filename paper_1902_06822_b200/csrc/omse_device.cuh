@@ -195,6 +195,7 @@ __device__ __forceinline__ void sweep_dispatch(int nact, int ncl, const float4* 
         case 2: if constexpr (CPT >= 2) sweep_ncl<CPT, 2>(ncl, xs4, beg4, end4, inv2, na2, dacc, clo, chi); break;
         case 3: if constexpr (CPT >= 4) sweep_ncl<CPT, 3>(ncl, xs4, beg4, end4, inv2, na2, dacc, clo, chi); break;
         case 4: if constexpr (CPT >= 4) sweep_ncl<CPT, 4>(ncl, xs4, beg4, end4, inv2, na2, dacc, clo, chi); break;
+        case 5: if constexpr (CPT >= 8) sweep_ncl<CPT, 5>(ncl, xs4, beg4, end4, inv2, na2, dacc, clo, chi); break;
         case 6: if constexpr (CPT >= 8) sweep_ncl<CPT, 6>(ncl, xs4, beg4, end4, inv2, na2, dacc, clo, chi); break;
         default: sweep_ncl<CPT, CPT>(ncl, xs4, beg4, end4, inv2, na2, dacc, clo, chi); break;
     }
@@ -273,6 +274,7 @@ __device__ __forceinline__ void sweep_accum_dispatch(int nact, int ncl, const fl
         case 2: if constexpr (CPT >= 2) sweep_accum_ncl<CPT, 2>(ncl, xs4, beg4, end4, inv2, na2, acc2, clo, chi); break;
         case 3: if constexpr (CPT >= 4) sweep_accum_ncl<CPT, 3>(ncl, xs4, beg4, end4, inv2, na2, acc2, clo, chi); break;
         case 4: if constexpr (CPT >= 4) sweep_accum_ncl<CPT, 4>(ncl, xs4, beg4, end4, inv2, na2, acc2, clo, chi); break;
+        case 5: if constexpr (CPT >= 8) sweep_accum_ncl<CPT, 5>(ncl, xs4, beg4, end4, inv2, na2, acc2, clo, chi); break;
         case 6: if constexpr (CPT >= 8) sweep_accum_ncl<CPT, 6>(ncl, xs4, beg4, end4, inv2, na2, acc2, clo, chi); break;
         default: sweep_accum_ncl<CPT, CPT>(ncl, xs4, beg4, end4, inv2, na2, acc2, clo, chi); break;
     }
@@ -381,7 +383,7 @@ __device__ __forceinline__ int magnitude_class(float x, float inv_thr, float inv
     if (r <= 1.0f) return 0;
     const float f = (r - 1.0f) * inv_tg;       // slot sl needs x iff r > sl*tg + 1
     int nb = f >= (float)CPT ? CPT : (int)f + 1;
-    if (CPT == 8 && (nb == 5 || nb == 7)) ++nb;   // classes 5 and 7 are merged upwards: fewer sweep variants
+    if (CPT == 8 && nb == 7) ++nb;   // class 7 is merged upwards: fewer sweep variants (a class 5 of its own pays, a class 7 does not)
     return nb;
 }
 
